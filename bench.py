@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the MiLoRA adapter path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c2]
+
+One step = one pass of the whole hot path over one batch of the LLaMA-2-7B single-layer workload:
+route the 64 prompts (router kernel), group the prompt tokens, apply the routed adapters on all
+prompt tokens at the 7 module call sites (prefill kernel), group the 64 decode tokens, apply the
+adapters on them at the 7 call sites (decode kernel).  Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = ("decode adapter-apply tokens/s and HBM GB/s vs 8 TB/s peak; prefill TFLOP/s; router us/prompt "
+          "[value = adapter-apply token-layers/s over the whole step: route + group + prefill apply + decode apply]")
+UNIT = "token-layers/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons = [], [], set()
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); smax.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# workload + algorithmic work
+# ------------------------------------------------------------------------------------------------
+def algorithmic_work(w, routes_col, prefill_ids, decode_ids):
+    """Bytes and flops the method must move for one step at one layer (host arithmetic on the route table).
+
+    router : e*n_p*d (H) + e*7*d (W_r) per prompt
+    prefill: per routed prompt  e*L*(d1 + 2*d2) + e*r*(d1+d2);  flops 2*L*r*(d1+d2)
+    decode : per distinct (tenant, module) e*r*(d1+d2); per token e*d1 + 2*e*d2; flops 2*r*(d1+d2) per token
+    """
+    e, r = w.elem_bytes, w.rank
+    out = {"router_bytes": 0, "prefill_bytes": 0, "prefill_flops": 0, "decode_bytes": 0, "decode_flops": 0}
+    for i in prefill_ids:
+        L = int(w.prompt_len[i])
+        out["router_bytes"] += e * L * w.d_model + e * 7 * w.d_model
+        m = int(routes_col[i])
+        if m < 0:
+            continue
+        d1, d2 = w.dims(m)
+        out["prefill_bytes"] += e * L * (d1 + 2 * d2) + e * r * (d1 + d2)
+        out["prefill_flops"] += 2 * L * r * (d1 + d2)
+    seen = set()
+    for i in decode_ids:
+        m = int(routes_col[i])
+        if m < 0:
+            continue
+        d1, d2 = w.dims(m)
+        key = (int(w.request_tenant[i]), m)
+        if key not in seen:
+            seen.add(key)
+            out["decode_bytes"] += e * r * (d1 + d2)
+        out["decode_bytes"] += e * d1 + 2 * e * d2
+        out["decode_flops"] += 2 * r * (d1 + d2)
+    out["decode_distinct_adapters"] = len(seen)
+    return out
+
+
+class Step:
+    """Device-resident inputs of one step and the sequence of library calls that make it."""
+
+    def __init__(self, lw, device):
+        w = lw.w
+        self.lw, self.w, self.device = lw, w, device
+        self.prefill_ids = [int(i) for i in w.prefill_ids]
+        self.decode_ids = [int(i) for i in w.decode_ids]
+        ml = lw.ml
+        self.H = w.hidden_batch(lw.layers[0], self.prefill_ids, device)
+        self.cu_p, self.slots_p, self.T_p = lw.seq_arrays(self.prefill_ids, [])
+        self.cu_d, self.slots_d, self.T_d = lw.seq_arrays([], self.decode_ids)
+        self.ws_p = ml.alloc_group_ws(1, len(self.prefill_ids), self.T_p)
+        self.ws_d = ml.alloc_group_ws(1, len(self.decode_ids), self.T_d)
+        self.g_p = ml.groups(self.ws_p[0], len(self.prefill_ids), self.T_p)
+        self.g_d = ml.groups(self.ws_d[0], len(self.decode_ids), self.T_d)
+        self.Xp, self.Yp, self.Xd, self.Yd = [], [], [], []
+        for m in range(7):
+            self.Xp.append(w.module_input(lw.layers[0], m, self.T_p, 0, device))
+            self.Yp.append(w.base_output(lw.layers[0], m, self.T_p, 0, device))
+            self.Xd.append(w.module_input(lw.layers[0], m, self.T_d, 1, device))
+            self.Yd.append(w.base_output(lw.layers[0], m, self.T_d, 1, device))
+        self.n_launches = 0
+
+    def run(self, ev=None):
+        """One pass of the path.  ev: optional list of 6 CUDA events recorded at the phase boundaries."""
+        ml = self.lw.ml
+        rec = (lambda i: ev[i].record()) if ev is not None else (lambda i: None)
+        rec(0)
+        ml.route(0, self.H, self.cu_p, self.slots_p)
+        rec(1)
+        ml.group(0, 1, self.cu_p, self.slots_p, len(self.prefill_ids), self.T_p, self.ws_p)
+        rec(2)
+        for m in range(7):
+            ml.apply_prefill(0, m, self.Xp[m], self.Yp[m], self.g_p)
+        rec(3)
+        ml.group(0, 1, self.cu_d, self.slots_d, len(self.decode_ids), self.T_d, self.ws_d)
+        rec(4)
+        for m in range(7):
+            ml.apply_decode(0, m, self.Xd[m], self.Yd[m], self.g_d)
+        rec(5)
+        self.n_launches = 1 + 1 + 7 + 1 + 7
+        return self.n_launches
+
+
+def run_ours(args, rank, world, device):
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth import get_workload
+
+    w = get_workload(args.config, seed=rank)          # weak scaling: every rank serves its own tenants' requests
+    lw = LoadedWorkload(w, device, layers=[0])
+    step = Step(lw, device)
+    tokens_per_step = step.T_p + step.T_d
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(device)
+
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+    barrier()
+    routes = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0]
+    work = algorithmic_work(w, routes, step.prefill_ids, step.decode_ids)
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        gpu_id = str(device.index or 0)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    launches = 0
+    for k in range(args.steps):
+        launches += step.run(evs[k])
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t0.elapsed_time(t1)
+    phase_ms = np.zeros(5)
+    for k in range(args.steps):
+        for i in range(5):
+            phase_ms[i] += evs[k][i].elapsed_time(evs[k][i + 1])
+    phase_ms /= args.steps
+    if world > 1:
+        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
+    e2e = run_e2e(step, args, world, device, tokens_per_step)
+
+    if rank != 0:
+        return None
+    peaks = load_peaks()
+    route_ms, gp_ms, prefill_ms, gd_ms, decode_ms = (float(v) for v in phase_ms)
+    shares = {"router": route_ms, "prefill_apply": prefill_ms, "decode_apply": decode_ms}
+    dom = max(shares, key=shares.get)
+    per_kernel = {
+        "router": {"ms": route_ms, "launches": 1, "bytes": work["router_bytes"]},
+        "prefill_apply": {"ms": prefill_ms, "launches": 7, "bytes": work["prefill_bytes"]},
+        "decode_apply": {"ms": decode_ms, "launches": 7, "bytes": work["decode_bytes"]},
+    }
+    rooflines = {}
+    for name, k in per_kernel.items():
+        gbs = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
+        rooflines[name] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                           "frac": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
+                           "peak_source": peaks["source"], "ms_per_step": k["ms"], "launches_per_step": k["launches"],
+                           "algorithmic_bytes_per_step": k["bytes"], "traffic": None}
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "note": w.note, "tokens_per_step": tokens_per_step, "prompts": len(step.prefill_ids),
+                   "decode_tokens": len(step.decode_ids), "rank": w.rank, "tenants": w.n_tenants,
+                   "l2": "inputs larger than L2: every step streams > 2 GB between two launches of the same kernel",
+                   "parallelism": f"requests sharded by tenant over {world} GPU(s), no collective"},
+        "breakdown": {
+            "decode_tokens_per_s": len(step.decode_ids) / (decode_ms * 1e-3),
+            "decode_gbs": rooflines["decode_apply"]["achieved"],
+            "decode_frac_of_8TBs": rooflines["decode_apply"]["frac_of_8TBs_nominal"],
+            "decode_distinct_adapters": work["decode_distinct_adapters"],
+            "prefill_tflops": work["prefill_flops"] / (prefill_ms * 1e-3) / 1e12,
+            "prefill_gbs": rooflines["prefill_apply"]["achieved"],
+            "prefill_frac_of_bf16_peak": work["prefill_flops"] / (prefill_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "router_us_per_prompt": route_ms * 1e3 / len(step.prefill_ids),
+            "router_gbs": rooflines["router"]["achieved"],
+            "group_prefill_us": gp_ms * 1e3, "group_decode_us": gd_ms * 1e3,
+        },
+        "roofline": dict(rooflines[dom], kernel=dom),
+        "rooflines": rooflines,
+        "e2e": e2e,
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    out["cpu_baseline"] = cpu_baseline(w, args)
+    return out
+
+
+def run_e2e(step, args, world, device, tokens_per_step):
+    """Same step, but every step's inputs start in pinned host memory and the outputs end there."""
+    steps = max(1, min(args.steps, 3))
+    host_in = [step.H] + step.Xp + step.Yp + step.Xd + step.Yd
+    pinned = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in host_in]
+    for p, t in zip(pinned, host_in):
+        p.copy_(t)
+    outs = step.Yp + step.Yd
+    pinned_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in outs)
+    torch.cuda.synchronize(device)
+    if world > 1:
+        torch.distributed.barrier()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        for p, t in zip(pinned, host_in):
+            t.copy_(p, non_blocking=True)
+        step.run()
+        for p, t in zip(pinned_out, outs):
+            p.copy_(t, non_blocking=True)
+    t1.record()
+    torch.cuda.synchronize(device)
+    ms = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_step = ms / steps
+    return {"value": world * tokens_per_step / (ms_step * 1e-3), "unit": UNIT, "ms_per_step": ms_step,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline, and the `--impl reference` arm)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_step(w, n_prompts):
+    """The oracle over a bounded sample of the step: n_prompts prompts routed and applied on all their
+    tokens, and the matching decode tokens.  Returns (token-layers processed, seconds)."""
+    from oracle import reference_run as R
+
+    ids = [int(i) for i in w.prefill_ids[:n_prompts]]
+    dec = [int(i) for i in w.decode_ids[:n_prompts]]
+    H = {i: w.hidden(0, i) for i in ids}
+    lens = [int(w.prompt_len[i]) for i in ids]
+    T_p = sum(lens)
+    token_slot_p = np.repeat(np.array(ids), lens)
+    Xp = [w.module_input(0, m, T_p, 0) for m in range(7)]
+    Yp = [w.base_output(0, m, T_p, 0) for m in range(7)]
+    Xd = [w.module_input(0, m, len(dec), 1) for m in range(7)]
+    Yd = [w.base_output(0, m, len(dec), 1) for m in range(7)]
+    t0 = time.perf_counter()
+    table = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+    R.route_requests(w, 0, ids, table, hidden=lambda i: H[i])
+    R.group_layer(w, token_slot_p, table[:, 0])
+    for m in range(7):
+        R.apply_site(w, 0, m, Xp[m], Yp[m], token_slot_p, table[:, 0])
+    if dec:
+        # decode requests of the sample need their routes as well (prompt already routed above when shared)
+        missing = [i for i in dec if table[i, 0] < 0]
+        if missing:
+            R.route_requests(w, 0, missing, table)
+        R.group_layer(w, np.array(dec), table[:, 0])
+        for m in range(7):
+            R.apply_site(w, 0, m, Xd[m], Yd[m], np.array(dec), table[:, 0])
+    dt = time.perf_counter() - t0
+    return T_p + len(dec), dt
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def cpu_baseline(w, args, n_prompts=16):
+    tokens, dt = oracle_sample_step(w, n_prompts)
+    return {"value": tokens / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": f"first {n_prompts} of {len(w.prefill_ids)} prompts (all their tokens) and the same "
+                      f"{n_prompts} decode requests: {tokens} token-layers in {dt:.2f} s, fp64 numpy",
+            "host_cpus": os.cpu_count()}
+
+
+def run_reference(args):
+    from synth import get_workload
+    w = get_workload(args.config, seed=0)
+    n_prompts = 2
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(w, n_prompts)
+    tot_tokens, tot_dt = 0, 0.0
+    for _ in range(args.steps):
+        tk, dt = oracle_sample_step(w, n_prompts)
+        tot_tokens += tk
+        tot_dt += dt
+    value = tot_tokens / tot_dt
+    sample = (f"each step = first {n_prompts} of {len(w.prefill_ids)} prompts (all their tokens) and the same "
+              f"{n_prompts} decode requests, fp64 numpy oracle on the host cores")
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": tot_dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "note": w.note, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the MiLoRA library has no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+    import __graft_entry__
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        torch.distributed.barrier()
+    out = run_ours(args, rank, world, device)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

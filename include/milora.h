@@ -1,0 +1,213 @@
+/*
+ * milora.h - C ABI of the MiLoRA adapter-apply library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the serving hot path of MiLoRA ("Mixture of Low-Rank
+ * Adaptation", prompt-aware routing):
+ *
+ *   - Section 3.3, Eq. 2-3: once per prompt and per Transformer layer, pool the prompt's
+ *     hidden states H^l, apply the activation g, multiply by the router weight W_r^l
+ *     (d x 7), softmax, and select the top-scoring of the 7 LoRA positions
+ *     q,k,v,o,gate,up,down.  The decision is stored in an int32 route table and reused
+ *     for every generated token of that request.
+ *   - Section 3.1, Eq. 1: x' = x W_m + s x W_m^A W_m^B + b_m is applied only on the selected
+ *     module m of each request.  The caller computes x W_m + b_m; the library adds the
+ *     LoRA term in place.
+ *   - Section 4.5 (efficiency analysis): adapters are not merged into the backbone, so one
+ *     batch mixes many tenants; tokens are bucketed by (module, tenant) first.
+ *
+ * Conventions
+ *   - Plain C.  Every function returns a milora_status (MILORA_OK = 0) and never aborts,
+ *     throws or exits.  Errors that the host can detect are reported before anything is
+ *     launched.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *     The caller owns every buffer it passes; the library borrows it until the work
+ *     enqueued by that call has finished on the stream.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device
+ *     work is enqueued on it and the call returns without waiting, except where stated.
+ *   - Matrices are dense row-major.  Element type of activations, adapters and router
+ *     weights is the context's dtype (fp32 or bf16); accumulation is always fp32.
+ *   - A context is not thread-safe; use one per host thread or lock around it.
+ *   - Device-side index problems (a slot id out of range inside a device array) never
+ *     fault: the offending item is skipped and a flag is raised that milora_poll_error reads.
+ */
+#ifndef MILORA_H_
+#define MILORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct milora_ctx milora_ctx;
+
+typedef enum {
+  MILORA_OK = 0,
+  MILORA_E_ARG = 1,          /* null pointer, negative size, index out of range            */
+  MILORA_E_SHAPE = 2,        /* dimension not supported (see milora_create)                 */
+  MILORA_E_DTYPE = 3,
+  MILORA_E_UNREGISTERED = 4, /* tenant / adapter / router / slot not registered             */
+  MILORA_E_CAPACITY = 5,     /* exceeds max_rank / max_tenants / max_requests / workspace   */
+  MILORA_E_STATE = 6,
+  MILORA_E_CUDA = 7,         /* a CUDA runtime call failed; see milora_last_cuda_error      */
+  MILORA_E_DEVICE_INDEX = 8  /* reported by milora_poll_error: a kernel skipped a bad index */
+} milora_status;
+
+typedef enum { MILORA_F32 = 0, MILORA_BF16 = 1 } milora_dtype;
+
+/* Section 3.3, Eq. 2: (b) average, (a) last-token, (c) max, (d) self-attention pooling (Appendix C). */
+typedef enum { MILORA_POOL_MEAN = 0, MILORA_POOL_LAST = 1, MILORA_POOL_MAX = 2, MILORA_POOL_SELFATTN = 3 } milora_pool;
+
+/* Activation g before the router (Section 3.3); RATIONAL is Eq. 7. */
+typedef enum { MILORA_ACT_TANH = 0, MILORA_ACT_IDENTITY = 1, MILORA_ACT_RELU = 2, MILORA_ACT_GELU = 3,
+               MILORA_ACT_RATIONAL = 4 } milora_act;
+
+/* Section 3.1: module order 0..6; N_mod = 7. */
+enum { MILORA_Q = 0, MILORA_K = 1, MILORA_V = 2, MILORA_O = 3, MILORA_GATE = 4, MILORA_UP = 5, MILORA_DOWN = 6,
+       MILORA_NMOD = 7 };
+
+enum { MILORA_MAX_RATIONAL_COEF = 16 };
+
+typedef struct {
+  int n_layers;
+  int d_model;      /* hidden size d; d_model, d_ff and d_kv must be multiples   */
+  int d_ff;         /* of 8 (bf16) or 4 (fp32) so that rows are 16-byte aligned, */
+  int d_kv;         /* else MILORA_E_SHAPE.  d_kv = output size of k and v.      */
+  milora_dtype dtype;
+  int max_rank;     /* largest LoRA rank that will be registered (1..256)       */
+  int max_tenants;
+  int max_requests; /* number of request slots (rows of the route table)        */
+} milora_model_desc;
+
+/* Create / destroy.  milora_create allocates the device tables (adapter table, router table,
+ * slot table, route table [max_requests][n_layers] initialised to -1) with cudaMalloc on the
+ * current device and waits for their initialisation.  milora_destroy frees everything the
+ * library allocated, including adapter copies. */
+milora_status milora_create(const milora_model_desc* desc, milora_ctx** out);
+milora_status milora_destroy(milora_ctx* ctx);
+const char* milora_status_string(milora_status s);
+/* Text of the last CUDA runtime error seen by this context ("" if none). */
+const char* milora_last_cuda_error(const milora_ctx* ctx);
+
+/* (d1, d2) of W_m for module m (Section 3.1): q,o d x d; k,v d x d_kv; gate,up d x d_ff; down d_ff x d. */
+milora_status milora_module_dims(const milora_ctx* ctx, int module, int* d1, int* d2);
+
+/* ---- adapter table (Eq. 1) ---------------------------------------------------------------
+ * Register W^A (A_dev: d1 x rank) and W^B (B_dev: rank x d2), in the paper's orientation, for
+ * (tenant, layer, module) with LoRA scale s (Eq. 1 is s = 1).  The library copies both into
+ * its own pool in its own layout (A transposed to rank x d1) on `stream`; the caller may free
+ * A_dev/B_dev once that stream work has finished.  Registering the same key again replaces it
+ * (the caller must make sure no apply call using the old copy is still running). */
+milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, int module, int rank, float scale,
+                                      const void* A_dev, const void* B_dev, void* stream);
+
+/* ---- router table (Eq. 2-3) --------------------------------------------------------------
+ * Register the router of (tenant, layer): Wr_dev is d x 7 (paper orientation, context dtype);
+ * bias_dev is 7 fp32 values or NULL (the paper prints no bias); Wsa_dev (d values, context
+ * dtype) is required only for MILORA_POOL_SELFATTN; coef_host holds a_0..a_{n_a-1} then
+ * b_1..b_{n_b} (host floats, n_a + n_b <= MILORA_MAX_RATIONAL_COEF) only for
+ * MILORA_ACT_RATIONAL.  Everything is copied on `stream`. */
+milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, const void* Wr_dev,
+                                     const float* bias_dev, milora_pool pool, const void* Wsa_dev, milora_act act,
+                                     const float* coef_host, int n_a, int n_b, void* stream);
+
+/* Drop every adapter and router of a tenant (host-side table update; takes effect for calls
+ * made afterwards).  Fails with MILORA_E_STATE while a request slot is bound to the tenant. */
+milora_status milora_unregister_tenant(milora_ctx* ctx, int tenant);
+
+/* ---- request slots -----------------------------------------------------------------------
+ * Bind a slot to a tenant when a request is admitted; release it when the request ends.
+ * Opening a slot resets its route row to -1 (not routed). */
+milora_status milora_request_open(milora_ctx* ctx, int slot, int tenant);
+milora_status milora_request_close(milora_ctx* ctx, int slot);
+
+/* ---- routing (Section 3.3, Eq. 2-3; computed once per prompt, then reused) ----------------
+ * Route P prompts at `layer`.  H_dev holds the prompts' hidden states back to back:
+ * rows [cu_seqlens[p], cu_seqlens[p+1]) of a [T_total, d_model] matrix belong to prompt p;
+ * T_total = cu_seqlens[P] must be passed by the host.  seq_slot_dev[p] is the request slot of
+ * prompt p (P <= 4096).  Writes route[slot][layer] (module id 0..6, ties to the lower index) and,
+ * when not NULL, logits_out_dev [P][7] fp32 (g(h) W_r + bias) and probs_out_dev [P][7] fp32 (their
+ * softmax).
+ * Prompts whose slot is closed or whose tenant has no router at this layer get route -1.
+ * One fused launch; deterministic (fixed reduction order).  The first call, and any call with more
+ * rows than every earlier one, grows an internal scratch buffer (cudaMalloc after a stream sync). */
+milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const int32_t* cu_seqlens_dev,
+                           const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
+                           float* probs_out_dev, void* stream);
+
+/* Device pointer to the route table, int32 [max_requests][n_layers], read-only for callers. */
+milora_status milora_route_table(const milora_ctx* ctx, const int32_t** table_dev);
+
+/* Copy route rows [slot_begin, slot_begin + n_slots) to / from host memory (n_slots * n_layers int32).
+ * Both wait for `stream` first and return when the copy is done.  Writing lets a caller restore
+ * decisions that were computed earlier (for example after moving a request to another replica);
+ * values must be -1 or 0..6. */
+milora_status milora_route_table_read(milora_ctx* ctx, int slot_begin, int n_slots, int32_t* rows_host, void* stream);
+milora_status milora_route_table_write(milora_ctx* ctx, int slot_begin, int n_slots, const int32_t* rows_host,
+                                       void* stream);
+
+/* ---- grouping (multi-tenant batches, Section 4.5) ------------------------------------------
+ * A step's tokens are n_seq sequences laid out back to back (rows [cu_seqlens[i], cu_seqlens[i+1])
+ * of every X / Y matrix; n_seq <= 4096); a decode request is a sequence of length 1 (cu_seqlens_dev
+ * == NULL means every sequence has length 1).  For layers [layer_begin, layer_begin + n_layers) the tokens are
+ * bucketed by key = route[slot][layer] * max_tenants + tenant(slot).  Sequences whose slot is
+ * closed, not routed, or whose tenant has no adapter on the routed module are excluded.
+ *
+ * Output: one int32 block per layer in ws_dev (block l at ws_dev + l * ws_stride), laid out as
+ * milora_group_layout describes:
+ *   header[16]     [0] n_seg  [1] n_excluded tokens  [2] n_active tokens  [3] n_tiles  [4] n_gather
+ *   mod_offset[8]  segment-index range of each module
+ *   seg_key[]      key of every non-empty bucket, ascending
+ *   seg_offset[]   bucket boundaries in perm
+ *   perm[]         active token rows ordered by (module, tenant, row)
+ * followed by the work lists the apply kernels consume (dense tiles of consecutive rows for
+ * long sequences; gathered rows for short ones). */
+typedef struct {
+  size_t header, mod_offset, mod_tile_offset, mod_gather_offset;
+  size_t seg_key, seg_offset, perm, tiles, gather_rows, gather;
+  size_t total;              /* int32 elements of one layer block (multiple of 4) */
+  int max_tiles, max_gather;
+} milora_group_layout_t;
+
+milora_status milora_group_layout(const milora_ctx* ctx, int n_seq, int T, milora_group_layout_t* out);
+
+milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const int32_t* cu_seqlens_dev,
+                           const int32_t* seq_slot_dev, int n_seq, int T, int32_t* ws_dev, size_t ws_stride,
+                           void* stream);
+
+/* One layer's group block, as written by milora_group with the same n_seq and T. */
+typedef struct {
+  const int32_t* ws_dev;
+  int n_seq;
+  int T;
+} milora_groups;
+
+/* ---- apply (Eq. 1 on the selected module) ------------------------------------------------
+ * X_dev [T][d1] inputs of module `module`; Y_dev [T][d2] holds x W_m + b_m on entry and
+ * x W_m + b_m + s (x W^A) W^B on exit for the rows whose request routes to `module` at `layer`;
+ * all other rows are left untouched (bit-identical).  milora_apply_decode processes the rows of
+ * short sequences (the gathered work list: decode tokens), milora_apply_prefill the rows of long
+ * sequences (dense tiles: prompt tokens); a mixed batch calls both. */
+milora_status milora_apply_decode(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
+                                  const milora_groups* groups, void* stream);
+milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
+                                   const milora_groups* groups, void* stream);
+
+/* Several module call sites of one layer in a single launch (for example q,k,v share an input,
+ * gate,up share an input).  modules[i], X_dev[i], Y_dev[i] describe site i; a module may appear once. */
+milora_status milora_apply_decode_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,
+                                        const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
+                                        void* stream);
+milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,
+                                         const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
+                                         void* stream);
+
+/* Waits for `stream`, then reads and clears the device error flag.  *device_flag_out is 0 when no
+ * kernel skipped anything; the return value is MILORA_E_DEVICE_INDEX otherwise. */
+milora_status milora_poll_error(milora_ctx* ctx, int* device_flag_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MILORA_H_ */

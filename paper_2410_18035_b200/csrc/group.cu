@@ -1,0 +1,275 @@
+// Token grouping for multi-tenant batches: bucket a step's tokens by (module, tenant) for one layer
+// and build the work lists of the apply kernels.
+//
+// A step is given as sequences of consecutive rows, and the key of a token depends only on its
+// sequence's request slot, so the sort runs over sequences (at most kMaxSeq), not over tokens:
+// one CTA per layer sorts the composite keys (key << 12 | sequence index), which are unique, with
+// a bitonic network in shared memory; equal keys then sit next to each other in sequence order,
+// which is row order.  Everything after that is prefix sums.  Integer work only; the result is
+// the same as a stable sort of the tokens by key.
+#include <climits>
+
+#include "milora_internal.h"
+
+namespace milora {
+namespace {
+
+constexpr int kGThreads = 1024;
+constexpr int kSeqBits = 12;  // kMaxSeq = 4096 sequences
+static_assert((1 << kSeqBits) == kMaxSeq, "kSeqBits must match kMaxSeq");
+
+// Exclusive prefix sum over the block of one int per thread; returns the exclusive value, *total gets the sum.
+__device__ inline int block_exscan(int v, int* total, int* wsum /* [33] */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = wsum[lane];
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    wsum[lane] = winc - w;
+    if (lane == 31) wsum[32] = winc;
+  }
+  __syncthreads();
+  *total = wsum[32];
+  return wsum[warp] + inc - v;
+}
+
+struct GroupArgs {
+  DeviceTables tab;
+  const int32_t* cu;        // may be null: every sequence has one row
+  const int32_t* seq_slot;
+  int32_t* ws;
+  size_t ws_stride;
+  milora_group_layout_t lay;
+  int layer_begin, n_seq, n_pad, T;
+};
+
+// Shared memory: comp[n_pad], tok_off[n_pad+1], seg_of[n_pad], seg_tile[n_pad+1], seg_short[n_pad+1],
+// seg_gather[n_pad+1].
+__global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
+  extern __shared__ int32_t sm[];
+  __shared__ int wsum[33];
+  const int n_pad = a.n_pad, n_seq = a.n_seq;
+  int32_t* comp = sm;
+  int32_t* tok_off = comp + n_pad;
+  int32_t* seg_of = tok_off + n_pad + 1;
+  int32_t* seg_tile = seg_of + n_pad;
+  int32_t* seg_short = seg_tile + n_pad + 1;
+  int32_t* seg_gather = seg_short + n_pad + 1;
+  const int tid = threadIdx.x;
+  const int layer = a.layer_begin + blockIdx.x;
+  int32_t* ws = a.ws + (size_t)blockIdx.x * a.ws_stride;
+  const int max_tenants = a.tab.max_tenants;
+
+  auto seq_rows = [&](int i, int* lo, int* hi) {
+    if (a.cu) { *lo = a.cu[i]; *hi = a.cu[i + 1]; }
+    else { *lo = i; *hi = i + 1; }
+  };
+
+  // ---- 1. composite keys, excluded-token count --------------------------------------------
+  int excl = 0;
+  for (int i = tid; i < n_pad; i += kGThreads) {
+    int c = INT_MAX;
+    if (i < n_seq) {
+      int lo, hi;
+      seq_rows(i, &lo, &hi);
+      bool rows_ok = lo >= 0 && hi >= lo && hi <= a.T;
+      if (!rows_ok) atomicOr(a.tab.err, ERR_BAD_ROW);
+      int len = rows_ok ? hi - lo : 0;
+      int slot = a.seq_slot[i];
+      bool ok = slot >= 0 && slot < a.tab.max_requests;
+      if (!ok) atomicOr(a.tab.err, ERR_BAD_SLOT);
+      int key = -1;
+      if (ok && len > 0) {
+        int tenant = a.tab.slot_tenant[slot];
+        int module = a.tab.route[(size_t)slot * a.tab.n_layers + layer];
+        if (tenant >= 0 && tenant < max_tenants && module >= 0 && module < MILORA_NMOD) {
+          const AdapterEntry& e = a.tab.adapters[adapter_index(tenant, layer, module, a.tab.n_layers)];
+          if (e.rank > 0) key = module * max_tenants + tenant;
+        }
+      }
+      if (key >= 0) c = (key << kSeqBits) | i;
+      else excl += len;
+    }
+    comp[i] = c;
+  }
+  int n_excl;
+  block_exscan(excl, &n_excl, wsum);
+
+  // ---- 2. bitonic sort of the composite keys ----------------------------------------------
+  for (int k = 2; k <= n_pad; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      __syncthreads();
+      for (int t = tid; t < n_pad / 2; t += kGThreads) {
+        int i = 2 * t - (t & (j - 1));      // index with bit j clear
+        int l = i + j;
+        bool up = (i & k) == 0;
+        int x = comp[i], y = comp[l];
+        if ((x > y) == up) { comp[i] = y; comp[l] = x; }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- 3. per-sequence quantities in sorted order; each thread owns consecutive positions ----
+  const int per = (n_pad + kGThreads - 1) / kGThreads;
+  const int j0 = tid * per, j1 = min(j0 + per, n_pad);
+  int s_tok = 0, s_head = 0, s_tile = 0, s_short = 0;
+  for (int j = j0; j < j1; ++j) {
+    int c = comp[j];
+    if (c == INT_MAX) break;
+    int lo, hi;
+    seq_rows(c & (kMaxSeq - 1), &lo, &hi);
+    int len = hi - lo;
+    s_tok += len;
+    s_head += (j == 0 || (comp[j - 1] >> kSeqBits) != (c >> kSeqBits)) ? 1 : 0;
+    if (len >= kLongSeq) s_tile += (len + kTileRows - 1) / kTileRows;
+    else s_short += len;
+  }
+  int n_active, n_seg, n_tiles, n_short;
+  int o_tok = block_exscan(s_tok, &n_active, wsum);
+  int o_head = block_exscan(s_head, &n_seg, wsum);
+  int o_tile = block_exscan(s_tile, &n_tiles, wsum);
+  int o_short = block_exscan(s_short, &n_short, wsum);
+
+  WorkItem* tiles = reinterpret_cast<WorkItem*>(ws + a.lay.tiles);
+  int32_t* gather_rows = ws + a.lay.gather_rows;
+  int32_t* seg_key = ws + a.lay.seg_key;
+  int32_t* seg_offset = ws + a.lay.seg_offset;
+  for (int j = j0; j < j1; ++j) {
+    int c = comp[j];
+    if (c == INT_MAX) break;
+    int key = c >> kSeqBits;
+    int lo, hi;
+    seq_rows(c & (kMaxSeq - 1), &lo, &hi);
+    int len = hi - lo;
+    bool head = (j == 0 || (comp[j - 1] >> kSeqBits) != key);
+    if (head) {
+      seg_key[o_head] = key;
+      seg_offset[o_head] = o_tok;
+      seg_tile[o_head] = o_tile;
+      seg_short[o_head] = o_short;
+      ++o_head;
+    }
+    const int seg = o_head - 1;
+    seg_of[j] = seg;
+    tok_off[j] = o_tok;
+    o_tok += len;
+    if (len >= kLongSeq) {
+      for (int r = 0; r < len; r += kTileRows) {
+        WorkItem w;
+        w.seg = seg; w.start = lo + r; w.count = min(kTileRows, len - r); w.module = key / max_tenants;
+        tiles[o_tile++] = w;
+      }
+    } else {
+      for (int r = 0; r < len; ++r) gather_rows[o_short++] = lo + r;
+    }
+  }
+  if (tid == 0) {
+    seg_offset[n_seg] = n_active;
+    seg_tile[n_seg] = n_tiles;
+    seg_short[n_seg] = n_short;
+  }
+  // number of sorted (active) sequences = first sentinel
+  __syncthreads();
+  int n_act_seq;
+  {
+    int cnt = 0;
+    for (int j = j0; j < j1; ++j) cnt += comp[j] != INT_MAX;
+    block_exscan(cnt, &n_act_seq, wsum);
+  }
+  if (tid == 0) tok_off[n_act_seq] = n_active;
+  __syncthreads();
+
+  // ---- 4. perm: token q of the sorted order ------------------------------------------------
+  int32_t* perm = ws + a.lay.perm;
+  for (int q = tid; q < n_active; q += kGThreads) {
+    int lo = 0, hi = n_act_seq;           // last j with tok_off[j] <= q
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (tok_off[mid] <= q) lo = mid; else hi = mid;
+    }
+    int rlo, rhi;
+    seq_rows(comp[lo] & (kMaxSeq - 1), &rlo, &rhi);
+    perm[q] = rlo + (q - tok_off[lo]);
+  }
+
+  // ---- 5. gather entries: chunks of kGatherRows short rows per segment ------------------------
+  const int sper = (n_seg + kGThreads - 1) / kGThreads;
+  const int s0 = min(tid * sper, n_seg), s1 = min(s0 + sper, n_seg);
+  int g_cnt = 0;
+  for (int s = s0; s < s1; ++s) g_cnt += (seg_short[s + 1] - seg_short[s] + kGatherRows - 1) / kGatherRows;
+  int n_gather;
+  int o_g = block_exscan(g_cnt, &n_gather, wsum);
+  WorkItem* gather = reinterpret_cast<WorkItem*>(ws + a.lay.gather);
+  for (int s = s0; s < s1; ++s) {
+    seg_gather[s] = o_g;
+    int b = seg_short[s], e = seg_short[s + 1];
+    int module = seg_key[s] / max_tenants;
+    for (int r = b; r < e; r += kGatherRows) {
+      WorkItem w;
+      w.seg = s; w.start = r; w.count = min(kGatherRows, e - r); w.module = module;
+      gather[o_g++] = w;
+    }
+  }
+  if (tid == 0) seg_gather[n_seg] = n_gather;
+  __syncthreads();
+
+  // ---- 6. header and per-module ranges -----------------------------------------------------
+  if (tid < 8) {
+    // first segment whose module is >= tid
+    int lo = 0, hi = n_seg;
+    while (lo < hi) {
+      int mid = (lo + hi) >> 1;
+      if (seg_key[mid] / max_tenants < tid) lo = mid + 1; else hi = mid;
+    }
+    ws[a.lay.mod_offset + tid] = lo;
+    ws[a.lay.mod_tile_offset + tid] = seg_tile[lo];
+    ws[a.lay.mod_gather_offset + tid] = seg_gather[lo];
+  }
+  if (tid < kHeaderInts) {
+    int v = 0;
+    if (tid == H_NSEG) v = n_seg;
+    else if (tid == H_NEXCL) v = n_excl;
+    else if (tid == H_NACTIVE) v = n_active;
+    else if (tid == H_NTILES) v = n_tiles;
+    else if (tid == H_NGATHER) v = n_gather;
+    ws[a.lay.header + tid] = v;
+  }
+}
+
+}  // namespace
+
+milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const int32_t* cu, const int32_t* seq_slot,
+                           int n_seq, int T, int32_t* ws, size_t ws_stride, cudaStream_t s) {
+  if ((long long)ctx->desc.max_tenants * MILORA_NMOD >= (1ll << (31 - kSeqBits))) return MILORA_E_CAPACITY;
+  GroupArgs a;
+  a.tab = device_tables(ctx);
+  a.cu = cu; a.seq_slot = seq_slot; a.ws = ws; a.ws_stride = ws_stride;
+  a.lay = group_layout(n_seq, T);
+  a.layer_begin = layer_begin; a.n_seq = n_seq; a.T = T;
+  int n_pad = 2;
+  while (n_pad < n_seq) n_pad <<= 1;
+  a.n_pad = n_pad;
+  size_t smem = ((size_t)n_pad * 6 + 4) * sizeof(int32_t);
+  if (smem > 48 * 1024) {
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  }
+  group_kernel<<<n_layers, kGThreads, smem, s>>>(a);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+}  // namespace milora

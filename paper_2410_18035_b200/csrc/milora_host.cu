@@ -1,0 +1,478 @@
+// Host side of libmilora: context, adapter / router / slot tables, argument validation.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "milora_internal.h"
+
+namespace milora {
+
+milora_status cuda_fail(milora_ctx* ctx, cudaError_t e, const char* where) {
+  if (ctx) {
+    ctx->cuda_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " at " + where;
+  }
+  cudaGetLastError();  // clear the sticky-free error state
+  return MILORA_E_CUDA;
+}
+
+void* Arena::alloc(size_t bytes, cudaError_t* err) {
+  *err = cudaSuccess;
+  bytes = (bytes + 255) & ~size_t(255);
+  for (auto& c : chunks) {
+    if (c.size - c.used >= bytes) {
+      void* p = c.base + c.used;
+      c.used += bytes;
+      return p;
+    }
+  }
+  size_t sz = std::max(bytes, size_t(64) << 20);
+  char* base = nullptr;
+  *err = cudaMalloc(&base, sz);
+  if (*err != cudaSuccess) return nullptr;
+  chunks.push_back({base, sz, bytes});
+  return base;
+}
+
+void Arena::release() {
+  for (auto& c : chunks) cudaFree(c.base);
+  chunks.clear();
+}
+
+void module_dims(const milora_model_desc& d, int module, int* d1, int* d2) {
+  switch (module) {
+    case MILORA_Q:
+    case MILORA_O: *d1 = d.d_model; *d2 = d.d_model; break;
+    case MILORA_K:
+    case MILORA_V: *d1 = d.d_model; *d2 = d.d_kv; break;
+    case MILORA_GATE:
+    case MILORA_UP: *d1 = d.d_model; *d2 = d.d_ff; break;
+    default: *d1 = d.d_ff; *d2 = d.d_model; break;
+  }
+}
+
+static size_t round4(size_t v) { return (v + 3) & ~size_t(3); }
+
+milora_group_layout_t group_layout(int n_seq, int T) {
+  milora_group_layout_t L;
+  size_t o = 0;
+  L.header = o; o += kHeaderInts;
+  L.mod_offset = o; o += 8;
+  L.mod_tile_offset = o; o += 8;
+  L.mod_gather_offset = o; o += 8;
+  L.seg_key = o; o += round4((size_t)n_seq);
+  L.seg_offset = o; o += round4((size_t)n_seq + 1);
+  L.perm = o; o += round4((size_t)T);
+  L.max_tiles = T / kTileRows + n_seq;
+  L.tiles = o; o += (size_t)L.max_tiles * 4;
+  L.gather_rows = o; o += round4((size_t)T);
+  L.max_gather = T / kGatherRows + n_seq + 1;
+  L.gather = o; o += (size_t)L.max_gather * 4;
+  L.total = round4(o);
+  return L;
+}
+
+DeviceTables device_tables(const milora_ctx* ctx) {
+  DeviceTables t;
+  t.adapters = ctx->d_adapters;
+  t.routers = ctx->d_routers;
+  t.slot_tenant = ctx->d_slot_tenant;
+  t.route = ctx->d_route;
+  t.err = ctx->d_err;
+  t.n_layers = ctx->desc.n_layers;
+  t.max_tenants = ctx->desc.max_tenants;
+  t.max_requests = ctx->desc.max_requests;
+  return t;
+}
+
+template <class T>
+static milora_status upload_range(milora_ctx* ctx, T* dev, const std::vector<T>& host, size_t& lo, size_t& hi,
+                                  cudaStream_t s) {
+  if (lo < hi) {
+    MILORA_CUDA(ctx, cudaMemcpyAsync(dev + lo, host.data() + lo, (hi - lo) * sizeof(T), cudaMemcpyHostToDevice, s));
+    // The source is pageable memory that the next registration may change: wait until it is consumed.
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  }
+  lo = host.size();
+  hi = 0;
+  return MILORA_OK;
+}
+
+milora_status sync_tables(milora_ctx* ctx, cudaStream_t s) {
+  milora_status st;
+  if ((st = upload_range(ctx, ctx->d_adapters, ctx->h_adapters, ctx->adapters_dirty_lo, ctx->adapters_dirty_hi, s)))
+    return st;
+  if ((st = upload_range(ctx, ctx->d_routers, ctx->h_routers, ctx->routers_dirty_lo, ctx->routers_dirty_hi, s)))
+    return st;
+  if ((st = upload_range(ctx, ctx->d_slot_tenant, ctx->h_slot_tenant, ctx->slots_dirty_lo, ctx->slots_dirty_hi, s)))
+    return st;
+  return MILORA_OK;
+}
+
+static void mark(size_t& lo, size_t& hi, size_t i) {
+  lo = std::min(lo, i);
+  hi = std::max(hi, i + 1);
+}
+
+static cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+}  // namespace milora
+
+using namespace milora;
+
+extern "C" {
+
+const char* milora_status_string(milora_status s) {
+  switch (s) {
+    case MILORA_OK: return "ok";
+    case MILORA_E_ARG: return "invalid argument";
+    case MILORA_E_SHAPE: return "unsupported shape";
+    case MILORA_E_DTYPE: return "unsupported dtype";
+    case MILORA_E_UNREGISTERED: return "not registered";
+    case MILORA_E_CAPACITY: return "capacity exceeded";
+    case MILORA_E_STATE: return "invalid state";
+    case MILORA_E_CUDA: return "CUDA error";
+    case MILORA_E_DEVICE_INDEX: return "a kernel skipped an out-of-range index";
+  }
+  return "unknown status";
+}
+
+const char* milora_last_cuda_error(const milora_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
+  if (!desc || !out) return MILORA_E_ARG;
+  *out = nullptr;
+  if (desc->dtype != MILORA_F32 && desc->dtype != MILORA_BF16) return MILORA_E_DTYPE;
+  if (desc->n_layers < 1 || desc->d_model < 1 || desc->d_ff < 1 || desc->d_kv < 1) return MILORA_E_SHAPE;
+  {
+    // every row of every matrix must start on a 16-byte boundary (128-bit loads, bulk copies)
+    const int vec = desc->dtype == MILORA_F32 ? 4 : 8;
+    if (desc->d_model % vec || desc->d_ff % vec || desc->d_kv % vec) return MILORA_E_SHAPE;
+  }
+  if (desc->max_rank < 1 || desc->max_rank > 256) return MILORA_E_CAPACITY;
+  if (desc->max_tenants < 1 || desc->max_requests < 1) return MILORA_E_CAPACITY;
+  if ((long long)desc->max_tenants * MILORA_NMOD > (1ll << 30)) return MILORA_E_CAPACITY;
+  milora_ctx* ctx = new (std::nothrow) milora_ctx();
+  if (!ctx) return MILORA_E_CAPACITY;
+  ctx->desc = *desc;
+  ctx->elem = desc->dtype == MILORA_F32 ? 4 : 2;
+  ctx->d_adapters = nullptr; ctx->d_routers = nullptr; ctx->d_slot_tenant = nullptr; ctx->d_route = nullptr;
+  ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
+  ctx->n_counters = 0;
+  milora_status st = MILORA_OK;
+  auto fail = [&](milora_status s) { milora_destroy(ctx); return s; };
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e != cudaSuccess) { st = cuda_fail(ctx, e, "cudaGetDevice"); return fail(st); }
+  e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e != cudaSuccess) { st = cuda_fail(ctx, e, "cudaDeviceGetAttribute"); return fail(st); }
+  size_t n_ad = (size_t)desc->max_tenants * desc->n_layers * MILORA_NMOD;
+  size_t n_rt = (size_t)desc->max_tenants * desc->n_layers;
+  try {
+    ctx->h_adapters.assign(n_ad, AdapterEntry{nullptr, nullptr, 0, 0.f, {0, 0}});
+    RouterEntry r0;
+    std::memset(&r0, 0, sizeof(r0));
+    ctx->h_routers.assign(n_rt, r0);
+    ctx->h_slot_tenant.assign(desc->max_requests, -1);
+    ctx->adapter_bytes.assign(n_ad, 0);
+    ctx->router_bytes.assign(n_rt, 0);
+  } catch (...) {
+    return fail(MILORA_E_CAPACITY);
+  }
+  ctx->adapters_dirty_lo = 0; ctx->adapters_dirty_hi = n_ad;
+  ctx->routers_dirty_lo = 0; ctx->routers_dirty_hi = n_rt;
+  ctx->slots_dirty_lo = 0; ctx->slots_dirty_hi = desc->max_requests;
+  size_t route_bytes = (size_t)desc->max_requests * desc->n_layers * sizeof(int32_t);
+#define CREATE_CUDA(call)                                            \
+  do {                                                               \
+    cudaError_t e__ = (call);                                        \
+    if (e__ != cudaSuccess) return fail(cuda_fail(ctx, e__, #call)); \
+  } while (0)
+  CREATE_CUDA(cudaMalloc(&ctx->d_adapters, n_ad * sizeof(AdapterEntry)));
+  CREATE_CUDA(cudaMalloc(&ctx->d_routers, n_rt * sizeof(RouterEntry)));
+  CREATE_CUDA(cudaMalloc(&ctx->d_slot_tenant, desc->max_requests * sizeof(int32_t)));
+  CREATE_CUDA(cudaMalloc(&ctx->d_route, route_bytes));
+  CREATE_CUDA(cudaMalloc(&ctx->d_err, 256));
+  CREATE_CUDA(cudaMemset(ctx->d_route, 0xFF, route_bytes));
+  CREATE_CUDA(cudaMemset(ctx->d_err, 0, 256));
+  st = sync_tables(ctx, nullptr);
+  if (st != MILORA_OK) return fail(st);
+  CREATE_CUDA(cudaDeviceSynchronize());
+#undef CREATE_CUDA
+  *out = ctx;
+  return MILORA_OK;
+}
+
+milora_status milora_destroy(milora_ctx* ctx) {
+  if (!ctx) return MILORA_OK;
+  cudaFree(ctx->d_adapters);
+  cudaFree(ctx->d_routers);
+  cudaFree(ctx->d_slot_tenant);
+  cudaFree(ctx->d_route);
+  cudaFree(ctx->d_err);
+  cudaFree(ctx->d_scratch);
+  cudaFree(ctx->d_counters);
+  ctx->arena.release();
+  delete ctx;
+  return MILORA_OK;
+}
+
+milora_status milora_module_dims(const milora_ctx* ctx, int module, int* d1, int* d2) {
+  if (!ctx || !d1 || !d2 || module < 0 || module >= MILORA_NMOD) return MILORA_E_ARG;
+  module_dims(ctx->desc, module, d1, d2);
+  return MILORA_OK;
+}
+
+milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, int module, int rank, float scale,
+                                      const void* A_dev, const void* B_dev, void* stream) {
+  if (!ctx || !A_dev || !B_dev) return MILORA_E_ARG;
+  if (tenant < 0 || tenant >= ctx->desc.max_tenants || layer < 0 || layer >= ctx->desc.n_layers || module < 0 ||
+      module >= MILORA_NMOD)
+    return MILORA_E_ARG;
+  if (rank < 1) return MILORA_E_ARG;
+  if (rank > ctx->desc.max_rank) return MILORA_E_CAPACITY;
+  int d1, d2;
+  module_dims(ctx->desc, module, &d1, &d2);
+  size_t idx = adapter_index(tenant, layer, module, ctx->desc.n_layers);
+  size_t bytes_a = ((size_t)rank * d1 * ctx->elem + 255) & ~size_t(255);
+  size_t bytes_b = ((size_t)rank * d2 * ctx->elem + 255) & ~size_t(255);
+  AdapterEntry& ent = ctx->h_adapters[idx];
+  void* store = const_cast<void*>(ent.At);
+  if (!store || ctx->adapter_bytes[idx] != bytes_a + bytes_b) {
+    cudaError_t e;
+    store = ctx->arena.alloc(bytes_a + bytes_b, &e);
+    if (!store) return cuda_fail(ctx, e, "adapter pool cudaMalloc");
+    ctx->adapter_bytes[idx] = bytes_a + bytes_b;
+  }
+  void* At = store;
+  void* Bs = static_cast<char*>(store) + bytes_a;
+  milora_status st = launch_repack_adapter(ctx, A_dev, B_dev, At, Bs, d1, d2, rank, as_stream(stream));
+  if (st != MILORA_OK) return st;
+  ent.At = At;
+  ent.B = Bs;
+  ent.rank = rank;
+  ent.scale = scale;
+  mark(ctx->adapters_dirty_lo, ctx->adapters_dirty_hi, idx);
+  return MILORA_OK;
+}
+
+milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, const void* Wr_dev,
+                                     const float* bias_dev, milora_pool pool, const void* Wsa_dev, milora_act act,
+                                     const float* coef_host, int n_a, int n_b, void* stream) {
+  if (!ctx || !Wr_dev) return MILORA_E_ARG;
+  if (tenant < 0 || tenant >= ctx->desc.max_tenants || layer < 0 || layer >= ctx->desc.n_layers) return MILORA_E_ARG;
+  if (pool < MILORA_POOL_MEAN || pool > MILORA_POOL_SELFATTN) return MILORA_E_ARG;
+  if (act < MILORA_ACT_TANH || act > MILORA_ACT_RATIONAL) return MILORA_E_ARG;
+  if (pool == MILORA_POOL_SELFATTN && !Wsa_dev) return MILORA_E_ARG;
+  if (act == MILORA_ACT_RATIONAL) {
+    if (!coef_host || n_a < 1 || n_b < 0 || n_a + n_b > MILORA_MAX_RATIONAL_COEF) return MILORA_E_ARG;
+  } else {
+    n_a = n_b = 0;
+  }
+  cudaStream_t s = as_stream(stream);
+  size_t idx = (size_t)tenant * ctx->desc.n_layers + layer;
+  int d = ctx->desc.d_model;
+  size_t bytes_w = ((size_t)MILORA_NMOD * d * ctx->elem + 255) & ~size_t(255);
+  size_t bytes_sa = ((size_t)d * ctx->elem + 255) & ~size_t(255);
+  RouterEntry& ent = ctx->h_routers[idx];
+  void* store = const_cast<void*>(ent.W);
+  if (!store || ctx->router_bytes[idx] != bytes_w + bytes_sa) {
+    cudaError_t e;
+    store = ctx->arena.alloc(bytes_w + bytes_sa, &e);
+    if (!store) return cuda_fail(ctx, e, "router pool cudaMalloc");
+    ctx->router_bytes[idx] = bytes_w + bytes_sa;
+  }
+  void* Wt = store;
+  void* Wsa = static_cast<char*>(store) + bytes_w;
+  milora_status st = launch_repack_router(ctx, Wr_dev, Wt, d, s);
+  if (st != MILORA_OK) return st;
+  if (Wsa_dev) MILORA_CUDA(ctx, cudaMemcpyAsync(Wsa, Wsa_dev, (size_t)d * ctx->elem, cudaMemcpyDeviceToDevice, s));
+  std::memset(ent.bias, 0, sizeof(ent.bias));
+  if (bias_dev) {
+    MILORA_CUDA(ctx, cudaMemcpyAsync(ent.bias, bias_dev, MILORA_NMOD * sizeof(float), cudaMemcpyDeviceToHost, s));
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  }
+  std::memset(ent.coef, 0, sizeof(ent.coef));
+  for (int i = 0; i < n_a + n_b; ++i) ent.coef[i] = coef_host[i];
+  ent.W = Wt;
+  ent.Wsa = Wsa_dev ? Wsa : nullptr;
+  ent.pool = pool;
+  ent.act = act;
+  ent.n_a = n_a;
+  ent.n_b = n_b;
+  mark(ctx->routers_dirty_lo, ctx->routers_dirty_hi, idx);
+  return MILORA_OK;
+}
+
+milora_status milora_unregister_tenant(milora_ctx* ctx, int tenant) {
+  if (!ctx || tenant < 0 || tenant >= ctx->desc.max_tenants) return MILORA_E_ARG;
+  for (int t : ctx->h_slot_tenant)
+    if (t == tenant) return MILORA_E_STATE;
+  int L = ctx->desc.n_layers;
+  for (int l = 0; l < L; ++l) {
+    for (int m = 0; m < MILORA_NMOD; ++m) {
+      size_t idx = adapter_index(tenant, l, m, L);
+      ctx->h_adapters[idx].rank = 0;  // storage pointer is kept for reuse by a later registration
+      mark(ctx->adapters_dirty_lo, ctx->adapters_dirty_hi, idx);
+    }
+    size_t r = (size_t)tenant * L + l;
+    ctx->h_routers[r].pool = -1;  // marks "not registered" while keeping the storage pointer
+    mark(ctx->routers_dirty_lo, ctx->routers_dirty_hi, r);
+  }
+  return MILORA_OK;
+}
+
+milora_status milora_request_open(milora_ctx* ctx, int slot, int tenant) {
+  if (!ctx || slot < 0 || slot >= ctx->desc.max_requests || tenant < 0 || tenant >= ctx->desc.max_tenants)
+    return MILORA_E_ARG;
+  if (ctx->h_slot_tenant[slot] >= 0) return MILORA_E_STATE;
+  // The route row of a freshly opened slot must read "not routed".
+  // The slot is closed, so no kernel in flight reads this row; the reset is finished before returning.
+  MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_route + (size_t)slot * ctx->desc.n_layers, 0xFF,
+                                   (size_t)ctx->desc.n_layers * sizeof(int32_t), nullptr));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(nullptr));
+  ctx->h_slot_tenant[slot] = tenant;
+  mark(ctx->slots_dirty_lo, ctx->slots_dirty_hi, (size_t)slot);
+  return MILORA_OK;
+}
+
+milora_status milora_request_close(milora_ctx* ctx, int slot) {
+  if (!ctx || slot < 0 || slot >= ctx->desc.max_requests) return MILORA_E_ARG;
+  if (ctx->h_slot_tenant[slot] < 0) return MILORA_E_STATE;
+  ctx->h_slot_tenant[slot] = -1;
+  mark(ctx->slots_dirty_lo, ctx->slots_dirty_hi, (size_t)slot);
+  return MILORA_OK;
+}
+
+milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const int32_t* cu_seqlens_dev,
+                           const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
+                           float* probs_out_dev, void* stream) {
+  if (!ctx) return MILORA_E_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers || P < 0 || T_total < 0) return MILORA_E_ARG;
+  if (P > kMaxSeq) return MILORA_E_CAPACITY;
+  if (P == 0) return MILORA_OK;
+  if (!cu_seqlens_dev || !seq_slot_dev || (T_total > 0 && !H_dev)) return MILORA_E_ARG;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);
+  if (st != MILORA_OK) return st;
+  return launch_route(ctx, layer, H_dev, cu_seqlens_dev, seq_slot_dev, P, T_total, logits_out_dev, probs_out_dev, s);
+}
+
+milora_status milora_route_table(const milora_ctx* ctx, const int32_t** table_dev) {
+  if (!ctx || !table_dev) return MILORA_E_ARG;
+  *table_dev = ctx->d_route;
+  return MILORA_OK;
+}
+
+milora_status milora_route_table_read(milora_ctx* ctx, int slot_begin, int n_slots, int32_t* rows_host, void* stream) {
+  if (!ctx || !rows_host || slot_begin < 0 || n_slots < 0 || slot_begin + n_slots > ctx->desc.max_requests)
+    return MILORA_E_ARG;
+  if (n_slots == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  size_t L = ctx->desc.n_layers;
+  MILORA_CUDA(ctx, cudaMemcpyAsync(rows_host, ctx->d_route + (size_t)slot_begin * L, (size_t)n_slots * L * sizeof(int32_t),
+                                   cudaMemcpyDeviceToHost, s));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  return MILORA_OK;
+}
+
+milora_status milora_route_table_write(milora_ctx* ctx, int slot_begin, int n_slots, const int32_t* rows_host,
+                                       void* stream) {
+  if (!ctx || !rows_host || slot_begin < 0 || n_slots < 0 || slot_begin + n_slots > ctx->desc.max_requests)
+    return MILORA_E_ARG;
+  size_t L = ctx->desc.n_layers;
+  for (size_t i = 0; i < (size_t)n_slots * L; ++i)
+    if (rows_host[i] < -1 || rows_host[i] >= MILORA_NMOD) return MILORA_E_ARG;
+  if (n_slots == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  MILORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_route + (size_t)slot_begin * L, rows_host, (size_t)n_slots * L * sizeof(int32_t),
+                                   cudaMemcpyHostToDevice, s));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  return MILORA_OK;
+}
+
+milora_status milora_group_layout(const milora_ctx* ctx, int n_seq, int T, milora_group_layout_t* out) {
+  if (!ctx || !out || n_seq < 0 || T < 0) return MILORA_E_ARG;
+  if (n_seq > kMaxSeq) return MILORA_E_CAPACITY;
+  *out = group_layout(n_seq, T);
+  return MILORA_OK;
+}
+
+milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const int32_t* cu_seqlens_dev,
+                           const int32_t* seq_slot_dev, int n_seq, int T, int32_t* ws_dev, size_t ws_stride,
+                           void* stream) {
+  if (!ctx || !ws_dev) return MILORA_E_ARG;
+  if (layer_begin < 0 || n_layers < 1 || layer_begin + n_layers > ctx->desc.n_layers) return MILORA_E_ARG;
+  if (n_seq < 0 || T < 0 || (n_seq > 0 && !seq_slot_dev)) return MILORA_E_ARG;
+  if (n_seq > kMaxSeq) return MILORA_E_CAPACITY;
+  if (!cu_seqlens_dev && T != n_seq) return MILORA_E_ARG;
+  milora_group_layout_t L = group_layout(n_seq, T);
+  if (ws_stride < L.total || (ws_stride & 3) || (reinterpret_cast<uintptr_t>(ws_dev) & 15)) return MILORA_E_ARG;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);
+  if (st != MILORA_OK) return st;
+  return launch_group(ctx, layer_begin, n_layers, cu_seqlens_dev, seq_slot_dev, n_seq, T, ws_dev, ws_stride, s);
+}
+
+static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const int* modules,
+                                  const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
+                                  bool dense, void* stream) {
+  if (!ctx || !groups || !modules || !X_dev || !Y_dev) return MILORA_E_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return MILORA_E_ARG;
+  if (n_sites < 1 || n_sites > kMaxSites) return MILORA_E_ARG;
+  if (!groups->ws_dev || groups->n_seq < 0 || groups->T < 0 || groups->n_seq > kMaxSeq) return MILORA_E_ARG;
+  ApplySites sites;
+  sites.n = n_sites;
+  unsigned seen = 0;
+  for (int i = 0; i < n_sites; ++i) {
+    int m = modules[i];
+    if (m < 0 || m >= MILORA_NMOD || (seen >> m & 1)) return MILORA_E_ARG;
+    seen |= 1u << m;
+    if (groups->T > 0 && (!X_dev[i] || !Y_dev[i])) return MILORA_E_ARG;
+    sites.site[i].module = m;
+    sites.site[i].X = X_dev[i];
+    sites.site[i].Y = Y_dev[i];
+    module_dims(ctx->desc, m, &sites.site[i].d1, &sites.site[i].d2);
+  }
+  if (groups->T == 0 || groups->n_seq == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);
+  if (st != MILORA_OK) return st;
+  return launch_apply_generic(ctx, layer, sites, groups, dense, s);
+}
+
+milora_status milora_apply_decode(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
+                                  const milora_groups* groups, void* stream) {
+  return apply_common(ctx, layer, 1, &module, &X_dev, &Y_dev, groups, false, stream);
+}
+
+milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
+                                   const milora_groups* groups, void* stream) {
+  return apply_common(ctx, layer, 1, &module, &X_dev, &Y_dev, groups, true, stream);
+}
+
+milora_status milora_apply_decode_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,
+                                        const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
+                                        void* stream) {
+  return apply_common(ctx, layer, n_sites, modules, X_dev, Y_dev, groups, false, stream);
+}
+
+milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,
+                                         const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
+                                         void* stream) {
+  return apply_common(ctx, layer, n_sites, modules, X_dev, Y_dev, groups, true, stream);
+}
+
+milora_status milora_poll_error(milora_ctx* ctx, int* device_flag_out, void* stream) {
+  if (!ctx || !device_flag_out) return MILORA_E_ARG;
+  cudaStream_t s = as_stream(stream);
+  int32_t flag = 0;
+  MILORA_CUDA(ctx, cudaMemcpyAsync(&flag, ctx->d_err, sizeof(flag), cudaMemcpyDeviceToHost, s));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  if (flag) {
+    MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_err, 0, sizeof(int32_t), s));
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  }
+  *device_flag_out = flag;
+  return flag ? MILORA_E_DEVICE_INDEX : MILORA_OK;
+}
+
+}  // extern "C"

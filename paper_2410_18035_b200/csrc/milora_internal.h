@@ -1,0 +1,139 @@
+// Internal declarations shared by the host code and the kernels of libmilora.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "milora.h"
+
+namespace milora {
+
+// ---- device-visible tables -------------------------------------------------------------
+// One LoRA pair in library layout: At is rank x d1 (W^A transposed), B is rank x d2, both
+// row-major in the context dtype and 256-byte aligned.
+struct AdapterEntry {
+  const void* At;
+  const void* B;
+  int32_t rank;   // 0 = not registered
+  float scale;
+  int32_t pad[2];
+};
+static_assert(sizeof(AdapterEntry) == 32, "AdapterEntry must stay 32 bytes");
+
+// Router of one (tenant, layer): W is 7 x d (W_r transposed), context dtype.
+struct RouterEntry {
+  const void* W;      // nullptr = not registered
+  const void* Wsa;    // d values, only for the self-attention pooler
+  float bias[8];      // 7 used; zeros when the router has no bias
+  float coef[MILORA_MAX_RATIONAL_COEF];
+  int32_t pool, act, n_a, n_b;
+};
+
+// Work-list entry written by the grouping kernel (4 int32): a dense tile is `count` consecutive
+// rows starting at `start`; a gather entry is `count` rows listed at gather_rows[start ...].
+struct WorkItem {
+  int32_t seg, start, count, module;
+};
+
+constexpr int kHeaderInts = 16;
+constexpr int kTileRows = 128;     // rows per dense tile (prefill path)
+constexpr int kGatherRows = 8;     // rows per gather entry (decode path)
+constexpr int kLongSeq = 32;       // sequences of at least this many tokens go to dense tiles
+constexpr int kMaxSeq = 4096;      // sequences per grouping / routing call
+enum HeaderSlot { H_NSEG = 0, H_NEXCL = 1, H_NACTIVE = 2, H_NTILES = 3, H_NGATHER = 4 };
+
+// Device error flag bits.
+enum ErrBit { ERR_BAD_SLOT = 1, ERR_BAD_ROW = 2, ERR_WAIT_TIMEOUT = 4, ERR_BAD_ITEM = 8 };
+
+struct DeviceTables {
+  const AdapterEntry* adapters;   // [max_tenants][n_layers][7]
+  const RouterEntry* routers;     // [max_tenants][n_layers]
+  const int32_t* slot_tenant;     // [max_requests], -1 = closed
+  int32_t* route;                 // [max_requests][n_layers]
+  int32_t* err;                   // single flag word
+  int n_layers, max_tenants, max_requests;
+};
+
+__host__ __device__ inline size_t adapter_index(int tenant, int layer, int module, int n_layers) {
+  return ((size_t)tenant * n_layers + layer) * MILORA_NMOD + module;
+}
+
+struct Arena {
+  struct Chunk { char* base; size_t size, used; };
+  std::vector<Chunk> chunks;
+  void* alloc(size_t bytes, cudaError_t* err);
+  void release();
+};
+
+}  // namespace milora
+
+struct milora_ctx {
+  milora_model_desc desc;
+  int device;
+  int sm_count;
+  size_t elem;                                  // bytes per element of the context dtype
+  std::vector<milora::AdapterEntry> h_adapters; // host mirrors
+  std::vector<milora::RouterEntry> h_routers;
+  std::vector<int32_t> h_slot_tenant;
+  std::vector<size_t> adapter_bytes;            // pool bytes behind each adapter entry (for reuse)
+  std::vector<size_t> router_bytes;
+  size_t adapters_dirty_lo, adapters_dirty_hi;  // host-mirror ranges not yet uploaded
+  size_t routers_dirty_lo, routers_dirty_hi;
+  size_t slots_dirty_lo, slots_dirty_hi;
+  milora::AdapterEntry* d_adapters;
+  milora::RouterEntry* d_routers;
+  int32_t* d_slot_tenant;
+  int32_t* d_route;
+  int32_t* d_err;
+  float* d_scratch;                             // router partial sums
+  size_t scratch_floats;
+  int32_t* d_counters;                          // router completion counters, one per prompt
+  size_t n_counters;
+  milora::Arena arena;
+  std::string cuda_error;
+};
+
+namespace milora {
+
+milora_status cuda_fail(milora_ctx* ctx, cudaError_t e, const char* where);
+#define MILORA_CUDA(ctx, call)                                        \
+  do {                                                                \
+    cudaError_t e__ = (call);                                         \
+    if (e__ != cudaSuccess) return milora::cuda_fail((ctx), e__, #call); \
+  } while (0)
+
+// Uploads dirty ranges of the host mirrors on `stream`; called by every compute entry point.
+milora_status sync_tables(milora_ctx* ctx, cudaStream_t stream);
+DeviceTables device_tables(const milora_ctx* ctx);
+void module_dims(const milora_model_desc& d, int module, int* d1, int* d2);
+milora_group_layout_t group_layout(int n_seq, int T);
+
+// kernels (defined in their own .cu files)
+milora_status launch_repack_adapter(milora_ctx* ctx, const void* A, const void* B, void* At, void* Bout, int d1, int d2,
+                                    int rank, cudaStream_t s);
+milora_status launch_repack_router(milora_ctx* ctx, const void* Wr, void* Wt, int d, cudaStream_t s);
+milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot, int P,
+                           int T_total, float* logits_out, float* probs_out, cudaStream_t s);
+milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const int32_t* cu, const int32_t* seq_slot,
+                           int n_seq, int T, int32_t* ws, size_t ws_stride, cudaStream_t s);
+
+struct ApplySite {
+  int module;
+  const void* X;
+  void* Y;
+  int d1, d2;
+};
+constexpr int kMaxSites = MILORA_NMOD;
+struct ApplySites {
+  ApplySite site[kMaxSites];
+  int n;
+};
+// Generic SIMT path (any dtype, any shape): gathered rows (decode) or dense tiles (prefill).
+milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                   bool dense, cudaStream_t s);
+
+}  // namespace milora

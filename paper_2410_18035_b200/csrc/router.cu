@@ -1,0 +1,423 @@
+// Prompt-aware router (Section 3.3, Eq. 2-3; Appendix C; Eq. 7), one fused launch per layer:
+// pooling over the prompt's rows -> activation g -> 7 dot products with W_r -> softmax -> argmax,
+// written to the int32 route table.
+//
+// The kernel is bound by reading H (e * n_p * d bytes per prompt).  Work is cut into items of
+// kRows consecutive rows x one block of columns; every item writes fp32 partial column sums to
+// scratch, and the CTA that completes a prompt last (an atomic counter per prompt, no waiting)
+// combines the partials in chunk order, so the result does not depend on scheduling.
+#include <cfloat>
+
+#include "milora_internal.h"
+
+namespace milora {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRows = 64;
+
+template <typename T> struct VecOf;
+template <> struct VecOf<float> {
+  static constexpr int N = 4;
+  __device__ static void load(const float* p, float (&v)[4]) {
+    float4 q = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  }
+};
+template <> struct VecOf<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static void load(const __nv_bfloat16* p, float (&v)[8]) {
+    uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+};
+
+__device__ inline float to_float(float v) { return v; }
+__device__ inline float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+__device__ inline float activate(float h, const RouterEntry& r) {
+  switch (r.act) {
+    case MILORA_ACT_TANH: return tanhf(h);
+    case MILORA_ACT_RELU: return fmaxf(h, 0.f);
+    case MILORA_ACT_GELU: return 0.5f * h * (1.f + erff(h * 0.70710678118654752f));
+    case MILORA_ACT_RATIONAL: {
+      // Eq. 7: sum_j a_j x^j / (1 + |sum_i b_i x^i|), both by Horner's rule.
+      float num = 0.f;
+      for (int j = r.n_a - 1; j >= 0; --j) num = fmaf(num, h, r.coef[j]);
+      float den = 0.f;
+      for (int i = r.n_b - 1; i >= 0; --i) den = fmaf(den, h, r.coef[r.n_a + i]);
+      den *= h;
+      return num / (1.f + fabsf(den));
+    }
+    default: return h;
+  }
+}
+
+// Sum over the block in a fixed order: lanes by xor-shuffle, then warp 0 adds the warp totals in order.
+template <int NV>
+__device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][8] */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
+  }
+  __syncthreads();
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < NV; ++i) smem[i * 8 + warp] = v[i];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) s += smem[i * 8 + w];
+    v[i] = s;
+  }
+}
+
+struct RouteArgs {
+  DeviceTables tab;
+  const void* H;
+  const int32_t* cu;
+  const int32_t* seq_slot;
+  float* logits_out;
+  float* probs_out;
+  float* partial;     // [total_chunks][d]
+  float* stats;       // [total_chunks][2]  (self-attention pooler: chunk max, chunk sum of exp)
+  int32_t* counters;  // [P], zero on entry, zero again on exit
+  int layer, P, d, n_colblk;
+};
+
+// Dynamic shared memory: item_start[P+1], chunk_base[P+1].
+template <typename T>
+__global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
+  extern __shared__ int32_t sm_i[];
+  int32_t* item_start = sm_i;
+  int32_t* chunk_base = sm_i + (a.P + 1);
+  __shared__ float red[8 * 8];
+  __shared__ float u_sm[kRows];
+  __shared__ int32_t carry[2];
+  __shared__ int32_t is_last;
+  constexpr int V = VecOf<T>::N;
+  const int tid = threadIdx.x;
+  const int d = a.d;
+  const T* H = static_cast<const T*>(a.H);
+
+  // ---- per-CTA prefix over prompts: how many items and scratch rows each prompt owns ----
+  if (tid == 0) { carry[0] = 0; carry[1] = 0; }
+  __syncthreads();
+  for (int base = 0; base < a.P; base += kThreads) {
+    int p = base + tid;
+    int items = 0, chunks = 0;
+    if (p < a.P) {
+      int slot = a.seq_slot[p];
+      int n_p = a.cu[p + 1] - a.cu[p];
+      bool ok = slot >= 0 && slot < a.tab.max_requests && n_p > 0;
+      int tenant = ok ? a.tab.slot_tenant[slot] : -1;
+      ok = ok && tenant >= 0 && tenant < a.tab.max_tenants;
+      if (ok) {
+        const RouterEntry& r = a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer];
+        ok = r.W != nullptr && r.pool >= 0;
+        if (ok) {
+          if (r.pool == MILORA_POOL_LAST) n_p = 1;
+          chunks = (n_p + kRows - 1) / kRows;
+          items = chunks * (r.pool == MILORA_POOL_SELFATTN ? 1 : a.n_colblk);
+        }
+      }
+      if (!ok && blockIdx.x == 0) {
+        if (slot >= 0 && slot < a.tab.max_requests) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
+        else atomicOr(a.tab.err, ERR_BAD_SLOT);
+      }
+    }
+    // inclusive scan of (items, chunks) over the 256 prompts of this round
+    int si = items, sc = chunks;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int ti = __shfl_up_sync(0xffffffffu, si, o), tc = __shfl_up_sync(0xffffffffu, sc, o);
+      if (lane >= o) { si += ti; sc += tc; }
+    }
+    __shared__ int32_t wsum[2][8];
+    if (lane == 31) { wsum[0][warp] = si; wsum[1][warp] = sc; }
+    __syncthreads();
+    int offi = carry[0], offc = carry[1];
+    for (int w = 0; w < warp; ++w) { offi += wsum[0][w]; offc += wsum[1][w]; }
+    if (p < a.P) { item_start[p] = offi + si - items; chunk_base[p] = offc + sc - chunks; }
+    __syncthreads();
+    if (tid == kThreads - 1) { carry[0] = offi + si; carry[1] = offc + sc; }
+    __syncthreads();
+  }
+  if (tid == 0) { item_start[a.P] = carry[0]; chunk_base[a.P] = carry[1]; }
+  __syncthreads();
+  const int total_items = item_start[a.P];
+
+  for (int it = blockIdx.x; it < total_items; it += gridDim.x) {
+    // prompt of this item: last p with item_start[p] <= it
+    int lo = 0, hi = a.P;
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (item_start[mid] <= it) lo = mid; else hi = mid;
+    }
+    const int p = lo;
+    const int slot = a.seq_slot[p];
+    const int tenant = a.tab.slot_tenant[slot];
+    const RouterEntry& r = a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer];
+    const int pool = r.pool;
+    int row_lo = a.cu[p], row_hi = a.cu[p + 1];
+    const int n_p = row_hi - row_lo;
+    if (pool == MILORA_POOL_LAST) row_lo = row_hi - 1;
+    const int n_chunks = chunk_base[p + 1] - chunk_base[p];
+    const int local = it - item_start[p];
+    const bool sa = pool == MILORA_POOL_SELFATTN;
+    const int rc = sa ? local : local / a.n_colblk;
+    const int cb0 = sa ? 0 : local % a.n_colblk;
+    const int cb1 = sa ? a.n_colblk : cb0 + 1;
+    const int r0 = row_lo + rc * kRows;
+    const int nr = min(kRows, row_hi - r0);
+    float* part = a.partial + (size_t)(chunk_base[p] + rc) * d;
+
+    if (sa) {
+      // Appendix C: u_t = H[t,:] . w_sa for the rows of this chunk, then exp weights relative to the chunk max.
+      const T* wsa = static_cast<const T*>(r.Wsa);
+      const int lane = tid & 31, warp = tid >> 5;
+      for (int t = warp; t < nr; t += kThreads / 32) {
+        const T* row = H + (size_t)(r0 + t) * d;
+        float acc = 0.f;
+        for (int c = lane * V; c < d; c += 32 * V) {
+          float hv[V], wv[V];
+          VecOf<T>::load(row + c, hv);
+          VecOf<T>::load(wsa + c, wv);
+#pragma unroll
+          for (int i = 0; i < V; ++i) acc = fmaf(hv[i], wv[i], acc);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) u_sm[t] = acc;
+      }
+      __syncthreads();
+      float m = -FLT_MAX;
+      for (int t = 0; t < nr; ++t) m = fmaxf(m, u_sm[t]);
+      __syncthreads();
+      float l = 0.f;
+      if (tid < nr) u_sm[tid] = expf(u_sm[tid] - m);
+      __syncthreads();
+      for (int t = 0; t < nr; ++t) l += u_sm[t];
+      if (tid == 0) {
+        a.stats[2 * (size_t)(chunk_base[p] + rc)] = m;
+        a.stats[2 * (size_t)(chunk_base[p] + rc) + 1] = l;
+      }
+    }
+
+    for (int cb = cb0; cb < cb1; ++cb) {
+      const int c0 = (cb * kThreads + tid) * V;
+      if (c0 < d) {
+        float acc[V];
+        const bool is_max = pool == MILORA_POOL_MAX;
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = is_max ? -FLT_MAX : 0.f;
+        const T* col = H + (size_t)r0 * d + c0;
+        int t = 0;
+        for (; t + 8 <= nr; t += 8) {
+          float v[8][V];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) VecOf<T>::load(col + (size_t)(t + k) * d, v[k]);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+              if (is_max) acc[i] = fmaxf(acc[i], v[k][i]);
+              else if (sa) acc[i] = fmaf(u_sm[t + k], v[k][i], acc[i]);
+              else acc[i] += v[k][i];
+            }
+          }
+        }
+        for (; t < nr; ++t) {
+          float v[V];
+          VecOf<T>::load(col + (size_t)t * d, v);
+#pragma unroll
+          for (int i = 0; i < V; ++i) {
+            if (is_max) acc[i] = fmaxf(acc[i], v[i]);
+            else if (sa) acc[i] = fmaf(u_sm[t], v[i], acc[i]);
+            else acc[i] += v[i];
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < V; i += 4)
+          *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+      }
+    }
+
+    // ---- completion: the CTA that finishes the prompt's last item combines the partials ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      int n_items = item_start[p + 1] - item_start[p];
+      int old = atomicAdd(a.counters + p, 1);
+      is_last = (old == n_items - 1);
+    }
+    __syncthreads();
+    if (!is_last) continue;
+    __threadfence();
+    const float* part0 = a.partial + (size_t)chunk_base[p] * d;
+    const float* st0 = a.stats + 2 * (size_t)chunk_base[p];
+    float gmax = -FLT_MAX, denom = 1.f;
+    if (sa) {
+      for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, __ldcg(st0 + 2 * c));
+      denom = 0.f;
+      for (int c = 0; c < n_chunks; ++c) denom += expf(__ldcg(st0 + 2 * c) - gmax) * __ldcg(st0 + 2 * c + 1);
+    }
+    const T* W = static_cast<const T*>(r.W);
+    float z[MILORA_NMOD];
+#pragma unroll
+    for (int j = 0; j < MILORA_NMOD; ++j) z[j] = 0.f;
+    for (int c0 = tid * 4; c0 < d; c0 += kThreads * 4) {
+      float h[4];
+      if (pool == MILORA_POOL_MAX) {
+        h[0] = h[1] = h[2] = h[3] = -FLT_MAX;
+      } else {
+        h[0] = h[1] = h[2] = h[3] = 0.f;
+      }
+      for (int c = 0; c < n_chunks; ++c) {
+        float4 q = __ldcg(reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0));
+        if (pool == MILORA_POOL_MAX) {
+          h[0] = fmaxf(h[0], q.x); h[1] = fmaxf(h[1], q.y); h[2] = fmaxf(h[2], q.z); h[3] = fmaxf(h[3], q.w);
+        } else if (sa) {
+          float w = expf(__ldcg(st0 + 2 * c) - gmax);
+          h[0] = fmaf(w, q.x, h[0]); h[1] = fmaf(w, q.y, h[1]); h[2] = fmaf(w, q.z, h[2]); h[3] = fmaf(w, q.w, h[3]);
+        } else {
+          h[0] += q.x; h[1] += q.y; h[2] += q.z; h[3] += q.w;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float hv = h[i];
+        if (pool == MILORA_POOL_MEAN) hv = hv / (float)n_p;
+        else if (sa) hv = hv / denom;
+        float g = activate(hv, r);
+#pragma unroll
+        for (int j = 0; j < MILORA_NMOD; ++j) z[j] = fmaf(g, to_float(W[(size_t)j * d + c0 + i]), z[j]);
+      }
+    }
+    block_sum<MILORA_NMOD>(z, red);
+    if (tid == 0) {
+      float zmax = -FLT_MAX;
+      int best = 0;
+#pragma unroll
+      for (int j = 0; j < MILORA_NMOD; ++j) {
+        z[j] += r.bias[j];
+        if (z[j] > zmax) { zmax = z[j]; best = j; }   // strict: ties keep the lower index
+      }
+      float e[MILORA_NMOD], sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < MILORA_NMOD; ++j) { e[j] = expf(z[j] - zmax); sum += e[j]; }
+      a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = best;
+      if (a.logits_out) {
+#pragma unroll
+        for (int j = 0; j < MILORA_NMOD; ++j) a.logits_out[(size_t)p * MILORA_NMOD + j] = z[j];
+      }
+      if (a.probs_out) {
+#pragma unroll
+        for (int j = 0; j < MILORA_NMOD; ++j) a.probs_out[(size_t)p * MILORA_NMOD + j] = e[j] / sum;
+      }
+      a.counters[p] = 0;
+    }
+    __syncthreads();
+  }
+}
+
+// ---- registration-time repacking -----------------------------------------------------------
+// out[j][i] = in[i][j] for in of shape rows x cols (tiled through shared memory).
+template <typename T>
+__global__ void transpose_kernel(const T* __restrict__ in, T* __restrict__ out, int rows, int cols) {
+  __shared__ T tile[32][33];
+  int c = blockIdx.x * 32 + threadIdx.x;
+  for (int k = threadIdx.y; k < 32; k += blockDim.y) {
+    int rr = blockIdx.y * 32 + k;
+    if (rr < rows && c < cols) tile[k][threadIdx.x] = in[(size_t)rr * cols + c];
+  }
+  __syncthreads();
+  int orow0 = blockIdx.x * 32, ocol = blockIdx.y * 32 + threadIdx.x;
+  for (int k = threadIdx.y; k < 32; k += blockDim.y) {
+    int orow = orow0 + k;
+    if (orow < cols && ocol < rows) out[(size_t)orow * rows + ocol] = tile[threadIdx.x][k];
+  }
+}
+
+template <typename T>
+milora_status transpose(milora_ctx* ctx, const void* in, void* out, int rows, int cols, cudaStream_t s) {
+  dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+  transpose_kernel<T><<<grid, block, 0, s>>>(static_cast<const T*>(in), static_cast<T*>(out), rows, cols);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+}  // namespace
+
+milora_status launch_repack_adapter(milora_ctx* ctx, const void* A, const void* B, void* At, void* Bout, int d1, int d2,
+                                    int rank, cudaStream_t s) {
+  milora_status st = ctx->desc.dtype == MILORA_F32 ? transpose<float>(ctx, A, At, d1, rank, s)
+                                                   : transpose<__nv_bfloat16>(ctx, A, At, d1, rank, s);
+  if (st != MILORA_OK) return st;
+  MILORA_CUDA(ctx, cudaMemcpyAsync(Bout, B, (size_t)rank * d2 * ctx->elem, cudaMemcpyDeviceToDevice, s));
+  return MILORA_OK;
+}
+
+milora_status launch_repack_router(milora_ctx* ctx, const void* Wr, void* Wt, int d, cudaStream_t s) {
+  return ctx->desc.dtype == MILORA_F32 ? transpose<float>(ctx, Wr, Wt, d, MILORA_NMOD, s)
+                                       : transpose<__nv_bfloat16>(ctx, Wr, Wt, d, MILORA_NMOD, s);
+}
+
+milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot, int P,
+                           int T_total, float* logits_out, float* probs_out, cudaStream_t s) {
+  const int d = ctx->desc.d_model;
+  const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
+  const int n_colblk = (d + kThreads * V - 1) / (kThreads * V);
+  const size_t max_chunks = (size_t)T_total / kRows + P;
+  const size_t need = max_chunks * d + 2 * max_chunks;
+  if (need > ctx->scratch_floats) {
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+    if (ctx->d_scratch) MILORA_CUDA(ctx, cudaFree(ctx->d_scratch));
+    ctx->d_scratch = nullptr;
+    ctx->scratch_floats = 0;
+    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_scratch, need * sizeof(float)));
+    ctx->scratch_floats = need;
+  }
+  if ((size_t)P > ctx->n_counters) {
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+    if (ctx->d_counters) MILORA_CUDA(ctx, cudaFree(ctx->d_counters));
+    ctx->d_counters = nullptr;
+    ctx->n_counters = 0;
+    size_t n = std::max<size_t>(P, 1024);
+    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_counters, n * sizeof(int32_t)));
+    MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_counters, 0, n * sizeof(int32_t), s));
+    ctx->n_counters = n;
+  }
+  RouteArgs a;
+  a.tab = device_tables(ctx);
+  a.H = H; a.cu = cu; a.seq_slot = seq_slot;
+  a.logits_out = logits_out; a.probs_out = probs_out;
+  a.partial = ctx->d_scratch;
+  a.stats = ctx->d_scratch + max_chunks * d;
+  a.counters = ctx->d_counters;
+  a.layer = layer; a.P = P; a.d = d; a.n_colblk = n_colblk;
+  size_t max_items = max_chunks * n_colblk;
+  int grid = (int)std::min<size_t>(max_items, (size_t)ctx->sm_count * 4);
+  if (grid < 1) grid = 1;
+  size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
+  if (ctx->desc.dtype == MILORA_F32) {
+    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
+  } else {
+    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
+  }
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+}  // namespace milora

@@ -1,0 +1,265 @@
+"""GPU parity: every step of the hot path, through the C ABI, element by element against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import milora_oracle as O
+from oracle import reference_run as R
+from synth import get_workload
+from synth.workloads import scaled_workload
+
+from parity_utils import assert_apply_close, assert_groups_equal, compare_routes, read_group_block
+
+pytestmark = pytest.mark.gpu
+
+
+def _loaded(w, **kw):
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    return LoadedWorkload(w, "cuda", **kw)
+
+
+def _route_all_layers(lw, ids, **okw):
+    """Route on the GPU and with the oracle; returns (gpu table, oracle table, excused mismatches)."""
+    w = lw.w
+    table_o = np.full((w.n_requests, len(lw.layers)), -1, dtype=np.int32)
+    excused = 0
+    P = len(ids)
+    logits = torch.zeros((P, 7), dtype=torch.float32, device="cuda")
+    probs = torch.zeros((P, 7), dtype=torch.float32, device="cuda")
+    for li, layer in enumerate(lw.layers):
+        lw.route(li, ids, logits=logits, probs=probs)
+        tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+        lo, margins = R.route_requests(w, layer, ids, tmp, **okw)
+        table_o[:, li] = tmp[:, layer]
+        table_g = lw.ml.route_table_read(0, w.n_requests).numpy()
+        excused += compare_routes(table_g[list(ids), li], table_o[list(ids), li], margins)
+        # logits: fp32 accumulation over d terms against fp64
+        lg = logits.cpu().numpy().astype(np.float64)
+        scale = max(1e-3, float(np.abs(lo).max()))
+        assert np.abs(lg - lo).max() <= 2e-4 * scale, "router logits"
+        np.testing.assert_allclose(probs.cpu().numpy(), O.softmax(lo), atol=2e-4)
+    table_g = lw.ml.route_table_read(0, w.n_requests).numpy()
+    return table_g, table_o, excused
+
+
+def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False):
+    """group + apply (prefill and decode lists) on one step; compares grouping and all 7 module outputs."""
+    w, ml = lw.w, lw.ml
+    layer = lw.layers[li]
+    cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
+    n_seq = slots.numel()
+    ws = ml.alloc_group_ws(1, n_seq, T)
+    ml.group(li, 1, cu, slots, n_seq, T, ws)
+    cu_h = cu.cpu().numpy()
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
+    g_o = R.group_layer(w, token_slot, table[:, li])
+    g_o["max_tenants"] = w.n_tenants
+    g_g = read_group_block(ml, ws[0], n_seq, T)
+    assert_groups_equal(g_g, g_o, cu_h)
+    groups = ml.groups(ws[0], n_seq, T)
+    Xs, Ys, Ybs = [], [], []
+    for m in range(7):
+        X = w.module_input(layer, m, T, tag, "cuda")
+        if w.has_base_weights:
+            Yb = (X.float() @ w.base_weight(layer, m, "cuda").float()).to(w.torch_dtype)
+        else:
+            Yb = w.base_output(layer, m, T, tag, "cuda")
+        Xs.append(X); Ybs.append(Yb); Ys.append(Yb.clone())
+    if use_multi:
+        ml.apply_prefill_multi(li, list(range(7)), Xs, Ys, groups)
+        ml.apply_decode_multi(li, list(range(7)), Xs, Ys, groups)
+    else:
+        for m in range(7):
+            ml.apply_prefill(li, m, Xs[m], Ys[m], groups)
+            ml.apply_decode(li, m, Xs[m], Ys[m], groups)
+    torch.cuda.synchronize()
+    worst = 0.0
+    for m in range(7):
+        y_o = R.apply_site(w, layer, m, Xs[m].cpu(), Ybs[m].cpu(), token_slot, table[:, li])
+        worst = max(worst, assert_apply_close(Ys[m], y_o, Ybs[m], w.dtype, what=f"{w.name} layer {layer} module {m}"))
+    assert ml.poll_error() == 0
+    return worst
+
+
+def test_config1_full_path_fp32():
+    """Config 1: route from the prompts, prefill apply, then 4 decode steps that only read the table."""
+    w = get_workload("c1")
+    lw = _loaded(w)
+    ids = list(range(w.n_requests))
+    table_g, table_o, excused = _route_all_layers(lw, ids)
+    assert excused == 0 and np.array_equal(table_g, table_o)
+    for li in range(len(lw.layers)):
+        _step_parity(lw, li, ids, [], table_o, tag=0)
+    before = lw.ml.route_table_read().numpy().copy()
+    for step in range(w.decode_steps):
+        for li in range(len(lw.layers)):
+            _step_parity(lw, li, [], ids, table_o, tag=100 + step, use_multi=(step % 2 == 1))
+    assert np.array_equal(lw.ml.route_table_read().numpy(), before), "decode steps must not touch the route table"
+    lw.close()
+
+
+def test_config1_base_projection_identity():
+    """On the routed module the result equals x (W + s A B) computed by the oracle from the weights."""
+    w = get_workload("c1")
+    lw = _loaded(w)
+    ids = list(range(4))
+    _, table_o, _ = _route_all_layers(lw, ids)
+    li = 0
+    cu, slots, T = lw.seq_arrays(ids, [])
+    ws = lw.ml.alloc_group_ws(1, 4, T)
+    lw.ml.group(li, 1, cu, slots, 4, T, ws)
+    groups = lw.ml.groups(ws[0], 4, T)
+    token_slot = np.repeat(np.arange(4), 16)
+    for m in range(7):
+        X = w.module_input(0, m, T, 5, "cuda")
+        W = w.base_weight(0, m, "cuda")
+        Y = (X @ W).contiguous()
+        lw.ml.apply_prefill(li, m, X, Y, groups)
+        lw.ml.apply_decode(li, m, X, Y, groups)
+        yg = R.to_f64(Y)
+        for t in range(T):
+            slot = token_slot[t]
+            Wm = R.to_f64(W)
+            if table_o[slot, 0] == m:
+                A, B = w.adapter(int(w.request_tenant[slot]), 0, m)
+                Wm = O.merged_weight(Wm, R.to_f64(A), R.to_f64(B), w.scale)
+            ref = R.to_f64(X[t].cpu()) @ Wm
+            assert O.max_rel_err(yg[t], ref) <= 1e-4
+    lw.close()
+
+
+RAGGED = [1, 33, 130, 257, 31, 32, 7, 129]
+
+
+@pytest.mark.parametrize("dtype,d,d_ff,d_kv,r", [("f32", 256, 688, 256, 8), ("bf16", 512, 1376, 128, 16),
+                                                 ("bf16", 256, 688, 256, 40)])
+def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r):
+    """Sequences of 1..257 rows (both work lists, ragged tile tails) mixed with decode rows; tenants repeat so
+    that several sequences share a bucket; one slot is closed and one tenant has no adapters."""
+    base = get_workload("c1")
+    n = len(RAGGED) + 6
+    lens = np.array(RAGGED + [16] * 6, dtype=np.int32)
+    tenants = np.array([0, 1, 2, 0, 1, 3, 2, 0, 0, 1, 1, 2, 3, 0], dtype=np.int32)
+    w = scaled_workload(base, name=f"ragged_{dtype}", dtype=dtype, d_model=d, d_ff=d_ff, d_kv=d_kv, rank=r,
+                        n_tenants=5, request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(len(RAGGED)),
+                        decode_ids=np.arange(len(RAGGED), n), has_base_weights=False, n_layers=2)
+    lw = _loaded(w, tenants=[0, 1, 2, 3])
+    ids = list(range(n))
+    table_g, table_o, excused = _route_all_layers(lw, ids)
+    assert excused <= 1
+    table = table_g.copy()        # use the GPU's decisions downstream so that an excused near tie cannot cascade
+    prefill, decode = list(range(len(RAGGED))), list(range(len(RAGGED), n))
+    for li in range(2):
+        _step_parity(lw, li, prefill, decode, table, tag=7)
+        _step_parity(lw, li, prefill[::-1], decode, table, tag=8, use_multi=True)
+    # close a slot: its rows become excluded and stay bit-identical
+    lw.ml.request_close(3)
+    w.request_tenant = w.request_tenant.copy()
+    w.request_tenant[3] = -1
+    _step_parity(lw, 0, prefill, decode, table, tag=9)
+    lw.close()
+
+
+def test_tenant_without_adapter_is_excluded():
+    base = get_workload("c1")
+    w = scaled_workload(base, n_tenants=6)
+    lw = _loaded(w, register_adapters=False)
+    # tenant 0..3 get routers only; register adapters for tenants 0 and 2 on every module
+    for tenant in (0, 2):
+        for li in range(2):
+            for m in range(7):
+                A, B = w.adapter(tenant, li, m, "cuda")
+                lw.ml.register_adapter(tenant, li, m, A, B, w.scale)
+    ids = list(range(4))
+    table_g, table_o, _ = _route_all_layers(lw, ids)
+    cu, slots, T = lw.seq_arrays(ids, [])
+    ws = lw.ml.alloc_group_ws(1, 4, T)
+    lw.ml.group(0, 1, cu, slots, 4, T, ws)
+    g = read_group_block(lw.ml, ws[0], 4, T)
+    assert g["n_excluded"] == 32 and g["n_active"] == 32
+    token_slot = np.repeat(np.arange(4), 16)
+    g_o = O.group_tokens(token_slot, w.request_tenant, table_o[:, 0], lambda t, m: t in (0, 2), w.n_tenants)
+    assert np.array_equal(g["perm"], g_o["perm"]) and np.array_equal(g["seg_key"], g_o["seg_key"])
+    lw.close()
+
+
+def test_group_edge_cases_and_device_flags():
+    w = get_workload("c1")
+    lw = _loaded(w)
+    ml = lw.ml
+    ids = list(range(4))
+    _route_all_layers(lw, ids)
+    # empty step
+    ws = ml.alloc_group_ws(1, 0, 0)
+    ws.fill_(-7)
+    empty = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ml.group(0, 1, empty, empty, 0, 0, ws)
+    g = read_group_block(ml, ws[0], 0, 0)
+    assert (g["n_seg"], g["n_excluded"], g["n_active"], g["n_tiles"], g["n_gather"]) == (0, 0, 0, 0, 0)
+    assert g["mod_offset"].tolist() == [0] * 8
+    # an out-of-range slot id inside the device array is skipped and flagged, nothing faults
+    slots = torch.tensor([0, 99, 1], dtype=torch.int32, device="cuda")
+    ws = ml.alloc_group_ws(1, 3, 3)
+    ml.group(0, 1, None, slots, 3, 3, ws)
+    g = read_group_block(ml, ws[0], 3, 3)
+    assert g["n_active"] == 2 and g["n_excluded"] == 1
+    assert ml.poll_error() & 1
+    assert ml.poll_error() == 0
+    # zero-length sequences are ignored
+    cu = torch.tensor([0, 0, 5, 5], dtype=torch.int32, device="cuda")
+    slots = torch.tensor([0, 1, 2], dtype=torch.int32, device="cuda")
+    ws = ml.alloc_group_ws(1, 3, 5)
+    ml.group(0, 1, cu, slots, 3, 5, ws)
+    g = read_group_block(ml, ws[0], 3, 5)
+    assert g["n_seg"] == 1 and g["n_active"] == 5 and g["perm"].tolist() == [0, 1, 2, 3, 4]
+    lw.close()
+
+
+@pytest.mark.parametrize("pool,act,bias", [(O.POOL_MAX, O.ACT_RELU, False), (O.POOL_LAST, O.ACT_GELU, True),
+                                            (O.POOL_SELFATTN, O.ACT_RATIONAL, False),
+                                            (O.POOL_MEAN, O.ACT_IDENTITY, True), (O.POOL_SELFATTN, O.ACT_TANH, True)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_router_variants(pool, act, bias, dtype):
+    """All poolers of Eq. 2 / Appendix C and activations incl. Eq. 7, on ragged prompts."""
+    base = get_workload("c1")
+    lens = np.array([1, 5, 64, 65, 200, 333], dtype=np.int32)
+    w = scaled_workload(base, name="router_variants", dtype=dtype, d_model=512, d_ff=1376, d_kv=512, n_tenants=3,
+                        request_tenant=np.array([0, 1, 2, 0, 1, 2], dtype=np.int32), prompt_len=lens,
+                        prefill_ids=np.arange(6), decode_ids=np.zeros(0, dtype=np.int64), has_base_weights=False)
+    lw = _loaded(w, pool=pool, act=act, with_bias=bias, register_adapters=False)
+    _, _, excused = _route_all_layers(lw, list(range(6)), pooler=pool, activation=act, with_bias=bias)
+    assert excused <= 1
+    lw.close()
+
+
+def test_host_validation_reports_errors_before_launch():
+    from paper_2410_18035_b200 import Milora, MiloraError
+    with pytest.raises(MiloraError) as e:
+        Milora(1, 250, 688, 256, "bf16", 8, 4, 4)            # 250 is not a multiple of 8
+    assert e.value.status == 2
+    with pytest.raises(MiloraError) as e:
+        Milora(1, 256, 688, 256, "f32", 300, 4, 4)
+    assert e.value.status == 5
+    ml = Milora(2, 256, 688, 256, "f32", 8, 4, 4)
+    A = torch.zeros((256, 16), device="cuda"); B = torch.zeros((16, 256), device="cuda")
+    with pytest.raises(MiloraError) as e:
+        ml.register_adapter(0, 0, 0, A, B, 1.0)               # rank 16 > max_rank 8
+    assert e.value.status == 5
+    with pytest.raises(MiloraError) as e:
+        ml.request_open(9, 0)
+    assert e.value.status == 1
+    ml.request_open(1, 2)
+    with pytest.raises(MiloraError) as e:
+        ml.request_open(1, 2)
+    assert e.value.status == 6
+    with pytest.raises(MiloraError) as e:
+        ml.unregister_tenant(2)
+    assert e.value.status == 6
+    ml.request_close(1)
+    ml.unregister_tenant(2)
+    with pytest.raises(MiloraError) as e:
+        ml.route_table_write(0, [[7, 0]])
+    assert e.value.status == 1
+    ml.route_table_write(2, [[3, -1]])
+    assert ml.route_table_read(2, 1).tolist() == [[3, -1]]
+    ml.close()
