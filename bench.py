@@ -180,6 +180,7 @@ def run_ours(args, rank, world, device):
     from synth import get_workload
 
     w = get_workload(args.config, seed=rank)          # weak scaling: every rank serves its own tenants' requests
+    w.gen_device = str(device)                        # draw the (multi-GB) inputs with the device generator
     lw = LoadedWorkload(w, device, layers=[0])
     step = Step(lw, device)
     tokens_per_step = step.T_p + step.T_d

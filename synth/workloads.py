@@ -78,6 +78,9 @@ class Workload:
     decode_steps: int = 1
     has_base_weights: bool = False
     note: str = ""
+    # Device whose random-number generator draws every tensor ("cpu" or "cuda").  A tensor is drawn there and
+    # then moved to the device that was asked for, so all users of one workload see the same values.
+    gen_device: str = "cpu"
     _cache: dict = field(default_factory=dict, repr=False)
 
     # ---- structure -------------------------------------------------------
@@ -105,12 +108,12 @@ class Workload:
 
     # ---- tensors ---------------------------------------------------------
     def _normal(self, shape, std: float, kind: str, ids, device, dtype=None):
-        g = torch.Generator(device=device)
+        g = torch.Generator(device=self.gen_device)
         g.manual_seed(tensor_seed(self.seed, _KINDS[kind], *ids))
-        t = torch.randn(shape, generator=g, device=device, dtype=torch.float32)
+        t = torch.randn(shape, generator=g, device=self.gen_device, dtype=torch.float32)
         if std != 1.0:
             t.mul_(std)
-        return t.to(dtype if dtype is not None else self.torch_dtype)
+        return t.to(dtype if dtype is not None else self.torch_dtype).to(device)
 
     def adapter(self, tenant: int, layer: int, module: int, device="cpu"):
         """(A, B): A is d1 x r, B is r x d2 (the orientation of Eq. 1 of the paper)."""
