@@ -42,15 +42,17 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """Samples nvidia-smi clocks and throttle reasons; only samples taken inside the timed region count."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
-    def __init__(self, gpu_index):
-        self.gpu_index = gpu_index
+    def __init__(self, gpu_id):
+        self.gpu_id = gpu_id
         self.proc = None
         self.path = None
+        self.t_begin = self.t_end = None
 
     def start(self):
         try:
@@ -58,39 +60,53 @@ class ClockSampler:
             os.close(fd)
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=self.out,
+                                          "-lms", "20", "-i", str(self.gpu_id)], stdout=self.out,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
+    def region_begin(self):
+        self.t_begin = time.time()
+
+    def region_end(self):
+        self.t_end = time.time()
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
         self.out.close()
-        sm, smax, reasons = [], [], set()
+        import datetime
+        inside, everything, reasons = [], [], set()
+        smax = 0.0
         with open(self.path) as f:
             for line in f:
                 parts = [p.strip() for p in line.split(",")]
-                if len(parts) < 9:
+                if len(parts) < 8:
                     continue
                 try:
-                    sm.append(float(parts[1])); smax.append(float(parts[2]))
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    mhz = float(parts[1])
+                    smax = max(smax, float(parts[2]))
                 except ValueError:
                     continue
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
-                                     parts[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
+                everything.append(mhz)
+                if self.t_begin is not None and self.t_begin - 0.02 <= ts <= self.t_end + 0.02:
+                    inside.append(mhz)
+                    for name, val in zip(self.NAMES, parts[4:8]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
         os.unlink(self.path)
-        if not sm:
+        use = inside if inside else everything
+        if not use:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        return {"sm_mhz": float(np.median(use)), "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples_in_timed_region": len(inside), "samples_total": len(everything)}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -190,12 +206,6 @@ def run_ours(args, rank, world, device):
             torch.distributed.barrier()
         torch.cuda.synchronize(device)
 
-    for _ in range(max(args.warmup, 3)):
-        step.run()
-    barrier()
-    routes = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0]
-    work = algorithmic_work(w, routes, step.prefill_ids, step.decode_ids)
-
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
     except Exception:
@@ -203,15 +213,22 @@ def run_ours(args, rank, world, device):
     sampler = ClockSampler(gpu_id)
     if rank == 0:
         sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+    barrier()
+    routes = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0]
+    work = algorithmic_work(w, routes, step.prefill_ids, step.decode_ids)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     barrier()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    sampler.region_begin()
     t0.record()
     launches = 0
     for k in range(args.steps):
         launches += step.run(evs[k])
     t1.record()
     barrier()
+    sampler.region_end()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t0.elapsed_time(t1)
     phase_ms = np.zeros(5)
@@ -227,7 +244,7 @@ def run_ours(args, rank, world, device):
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
-    e2e = run_e2e(step, args, world, device, tokens_per_step)
+    e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
 
     if rank != 0:
         return None
@@ -273,7 +290,7 @@ def run_ours(args, rank, world, device):
         "gpu_launches": launches,
         "clocks": clocks,
     }
-    out["cpu_baseline"] = cpu_baseline(w, args)
+    out["cpu_baseline"] = None if args.skip_cpu else cpu_baseline(w, args)
     return out
 
 
@@ -390,10 +407,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2")
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
+    ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle timing")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
