@@ -136,6 +136,29 @@ milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const 
                            const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
                            float* probs_out_dev, void* stream);
 
+/* Routing for callers that must not allocate device memory (the paper has no counterpart; this is a
+ * deployment variant of milora_route).  milora_route grows a scratch buffer with cudaMalloc when a batch
+ * is larger than any before it.  That is not possible for a caller that runs inside a serving engine
+ * whose memory pool already owns the whole device, inside a region where the allocator is frozen, or on
+ * a latency path where the implicit device synchronisation of cudaMalloc/cudaFree is not acceptable.
+ * This entry point takes the same arguments and gives the same results, but keeps its scratch (partial
+ * column sums and per-prompt completion counters) in a fixed array inside the library image:
+ *   - the array is 16 MiB + 16 KiB and is held by every GPU that loads the library until the process
+ *     exits;
+ *   - a call needs (T_total / 64 + P) * (d_model + 2) floats of it and P counters; a call that needs
+ *     more than 4 Mi floats, or has P > 4096, is rejected with MILORA_E_CAPACITY before any launch;
+ *   - the first call on a device looks up the array's device address (cudaGetSymbolAddress); the
+ *     context's device must be current (else MILORA_E_STATE), and this first call should be made
+ *     before any stream capture begins;
+ *   - all calls, from every context on that device, share the array: the counters are cleared on
+ *     `stream` at the start of each call, but two calls that overlap on the GPU (different streams)
+ *     race on it, so keep calls of this entry point ordered on one stream;
+ *   - it calls no cudaMalloc, cudaFree or other allocating routine.  Pending table updates made by
+ *     register/open/close calls are still copied to the device first, as in milora_route. */
+milora_status milora_route_static(milora_ctx* ctx, int layer, const void* H_dev, const int32_t* cu_seqlens_dev,
+                                  const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
+                                  float* probs_out_dev, void* stream);
+
 /* Device pointer to the route table, int32 [max_requests][n_layers], read-only for callers. */
 milora_status milora_route_table(const milora_ctx* ctx, const int32_t** table_dev);
 

@@ -57,6 +57,7 @@ SIGNATURES = {
     "milora_request_open": (_I, [_VP, _I, _I]),
     "milora_request_close": (_I, [_VP, _I]),
     "milora_route": (_I, [_VP, _I, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP]),
+    "milora_route_static": (_I, [_VP, _I, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP]),
     "milora_route_table": (_I, [_VP, C.POINTER(_VP)]),
     "milora_route_table_read": (_I, [_VP, _I, _I, _VP, _VP]),
     "milora_route_table_write": (_I, [_VP, _I, _I, _VP, _VP]),
@@ -197,6 +198,23 @@ class Milora:
                 raise ValueError("route: output buffers need P*7 floats")
         self._check(self.lib.milora_route(self.h, layer, _ptr(H), _ptr(cu_seqlens), _ptr(seq_slot), P, H.shape[0],
                                           _ptr(logits_out), _ptr(probs_out), _stream(stream)), "milora_route")
+
+    def route_static(self, layer, H, cu_seqlens, seq_slot, logits_out=None, probs_out=None, stream=None):
+        """milora_route_static: same as route(), with the scratch in the library's fixed device array."""
+        self._tensor(H, self.torch_dtype, "H")
+        self._tensor(cu_seqlens, torch.int32, "cu_seqlens")
+        self._tensor(seq_slot, torch.int32, "seq_slot")
+        self._tensor(logits_out, torch.float32, "logits_out")
+        self._tensor(probs_out, torch.float32, "probs_out")
+        P = seq_slot.numel()
+        if cu_seqlens.numel() != P + 1 or H.shape[1] != self.desc.d_model:
+            raise ValueError("route_static: cu_seqlens must have P+1 entries and H d_model columns")
+        for o in (logits_out, probs_out):
+            if o is not None and o.numel() < P * N_MOD:
+                raise ValueError("route_static: output buffers need P*7 floats")
+        self._check(self.lib.milora_route_static(self.h, layer, _ptr(H), _ptr(cu_seqlens), _ptr(seq_slot), P,
+                                                 H.shape[0], _ptr(logits_out), _ptr(probs_out), _stream(stream)),
+                    "milora_route_static")
 
     def route_table_ptr(self) -> int:
         p = C.c_void_p()

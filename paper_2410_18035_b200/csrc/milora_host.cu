@@ -356,6 +356,21 @@ milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const 
   return launch_route(ctx, layer, H_dev, cu_seqlens_dev, seq_slot_dev, P, T_total, logits_out_dev, probs_out_dev, s);
 }
 
+milora_status milora_route_static(milora_ctx* ctx, int layer, const void* H_dev, const int32_t* cu_seqlens_dev,
+                                  const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
+                                  float* probs_out_dev, void* stream) {
+  if (!ctx) return MILORA_E_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers || P < 0 || T_total < 0) return MILORA_E_ARG;
+  if (P > kMaxSeq) return MILORA_E_CAPACITY;
+  if (P == 0) return MILORA_OK;
+  if (!cu_seqlens_dev || !seq_slot_dev || (T_total > 0 && !H_dev)) return MILORA_E_ARG;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);   // copies pending table updates; allocates nothing
+  if (st != MILORA_OK) return st;
+  return launch_route_static(ctx, layer, H_dev, cu_seqlens_dev, seq_slot_dev, P, T_total, logits_out_dev,
+                             probs_out_dev, s);
+}
+
 milora_status milora_route_table(const milora_ctx* ctx, const int32_t** table_dev) {
   if (!ctx || !table_dev) return MILORA_E_ARG;
   *table_dev = ctx->d_route;

@@ -118,6 +118,8 @@ milora_status launch_repack_adapter(milora_ctx* ctx, const void* A, const void* 
 milora_status launch_repack_router(milora_ctx* ctx, const void* Wr, void* Wt, int d, cudaStream_t s);
 milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot, int P,
                            int T_total, float* logits_out, float* probs_out, cudaStream_t s);
+milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot,
+                                  int P, int T_total, float* logits_out, float* probs_out, cudaStream_t s);
 milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const int32_t* cu, const int32_t* seq_slot,
                            int n_seq, int T, int32_t* ws, size_t ws_stride, cudaStream_t s);
 

@@ -10,6 +10,13 @@
 
 #include "milora_internal.h"
 
+// Scratch of milora_route_static: partial column sums and chunk statistics, followed by one completion
+// counter per prompt.  It lives in the library image, so every GPU that loads the library holds it
+// (16 MiB + 16 KiB) until the process exits, and every call of that entry point shares it.
+constexpr size_t kStaticPartialFloats = size_t(4) << 20;
+constexpr size_t kStaticCounters = 4096;
+static __device__ __align__(256) float g_route_static_scratch[kStaticPartialFloats + kStaticCounters];
+
 namespace milora {
 namespace {
 
@@ -406,6 +413,53 @@ milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int3
   a.partial = ctx->d_scratch;
   a.stats = ctx->d_scratch + max_chunks * d;
   a.counters = ctx->d_counters;
+  a.layer = layer; a.P = P; a.d = d; a.n_colblk = n_colblk;
+  size_t max_items = max_chunks * n_colblk;
+  int grid = (int)std::min<size_t>(max_items, (size_t)ctx->sm_count * 4);
+  if (grid < 1) grid = 1;
+  size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
+  if (ctx->desc.dtype == MILORA_F32) {
+    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
+  } else {
+    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
+  }
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+// Same kernel as launch_route, but the scratch is the file-scope device array above, so that nothing is
+// allocated.  In host code the array's name is only a handle: its device address is looked up once per
+// device with cudaGetSymbolAddress (with that device current) and cached.
+milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot,
+                                  int P, int T_total, float* logits_out, float* probs_out, cudaStream_t s) {
+  constexpr int kMaxDevices = 64;
+  static float* scratch_of_device[kMaxDevices] = {nullptr};
+  const int d = ctx->desc.d_model;
+  const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
+  const int n_colblk = (d + kThreads * V - 1) / (kThreads * V);
+  const size_t max_chunks = (size_t)T_total / kRows + P;
+  const size_t need = max_chunks * d + 2 * max_chunks;
+  if (need > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
+  int dev = -1;
+  MILORA_CUDA(ctx, cudaGetDevice(&dev));
+  if (dev != ctx->device) return MILORA_E_STATE;     // the context's device must be current
+  if (dev < 0 || dev >= kMaxDevices) return MILORA_E_CAPACITY;
+  if (!scratch_of_device[dev]) {
+    float* ptr = nullptr;
+    MILORA_CUDA(ctx, cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_route_static_scratch));
+    scratch_of_device[dev] = ptr;
+  }
+  float* scratch = scratch_of_device[dev];
+  int32_t* counters = reinterpret_cast<int32_t*>(scratch + kStaticPartialFloats);
+  // The array keeps whatever the previous call left; only the counters have to start at zero.
+  MILORA_CUDA(ctx, cudaMemsetAsync(counters, 0, (size_t)P * sizeof(int32_t), s));
+  RouteArgs a;
+  a.tab = device_tables(ctx);
+  a.H = H; a.cu = cu; a.seq_slot = seq_slot;
+  a.logits_out = logits_out; a.probs_out = probs_out;
+  a.partial = scratch;
+  a.stats = scratch + max_chunks * d;
+  a.counters = counters;
   a.layer = layer; a.P = P; a.d = d; a.n_colblk = n_colblk;
   size_t max_items = max_chunks * n_colblk;
   int grid = (int)std::min<size_t>(max_items, (size_t)ctx->sm_count * 4);
