@@ -1,0 +1,325 @@
+// Decode path of Eq. 1 for bf16 on sm_100a: y[row] += s * (x[row] . A) . B for the gathered rows of the
+// decode work list (rows of short sequences, at most kGatherRows per job, all sharing one adapter).
+//
+// The step is bound by streaming each active adapter once from HBM (r * (d1 + d2) * 2 bytes), so the
+// design is about getting every byte requested at once:
+//   * one thread-block cluster of kC CTAs per job; CTA c owns a 1/kC slice of the d1 columns (shrink)
+//     and a 1/kC slice of the d2 columns (expand);
+//   * at start, one warp issues bulk copies (cp.async.bulk, completion on an mbarrier) for the CTA's
+//     slice of B, and every thread loads its 16-byte pieces of y into registers - neither depends on
+//     the shrink result, so they are in flight while x . A is being reduced;
+//   * the A^T slice is consumed straight from global memory with 128-bit loads, four per thread in
+//     flight (it is read once, so staging it in shared memory would only cost occupancy);
+//   * each CTA reduces its d1 slice to partial sums v_c[row][j]; the partials are exchanged through
+//     distributed shared memory and added in CTA order (deterministic), then each CTA finishes its
+//     d2 slice and writes y with 128-bit stores.
+// No scratch in global memory, no atomics.  Every wait is bounded; a timeout raises ERR_WAIT_TIMEOUT.
+#include "milora_internal.h"
+
+namespace milora {
+namespace {
+
+constexpr int kC = 8;              // CTAs per cluster (portable maximum)
+constexpr int kThreads = 256;
+constexpr int kR = kGatherRows;
+constexpr int kSegs = 16;          // threads that share one rank row in the shrink
+constexpr int kRowsPerPass = kThreads / kSegs;
+constexpr uint32_t kSpinLimit = 4u << 20;
+constexpr int kYIter = 4;          // 16-byte pieces of y a thread may own (kR * per2max <= kYIter * kThreads)
+constexpr int kUnroll = 4;         // A^T loads a thread keeps in flight
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; returns false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t peer, float v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 q;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
+               : "l"(p));
+  return q;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& q, float (&v)[8]) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float (&v)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+struct DecodeArgs {
+  int32_t* err;
+  ApplySites sites;
+  const int32_t* ws;
+  milora_group_layout_t lay;
+  int T;
+  int rmax;        // rank rows reserved in shared memory
+  int per2max;     // 16-byte column groups reserved per row of the B staging
+};
+
+// Shared memory (dynamic): [0,16) mbarrier | part[kC][kR][rmax] f32 | mine[kR][rmax] f32 | v[kR][rmax] f32 |
+//                          B[rmax][per2max] uint4
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode_bf16_kernel(DecodeArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t crank = cluster_ctarank();
+  const int job_idx = blockIdx.x / kC;
+  const int n_jobs = a.ws[a.lay.header + H_NGATHER];
+  if (job_idx >= n_jobs || job_idx >= a.lay.max_gather) return;          // same decision in the whole cluster
+  const GatherJob job = reinterpret_cast<const GatherJob*>(a.ws + a.lay.gather)[job_idx];
+  int si = -1;
+#pragma unroll
+  for (int i = 0; i < kMaxSites; ++i)
+    if (i < a.sites.n && a.sites.site[i].module == job.module) si = i;
+  if (si < 0) return;
+  const int r = job.rank;
+  const int n = min(job.count, kR);
+  bool bad = r <= 0 || r > a.rmax || n <= 0 || !job.At || !job.B;
+  int rows[kR];
+#pragma unroll
+  for (int t = 0; t < kR; ++t) {
+    rows[t] = (t < n) ? job.rows[t] : -1;
+    if (t < n && (rows[t] < 0 || rows[t] >= a.T)) bad = true;
+  }
+  if (bad) {
+    if (tid == 0 && crank == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  const ApplySite& site = a.sites.site[si];
+  const int d1 = site.d1, d2 = site.d2;
+  const int nv1 = d1 >> 3, nv2 = d2 >> 3;                 // 16-byte column groups per row
+  const int per1 = (nv1 + kC - 1) / kC, per2 = (nv2 + kC - 1) / kC;
+  const int lo1 = min((int)crank * per1, nv1), cnt1 = min(per1, nv1 - lo1);
+  const int lo2 = min((int)crank * per2, nv2), cnt2 = min(per2, nv2 - lo2);
+  const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(site.X);
+  __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(site.Y);
+  const __nv_bfloat16* At = static_cast<const __nv_bfloat16*>(job.At);
+
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+  float* part = reinterpret_cast<float*>(smem + 16);                        // [kC][kR][rmax]
+  float* mine = part + kC * kR * a.rmax;                                    // [kR][rmax]
+  float* v_sm = mine + kR * a.rmax;                                         // [kR][rmax]
+  uint4* B_sm = reinterpret_cast<uint4*>(v_sm + kR * a.rmax);               // [rmax][per2max]
+  const uint32_t bar = smem_u32(&bars[0]);
+
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  cluster_arrive();       // "this CTA is running"; waited for right before the first remote store
+
+  // ---- B slice by bulk copies, y pieces into registers: nothing here depends on the shrink ------
+  if (warp == 0) {
+    const char* Bm = static_cast<const char*>(job.B);
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)r * cnt2 * 16u);
+    __syncwarp();
+    if (cnt2 > 0) {
+      for (int i = lane; i < r; i += 32)
+        bulk_g2s(smem_u32(B_sm + (size_t)i * a.per2max), Bm + ((size_t)i * d2 + lo2 * 8) * 2, cnt2 * 16, bar);
+    }
+  }
+  uint4 ypre[kYIter];
+#pragma unroll
+  for (int it = 0; it < kYIter; ++it) {
+    const int idx = tid + it * kThreads;
+    ypre[it] = make_uint4(0, 0, 0, 0);
+    if (idx < n * cnt2) {
+      const int t = idx / cnt2, g = idx % cnt2;
+      int row = rows[0];
+#pragma unroll
+      for (int q = 1; q < kR; ++q) row = (t == q) ? rows[q] : row;
+      ypre[it] = *reinterpret_cast<const uint4*>(Y + (size_t)row * d2 + (size_t)(lo2 + g) * 8);
+    }
+  }
+
+  // ---- shrink: partial v over this CTA's d1 slice, A^T straight from global memory -------------------
+  const int seg = tid % kSegs;
+  for (int j0 = 0; j0 < r; j0 += kRowsPerPass) {
+    const int j = j0 + tid / kSegs;
+    float acc[kR];
+#pragma unroll
+    for (int t = 0; t < kR; ++t) acc[t] = 0.f;
+    if (j < r) {
+      const __nv_bfloat16* arow = At + (size_t)j * d1 + (size_t)lo1 * 8;
+      for (int v0 = seg; v0 < cnt1; v0 += kSegs * kUnroll) {
+        uint4 aq[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          const int v = v0 + u * kSegs;
+          aq[u] = (v < cnt1) ? ldg_stream(arow + (size_t)v * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int t = 0; t < kR; ++t) {
+          if (t < n) {
+            const __nv_bfloat16* xrow = X + (size_t)rows[t] * d1 + (size_t)lo1 * 8;
+            uint4 xq[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+              const int v = v0 + u * kSegs;
+              xq[u] = (v < cnt1) ? *reinterpret_cast<const uint4*>(xrow + (size_t)v * 8) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+              float av[8], xv[8];
+              unpack8(aq[u], av);
+              unpack8(xq[u], xv);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) acc[t] = fmaf(xv[i], av[i], acc[t]);
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < kR; ++t) {
+#pragma unroll
+      for (int o = kSegs / 2; o > 0; o >>= 1) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], o);
+    }
+    if (seg == 0 && j < r) {
+#pragma unroll
+      for (int t = 0; t < kR; ++t) mine[t * a.rmax + j] = acc[t];
+    }
+  }
+  __syncthreads();
+  cluster_wait();         // every CTA of the cluster has started, so its shared memory can be written
+  // hand this CTA's partial sums to every CTA of the cluster (slot `crank` of their `part`), one store per thread
+  for (int idx = tid; idx < n * r * kC; idx += kThreads) {
+    const int peer = idx % kC, e = idx / kC, t = e / r, j = e % r;
+    st_cluster_f32(smem_u32(part + ((size_t)crank * kR + t) * a.rmax + j), (uint32_t)peer, mine[t * a.rmax + j]);
+  }
+  cluster_sync_all();     // all partial sums have landed everywhere; nobody writes remote memory after this
+
+  for (int idx = tid; idx < n * r; idx += kThreads) {
+    const int t = idx / r, j = idx % r;
+    float s = 0.f;
+#pragma unroll
+    for (int c = 0; c < kC; ++c) s += part[((size_t)c * kR + t) * a.rmax + j];
+    v_sm[t * a.rmax + j] = s * job.scale;
+  }
+  __syncthreads();
+
+  // ---- expand: this CTA's d2 slice ------------------------------------------------------------
+  if (!mbar_wait(bar, 0)) {
+    if (tid == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
+    mbar_wait(bar, 0);    // a second, equally bounded, chance for copies still in flight before leaving
+    return;
+  }
+#pragma unroll
+  for (int it = 0; it < kYIter; ++it) {
+    const int idx = tid + it * kThreads;
+    if (idx < n * cnt2) {
+      const int t = idx / cnt2, g = idx % cnt2;
+      float out[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) out[i] = 0.f;
+      for (int j = 0; j < r; ++j) {
+        float bv[8];
+        unpack8(B_sm[(size_t)j * a.per2max + g], bv);
+        const float vj = v_sm[t * a.rmax + j];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = fmaf(vj, bv[i], out[i]);
+      }
+      float yv[8];
+      unpack8(ypre[it], yv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) yv[i] += out[i];
+      int row = rows[0];
+#pragma unroll
+      for (int q = 1; q < kR; ++q) row = (t == q) ? rows[q] : row;
+      *reinterpret_cast<uint4*>(Y + (size_t)row * d2 + (size_t)(lo2 + g) * 8) = pack8(yv);
+    }
+  }
+}
+
+}  // namespace
+
+milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                       cudaStream_t s) {
+  (void)layer;
+  if (ctx->desc.dtype != MILORA_BF16) return MILORA_E_SHAPE;
+  DecodeArgs a;
+  a.err = ctx->d_err;
+  a.sites = sites;
+  a.ws = g->ws_dev;
+  a.lay = group_layout(g->n_seq, g->T);
+  a.T = g->T;
+  a.rmax = (ctx->desc.max_rank + 3) & ~3;
+  int per2 = 0;
+  for (int i = 0; i < sites.n; ++i) {
+    const ApplySite& st = sites.site[i];
+    if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (reinterpret_cast<uintptr_t>(st.Y) & 15)) return MILORA_E_SHAPE;
+    per2 = std::max(per2, (st.d2 / 8 + kC - 1) / kC);
+  }
+  if (kR * per2 > kYIter * kThreads) return MILORA_E_SHAPE;
+  a.per2max = per2;
+  size_t smem = 16 + (size_t)(kC + 2) * kR * a.rmax * sizeof(float) + (size_t)a.rmax * per2 * 16;
+  if (smem > 200 * 1024) return MILORA_E_SHAPE;
+  if (smem > 48 * 1024) {
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(decode_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  }
+  size_t grid = (size_t)a.lay.max_gather * kC;
+  if (grid > 0x7fffffffull) return MILORA_E_CAPACITY;
+  decode_bf16_kernel<<<(unsigned)grid, kThreads, smem, s>>>(a);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+}  // namespace milora

@@ -17,6 +17,7 @@ namespace {
 constexpr int kGThreads = 1024;
 constexpr int kSeqBits = 12;  // kMaxSeq = 4096 sequences
 static_assert((1 << kSeqBits) == kMaxSeq, "kSeqBits must match kMaxSeq");
+constexpr int kSmemArrays = 8;
 
 // Exclusive prefix sum over the block of one int per thread; returns the exclusive value, *total gets the sum.
 __device__ inline int block_exscan(int v, int* total, int* wsum /* [33] */) {
@@ -56,16 +57,17 @@ struct GroupArgs {
   int layer_begin, n_seq, n_pad, T;
 };
 
-// Shared memory: comp[n_pad], tok_off[n_pad+1], seg_of[n_pad], seg_tile[n_pad+1], seg_short[n_pad+1],
-// seg_gather[n_pad+1].
+// Shared memory (int32): comp[n_pad], seq_lo[n_pad], seq_len[n_pad], tok_off[n_pad+1], seg_tile[n_pad+1],
+// seg_short[n_pad+1], seg_gather[n_pad+1] (kSmemArrays * n_pad + 8 in total).
 __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
   extern __shared__ int32_t sm[];
   __shared__ int wsum[33];
   const int n_pad = a.n_pad, n_seq = a.n_seq;
   int32_t* comp = sm;
-  int32_t* tok_off = comp + n_pad;
-  int32_t* seg_of = tok_off + n_pad + 1;
-  int32_t* seg_tile = seg_of + n_pad;
+  int32_t* seq_lo = comp + n_pad;
+  int32_t* seq_len = seq_lo + n_pad;
+  int32_t* tok_off = seq_len + n_pad;
+  int32_t* seg_tile = tok_off + n_pad + 1;
   int32_t* seg_short = seg_tile + n_pad + 1;
   int32_t* seg_gather = seg_short + n_pad + 1;
   const int tid = threadIdx.x;
@@ -73,21 +75,18 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
   int32_t* ws = a.ws + (size_t)blockIdx.x * a.ws_stride;
   const int max_tenants = a.tab.max_tenants;
 
-  auto seq_rows = [&](int i, int* lo, int* hi) {
-    if (a.cu) { *lo = a.cu[i]; *hi = a.cu[i + 1]; }
-    else { *lo = i; *hi = i + 1; }
-  };
-
   // ---- 1. composite keys, excluded-token count --------------------------------------------
   int excl = 0;
   for (int i = tid; i < n_pad; i += kGThreads) {
     int c = INT_MAX;
     if (i < n_seq) {
-      int lo, hi;
-      seq_rows(i, &lo, &hi);
+      int lo = i, hi = i + 1;
+      if (a.cu) { lo = a.cu[i]; hi = a.cu[i + 1]; }
       bool rows_ok = lo >= 0 && hi >= lo && hi <= a.T;
       if (!rows_ok) atomicOr(a.tab.err, ERR_BAD_ROW);
       int len = rows_ok ? hi - lo : 0;
+      seq_lo[i] = lo;
+      seq_len[i] = len;
       int slot = a.seq_slot[i];
       bool ok = slot >= 0 && slot < a.tab.max_requests;
       if (!ok) atomicOr(a.tab.err, ERR_BAD_SLOT);
@@ -125,26 +124,26 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
 
   // ---- 3. per-sequence quantities in sorted order; each thread owns consecutive positions ----
   const int per = (n_pad + kGThreads - 1) / kGThreads;
-  const int j0 = tid * per, j1 = min(j0 + per, n_pad);
-  int s_tok = 0, s_head = 0, s_tile = 0, s_short = 0;
+  const int j0 = min(tid * per, n_pad), j1 = min(j0 + per, n_pad);
+  int s_tok = 0, s_head = 0, s_tile = 0, s_short = 0, s_act = 0;
   for (int j = j0; j < j1; ++j) {
     int c = comp[j];
     if (c == INT_MAX) break;
-    int lo, hi;
-    seq_rows(c & (kMaxSeq - 1), &lo, &hi);
-    int len = hi - lo;
+    int len = seq_len[c & (kMaxSeq - 1)];
+    s_act += 1;
     s_tok += len;
     s_head += (j == 0 || (comp[j - 1] >> kSeqBits) != (c >> kSeqBits)) ? 1 : 0;
     if (len >= kLongSeq) s_tile += (len + kTileRows - 1) / kTileRows;
     else s_short += len;
   }
-  int n_active, n_seg, n_tiles, n_short;
+  int n_active, n_seg, n_tiles, n_short, n_act_seq;
   int o_tok = block_exscan(s_tok, &n_active, wsum);
   int o_head = block_exscan(s_head, &n_seg, wsum);
   int o_tile = block_exscan(s_tile, &n_tiles, wsum);
   int o_short = block_exscan(s_short, &n_short, wsum);
+  block_exscan(s_act, &n_act_seq, wsum);
 
-  WorkItem* tiles = reinterpret_cast<WorkItem*>(ws + a.lay.tiles);
+  TileJob* tiles = reinterpret_cast<TileJob*>(ws + a.lay.tiles);
   int32_t* gather_rows = ws + a.lay.gather_rows;
   int32_t* seg_key = ws + a.lay.seg_key;
   int32_t* seg_offset = ws + a.lay.seg_offset;
@@ -152,9 +151,7 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
     int c = comp[j];
     if (c == INT_MAX) break;
     int key = c >> kSeqBits;
-    int lo, hi;
-    seq_rows(c & (kMaxSeq - 1), &lo, &hi);
-    int len = hi - lo;
+    int lo = seq_lo[c & (kMaxSeq - 1)], len = seq_len[c & (kMaxSeq - 1)];
     bool head = (j == 0 || (comp[j - 1] >> kSeqBits) != key);
     if (head) {
       seg_key[o_head] = key;
@@ -164,13 +161,17 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
       ++o_head;
     }
     const int seg = o_head - 1;
-    seg_of[j] = seg;
     tok_off[j] = o_tok;
     o_tok += len;
     if (len >= kLongSeq) {
+      const int module = key / max_tenants;
+      const AdapterEntry e = a.tab.adapters[adapter_index(key % max_tenants, layer, module, a.tab.n_layers)];
+      TileJob w;
+      w.At = e.At; w.B = e.B; w.At_img = e.At_img; w.B_img = e.B_img;
+      w.rank = e.rank; w.scale = e.scale; w.module = module; w.seg = seg; w.rank_pad = e.rank_pad; w.pad = 0;
       for (int r = 0; r < len; r += kTileRows) {
-        WorkItem w;
-        w.seg = seg; w.start = lo + r; w.count = min(kTileRows, len - r); w.module = key / max_tenants;
+        w.start = lo + r;
+        w.count = min(kTileRows, len - r);
         tiles[o_tile++] = w;
       }
     } else {
@@ -181,16 +182,8 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
     seg_offset[n_seg] = n_active;
     seg_tile[n_seg] = n_tiles;
     seg_short[n_seg] = n_short;
+    tok_off[n_act_seq] = n_active;
   }
-  // number of sorted (active) sequences = first sentinel
-  __syncthreads();
-  int n_act_seq;
-  {
-    int cnt = 0;
-    for (int j = j0; j < j1; ++j) cnt += comp[j] != INT_MAX;
-    block_exscan(cnt, &n_act_seq, wsum);
-  }
-  if (tid == 0) tok_off[n_act_seq] = n_active;
   __syncthreads();
 
   // ---- 4. perm: token q of the sorted order ------------------------------------------------
@@ -201,26 +194,30 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
       int mid = (lo + hi) >> 1;
       if (tok_off[mid] <= q) lo = mid; else hi = mid;
     }
-    int rlo, rhi;
-    seq_rows(comp[lo] & (kMaxSeq - 1), &rlo, &rhi);
-    perm[q] = rlo + (q - tok_off[lo]);
+    perm[q] = seq_lo[comp[lo] & (kMaxSeq - 1)] + (q - tok_off[lo]);
   }
 
-  // ---- 5. gather entries: chunks of kGatherRows short rows per segment ------------------------
+  // ---- 5. gather jobs: chunks of kGatherRows short rows per segment ---------------------------
   const int sper = (n_seg + kGThreads - 1) / kGThreads;
   const int s0 = min(tid * sper, n_seg), s1 = min(s0 + sper, n_seg);
   int g_cnt = 0;
   for (int s = s0; s < s1; ++s) g_cnt += (seg_short[s + 1] - seg_short[s] + kGatherRows - 1) / kGatherRows;
   int n_gather;
   int o_g = block_exscan(g_cnt, &n_gather, wsum);
-  WorkItem* gather = reinterpret_cast<WorkItem*>(ws + a.lay.gather);
+  GatherJob* gather = reinterpret_cast<GatherJob*>(ws + a.lay.gather);
   for (int s = s0; s < s1; ++s) {
     seg_gather[s] = o_g;
-    int b = seg_short[s], e = seg_short[s + 1];
-    int module = seg_key[s] / max_tenants;
+    const int b = seg_short[s], e = seg_short[s + 1];
+    if (b == e) continue;
+    const int key = seg_key[s];
+    const int module = key / max_tenants;
+    const AdapterEntry ent = a.tab.adapters[adapter_index(key % max_tenants, layer, module, a.tab.n_layers)];
+    GatherJob w;
+    w.At = ent.At; w.B = ent.B; w.rank = ent.rank; w.scale = ent.scale; w.module = module; w.seg = s; w.pad = 0;
     for (int r = b; r < e; r += kGatherRows) {
-      WorkItem w;
-      w.seg = s; w.start = r; w.count = min(kGatherRows, e - r); w.module = module;
+      w.count = min(kGatherRows, e - r);
+#pragma unroll
+      for (int t = 0; t < kGatherRows; ++t) w.rows[t] = (t < w.count) ? gather_rows[r + t] : -1;
       gather[o_g++] = w;
     }
   }
@@ -263,7 +260,7 @@ milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   int n_pad = 2;
   while (n_pad < n_seq) n_pad <<= 1;
   a.n_pad = n_pad;
-  size_t smem = ((size_t)n_pad * 6 + 4) * sizeof(int32_t);
+  size_t smem = ((size_t)n_pad * kSmemArrays + 8) * sizeof(int32_t);
   if (smem > 48 * 1024) {
     MILORA_CUDA(ctx, cudaFuncSetAttribute(group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }

@@ -63,10 +63,10 @@ milora_group_layout_t group_layout(int n_seq, int T) {
   L.seg_offset = o; o += round4((size_t)n_seq + 1);
   L.perm = o; o += round4((size_t)T);
   L.max_tiles = T / kTileRows + n_seq;
-  L.tiles = o; o += (size_t)L.max_tiles * 4;
+  L.tiles = o; o += (size_t)L.max_tiles * kJobInts;
   L.gather_rows = o; o += round4((size_t)T);
   L.max_gather = T / kGatherRows + n_seq + 1;
-  L.gather = o; o += (size_t)L.max_gather * 4;
+  L.gather = o; o += (size_t)L.max_gather * kJobInts;
   L.total = round4(o);
   return L;
 }
@@ -157,6 +157,7 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->elem = desc->dtype == MILORA_F32 ? 4 : 2;
   ctx->d_adapters = nullptr; ctx->d_routers = nullptr; ctx->d_slot_tenant = nullptr; ctx->d_route = nullptr;
   ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
+  ctx->d_vscratch = nullptr; ctx->vscratch_floats = 0;
   ctx->n_counters = 0;
   milora_status st = MILORA_OK;
   auto fail = [&](milora_status s) { milora_destroy(ctx); return s; };
@@ -167,7 +168,9 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   size_t n_ad = (size_t)desc->max_tenants * desc->n_layers * MILORA_NMOD;
   size_t n_rt = (size_t)desc->max_tenants * desc->n_layers;
   try {
-    ctx->h_adapters.assign(n_ad, AdapterEntry{nullptr, nullptr, 0, 0.f, {0, 0}});
+    AdapterEntry a0;
+    std::memset(&a0, 0, sizeof(a0));
+    ctx->h_adapters.assign(n_ad, a0);
     RouterEntry r0;
     std::memset(&r0, 0, sizeof(r0));
     ctx->h_routers.assign(n_rt, r0);
@@ -210,6 +213,7 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_err);
   cudaFree(ctx->d_scratch);
   cudaFree(ctx->d_counters);
+  cudaFree(ctx->d_vscratch);
   ctx->arena.release();
   delete ctx;
   return MILORA_OK;
@@ -451,6 +455,10 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
   cudaStream_t s = as_stream(stream);
   milora_status st = sync_tables(ctx, s);
   if (st != MILORA_OK) return st;
+  if (!dense && ctx->desc.dtype == MILORA_BF16) {
+    st = launch_apply_decode_bf16(ctx, layer, sites, groups, s);
+    if (st != MILORA_E_SHAPE) return st;     // MILORA_E_SHAPE: this batch does not fit the cluster kernel
+  }
   return launch_apply_generic(ctx, layer, sites, groups, dense, s);
 }
 

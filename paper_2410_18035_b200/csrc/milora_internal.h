@@ -13,16 +13,21 @@
 namespace milora {
 
 // ---- device-visible tables -------------------------------------------------------------
-// One LoRA pair in library layout: At is rank x d1 (W^A transposed), B is rank x d2, both
-// row-major in the context dtype and 256-byte aligned.
+// One LoRA pair in library layout.  At is rank x d1 (W^A transposed), B is rank x d2, both row-major
+// in the context dtype and 256-byte aligned.  At_img / B_img are the same matrices cut into the
+// shared-memory operand images the tensor-core kernels fetch with one bulk copy per chunk (bf16
+// contexts whose dimensions allow it; nullptr otherwise).
 struct AdapterEntry {
   const void* At;
   const void* B;
-  int32_t rank;   // 0 = not registered
+  const void* At_img;
+  const void* B_img;
+  int32_t rank;      // 0 = not registered
   float scale;
-  int32_t pad[2];
+  int32_t rank_pad;  // rank rounded up to a multiple of 16 (rows of the operand images)
+  int32_t pad[5];
 };
-static_assert(sizeof(AdapterEntry) == 32, "AdapterEntry must stay 32 bytes");
+static_assert(sizeof(AdapterEntry) == 64, "AdapterEntry must stay 64 bytes");
 
 // Router of one (tenant, layer): W is 7 x d (W_r transposed), context dtype.
 struct RouterEntry {
@@ -33,18 +38,36 @@ struct RouterEntry {
   int32_t pool, act, n_a, n_b;
 };
 
-// Work-list entry written by the grouping kernel (4 int32): a dense tile is `count` consecutive
-// rows starting at `start`; a gather entry is `count` rows listed at gather_rows[start ...].
-struct WorkItem {
-  int32_t seg, start, count, module;
-};
-
 constexpr int kHeaderInts = 16;
 constexpr int kTileRows = 128;     // rows per dense tile (prefill path)
-constexpr int kGatherRows = 8;     // rows per gather entry (decode path)
+constexpr int kGatherRows = 4;     // rows per gather job (decode path)
 constexpr int kLongSeq = 32;       // sequences of at least this many tokens go to dense tiles
 constexpr int kMaxSeq = 4096;      // sequences per grouping / routing call
+constexpr int kJobInts = 16;       // every job record is 64 bytes
 enum HeaderSlot { H_NSEG = 0, H_NEXCL = 1, H_NACTIVE = 2, H_NTILES = 3, H_NGATHER = 4 };
+
+// Work records written by the grouping kernel.  They carry the adapter pointers, so an apply kernel
+// needs one 64-byte load to know its whole job.  They stay valid until an adapter of the batch is
+// registered again or a slot of the batch is closed.
+struct GatherJob {       // up to kGatherRows rows anywhere in X / Y that share an adapter
+  const void* At;
+  const void* B;
+  int32_t rank;
+  float scale;
+  int32_t module, count, seg, pad;
+  int32_t rows[kGatherRows];
+  int32_t pad2[2];
+};
+struct TileJob {         // `count` consecutive rows starting at `start`
+  const void* At;
+  const void* B;
+  const void* At_img;
+  const void* B_img;
+  int32_t rank;
+  float scale;
+  int32_t module, count, seg, start, rank_pad, pad;
+};
+static_assert(sizeof(GatherJob) == 64 && sizeof(TileJob) == 64, "job records are 64 bytes");
 
 // Device error flag bits.
 enum ErrBit { ERR_BAD_SLOT = 1, ERR_BAD_ROW = 2, ERR_WAIT_TIMEOUT = 4, ERR_BAD_ITEM = 8 };
@@ -93,6 +116,8 @@ struct milora_ctx {
   size_t scratch_floats;
   int32_t* d_counters;                          // router completion counters, one per prompt
   size_t n_counters;
+  float* d_vscratch;                            // prefill: fp32 partial x.A products [k-split][T][rank_pad]
+  size_t vscratch_floats;
   milora::Arena arena;
   std::string cuda_error;
 };
@@ -137,5 +162,9 @@ struct ApplySites {
 // Generic SIMT path (any dtype, any shape): gathered rows (decode) or dense tiles (prefill).
 milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
                                    bool dense, cudaStream_t s);
+// bf16 decode path: one cluster of CTAs per gather job, bulk-copy staging, DSMEM reduction.
+// Returns MILORA_E_SHAPE when shapes or alignment do not fit it (the caller then uses the generic path).
+milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                       cudaStream_t s);
 
 }  // namespace milora

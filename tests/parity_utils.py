@@ -77,15 +77,21 @@ def read_group_block(ml, ws_layer: torch.Tensor, n_seq: int, T: int):
         "seg_key": ws[lay.seg_key:lay.seg_key + n_seg].copy(),
         "seg_offset": ws[lay.seg_offset:lay.seg_offset + n_seg + 1].copy(),
         "perm": ws[lay.perm:lay.perm + n_active].copy(),
-        "tiles": ws[lay.tiles:lay.tiles + 4 * n_tiles].reshape(-1, 4).copy(),
-        "gather": ws[lay.gather:lay.gather + 4 * n_gather].reshape(-1, 4).copy(),
-        "gather_rows": ws[lay.gather_rows:lay.gather_rows + T].copy(),
         "layout": lay,
     }
+    # job records are 16 int32 each: two / four 64-bit pointers first, then the integer fields
+    tiles = ws[lay.tiles:lay.tiles + 16 * n_tiles].reshape(-1, 16)
+    gather = ws[lay.gather:lay.gather + 16 * n_gather].reshape(-1, 16)
+    # (seg, start, count, module) per dense tile
+    out["tiles"] = np.stack([tiles[:, 12], tiles[:, 13], tiles[:, 11], tiles[:, 10]], axis=1) if n_tiles else np.zeros((0, 4), int)
+    out["tile_rank"] = tiles[:, 8].copy()
+    # (seg, count, module, rows[4]) per gather job
+    out["gather"] = [(int(g[8]), int(g[7]), int(g[6]), [int(v) for v in g[10:14]]) for g in gather]
+    out["gather_rank"] = gather[:, 4].copy()
     return out
 
 
-def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_rows=8):
+def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_rows=4):
     """perm / seg_key / seg_offset / mod_offset / n_excluded are compared bit for bit; the work lists must
     cover every active row exactly once, dense tiles with consecutive rows of long sequences only."""
     assert g_gpu["n_excluded"] == g_oracle["n_excluded"]
@@ -111,9 +117,10 @@ def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_
         assert all(seg_of_row[r] == seg for r in rows)
         assert module == g_gpu["seg_key"][seg] // (g_oracle["max_tenants"])
         covered += rows
-    for seg, start, count, module in g_gpu["gather"]:
+    for seg, count, module, job_rows in g_gpu["gather"]:
         assert 1 <= count <= gather_rows
-        rows = [int(r) for r in g_gpu["gather_rows"][start:start + count]]
+        rows = job_rows[:count]
+        assert all(r == -1 for r in job_rows[count:])
         assert all(seg_of_row[r] == seg and seq_len[seq_of_row[r]] < long_seq for r in rows)
         assert module == g_gpu["seg_key"][seg] // (g_oracle["max_tenants"])
         covered += rows
@@ -122,5 +129,5 @@ def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_
         t0, t1 = g_gpu["mod_tile_offset"][m], g_gpu["mod_tile_offset"][m + 1]
         assert all(row[3] == m for row in g_gpu["tiles"][t0:t1])
         q0, q1 = g_gpu["mod_gather_offset"][m], g_gpu["mod_gather_offset"][m + 1]
-        assert all(row[3] == m for row in g_gpu["gather"][q0:q1])
+        assert all(job[2] == m for job in g_gpu["gather"][q0:q1])
     assert g_gpu["mod_tile_offset"][7] == g_gpu["n_tiles"] and g_gpu["mod_gather_offset"][7] == g_gpu["n_gather"]
