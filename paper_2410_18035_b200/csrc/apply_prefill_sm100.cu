@@ -1,0 +1,523 @@
+// Prefill path of Eq. 1 for bf16 on sm_100a: Y[rows] += s * (X[rows] . A) . B for dense tiles of up to
+// 128 consecutive prompt rows that share one adapter.  Both contractions run on the 5th-generation
+// tensor cores (tcgen05.mma, accumulators in tensor memory); the op as a whole is bound by streaming
+// X once and reading and writing Y once, so the kernels are organised around keeping HBM busy:
+//
+//   shrink kernel  V_k[rows][r] = X[rows][k-slice] . A[k-slice][r]      one CTA per (tile, k-slice)
+//     X tiles arrive by TMA (128-byte swizzle) and the matching A chunks by one bulk copy each
+//     (the library keeps A pre-cut into shared-memory operand images) through a 6-stage ring;
+//     one thread issues 128 x r x 16 MMAs; the fp32 partial result goes to a small scratch.
+//   expand kernel  Y[rows][n-slice] += s * (sum_k V_k) . B[r][n-slice]   one CTA per (tile, n-slice)
+//     the summed V (rounded to bf16) is the shared-memory A operand; per 128-column chunk a TMA load
+//     brings Y and a bulk copy brings the B image, one MMA chain writes the delta to tensor memory
+//     (double buffered), the epilogue warps add it to Y in shared memory and a TMA store writes it
+//     back.  Tiles with fewer than 128 rows store their rows with plain 128-bit stores instead, so
+//     rows of neighbouring sequences are never touched.
+//
+// Splitting k and n over CTAs keeps all SMs busy even when a call covers only a few tiles; the partial
+// sums are added in k order, so the result does not depend on scheduling.  Every wait is bounded.
+#include <cuda.h>
+
+#include "milora_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace milora {
+namespace {
+
+using namespace ptx;
+
+constexpr int kKSplit = 4;            // k-slices of the shrink
+constexpr int kNSplit = 4;            // n-slices of the expand
+constexpr int kBK = 64;               // k elements per shrink stage (128 bytes: one swizzle row)
+constexpr int kBN = 128;              // y columns per expand chunk
+constexpr int kRPadMax = 64;          // largest padded rank this path takes
+constexpr int kShrinkStages = 6;
+constexpr int kExpandStages = 3;
+constexpr int kXStage = kTileRows * kBK * 2;    // 16 KiB
+constexpr int kYStage = kTileRows * kBN * 2;    // 32 KiB (two 64-column TMA boxes)
+constexpr int kShrinkThreads = 128;
+constexpr int kExpandThreads = 192;             // warp 0 copies, warp 1 issues MMAs, warps 2..5 epilogue
+
+struct PrefillSites {
+  int module[kMaxSites], d1[kMaxSites], d2[kMaxSites];
+  void* Y[kMaxSites];
+  int n;
+};
+
+struct ShrinkArgs {
+  CUtensorMap xmap[kMaxSites];
+  PrefillSites sites;
+  int32_t* err;
+  const int32_t* ws;
+  milora_group_layout_t lay;
+  float* vscratch;     // [kKSplit][T][rpad]
+  int T, rpad;
+};
+
+struct ExpandArgs {
+  CUtensorMap ymap[kMaxSites];
+  PrefillSites sites;
+  int32_t* err;
+  const int32_t* ws;
+  milora_group_layout_t lay;
+  const float* vscratch;
+  int T, rpad;
+};
+
+__device__ __forceinline__ int find_site(const PrefillSites& s, int module) {
+  int si = -1;
+#pragma unroll
+  for (int i = 0; i < kMaxSites; ++i)
+    if (i < s.n && s.module[i] == module) si = i;
+  return si;
+}
+
+// Bounded wait that also gives up as soon as another thread of the CTA has raised `abort`.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort, int32_t* err) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort) return false;
+  }
+  *abort = 1;
+  atomicOr(err, ERR_WAIT_TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ uint32_t tmem_cols_for(int rp) { return rp <= 32 ? 32u : 64u; }
+
+// ------------------------------------------------------------------------------------------------------
+// shrink
+// ------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __grid_constant__ ShrinkArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile_idx = blockIdx.x / kKSplit, ks = blockIdx.x % kKSplit;
+  const int n_tiles = a.ws[a.lay.header + H_NTILES];
+  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
+  const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
+  const int si = find_site(a.sites, job.module);
+  if (si < 0) return;
+  const int rp = job.rank_pad;
+  const uint32_t base = smem_u32(smem_raw);
+  if (!job.At_img || rp < 16 || rp > a.rpad || (rp & 15) || (base & 1023) || job.count < 1 || job.count > kTileRows ||
+      job.start < 0 || job.start + job.count > a.T) {
+    if (tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  const int d1 = a.sites.d1[si];
+  const int nchunks = d1 / kBK, cps = (nchunks + kKSplit - 1) / kKSplit;
+  const int kc0 = ks * cps, kc1 = min(nchunks, kc0 + cps), nk = max(kc1 - kc0, 0);
+
+  const uint32_t xs = base;
+  const uint32_t as = xs + kShrinkStages * kXStage;
+  const uint32_t a_stage = (uint32_t)a.rpad * 128u;
+  const uint32_t bars = as + kShrinkStages * a_stage;
+  auto full = [&](int i) { return bars + 8u * i; };
+  auto empty = [&](int i) { return bars + 8u * (kShrinkStages + i); };
+  const uint32_t accb = bars + 16u * kShrinkStages;
+  const uint32_t slot = accb + 8u;
+  volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  const uint32_t ncols = tmem_cols_for(rp);
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < kShrinkStages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+    mbar_init(accb, 1);
+    fence_barrier_init();
+    prefetch_tensormap(&a.xmap[si]);
+  }
+  __syncthreads();
+  if (warp == 0) { tmem_alloc(slot, ncols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *slot_ptr;
+
+  if (nk > 0) {
+    if (warp == 0 && lane == 0) {
+      // ---- copies: X tile by TMA, A image chunk by one bulk copy ----
+      const char* img = static_cast<const char*>(job.At_img);
+      for (int i = 0; i < nk; ++i) {
+        const int s = i % kShrinkStages, ph = (i / kShrinkStages) & 1;
+        if (i >= kShrinkStages && !wait_bar(empty(s), ph ^ 1, &abort_flag, a.err)) break;
+        mbar_expect_tx(full(s), kXStage + rp * 128);
+        tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
+        bulk_g2s(as + s * a_stage, img + (size_t)(kc0 + i) * rp * 128, rp * 128, full(s));
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---- MMAs: D[128 x rp] += X[128 x 16] * A[16 x rp], four per stage ----
+      const uint32_t idesc = idesc_bf16_f32(kTileRows, rp);
+      const uint32_t lbo = (uint32_t)(rp / 8) * 128u;        // A image: k-adjacent core matrices
+      bool ok = true;
+      for (int i = 0; i < nk && ok; ++i) {
+        const int s = i % kShrinkStages, ph = (i / kShrinkStages) & 1;
+        ok = wait_bar(full(s), ph, &abort_flag, a.err);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kBK / 16; ++kk) {
+          const uint64_t da = smem_desc(xs + s * kXStage + kk * 32, 16, 1024, 2);
+          const uint64_t db = smem_desc(as + s * a_stage + kk * 2 * lbo, lbo, 128, 0);
+          mma_bf16_ss(tmem_base, da, db, idesc, (i | kk) != 0);
+        }
+        mma_commit(empty(s));
+      }
+      mma_commit(accb);
+    }
+  }
+  __syncwarp();
+
+  // ---- epilogue: fp32 partial product to the scratch ----
+  bool ok = true;
+  if (nk > 0) ok = wait_bar(accb, 0, &abort_flag, a.err);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  const int m = warp * 32 + lane;
+  float* dst = a.vscratch + ((size_t)ks * a.T + job.start + m) * a.rpad;
+  for (int c0 = 0; c0 < rp; c0 += 16) {
+    uint32_t v[16];
+    if (nk > 0 && ok) {
+      tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+      tmem_wait_ld();
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] = 0u;
+    }
+    if (m < job.count) {
+#pragma unroll
+      for (int i = 0; i < 16; i += 4)
+        *reinterpret_cast<uint4*>(dst + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, ncols);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// expand
+// ------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void add8(uint4& y, const uint32_t* d) {
+  uint32_t w[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float lo = __uint_as_float(w[i] << 16) + __uint_as_float(d[2 * i]);
+    float hi = __uint_as_float(w[i] & 0xFFFF0000u) + __uint_as_float(d[2 * i + 1]);
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  y = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __grid_constant__ ExpandArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile_idx = blockIdx.x / kNSplit, ns = blockIdx.x % kNSplit;
+  const int n_tiles = a.ws[a.lay.header + H_NTILES];
+  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
+  const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
+  const int si = find_site(a.sites, job.module);
+  if (si < 0) return;
+  const int rp = job.rank_pad;
+  const uint32_t base = smem_u32(smem_raw);
+  if (!job.B_img || rp < 16 || rp > a.rpad || (rp & 15) || (base & 1023) || job.count < 1 || job.count > kTileRows ||
+      job.start < 0 || job.start + job.count > a.T) {
+    if (tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  const int d2 = a.sites.d2[si];
+  const int nchunks = d2 / kBN, cps = (nchunks + kNSplit - 1) / kNSplit;
+  const int nc0 = ns * cps, nc1 = min(nchunks, nc0 + cps), nn = nc1 - nc0;
+  if (nn <= 0) return;
+
+  const uint32_t ys = base;
+  const uint32_t bs = ys + kExpandStages * kYStage;
+  const uint32_t b_stage = (uint32_t)a.rpad * 256u;
+  const uint32_t vs = bs + kExpandStages * b_stage;
+  const uint32_t bars = vs + (uint32_t)kTileRows * a.rpad * 2u;
+  auto full = [&](int i) { return bars + 8u * i; };
+  auto empty = [&](int i) { return bars + 8u * (kExpandStages + i); };
+  auto tfull = [&](int i) { return bars + 8u * (2 * kExpandStages + i); };
+  auto tempty = [&](int i) { return bars + 8u * (2 * kExpandStages + 2 + i); };
+  const uint32_t slot = bars + 8u * (2 * kExpandStages + 4);
+  volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  constexpr uint32_t kCols = 2 * kBN;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < kExpandStages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
+    fence_barrier_init();
+    prefetch_tensormap(&a.ymap[si]);
+  }
+  __syncthreads();
+  if (warp == 0) { tmem_alloc(slot, kCols); tmem_relinquish(); }
+
+  // epilogue threads also build the A operand: V = s * sum_k V_k, bf16, 8 x 16-byte core-matrix rows
+  const int q = warp & 3;               // tensor-memory lane quarter this warp may read
+  const int m = q * 32 + lane;          // row of the tile this thread owns
+  if (warp >= 2) {
+    unsigned char* vrow = smem_raw + (vs - base) + (size_t)(m >> 3) * 128 + (size_t)(m & 7) * 16;
+    for (int c0 = 0; c0 < rp; c0 += 8) {
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+      if (m < job.count) {
+#pragma unroll
+        for (int k = 0; k < kKSplit; ++k) {
+          const float4* src =
+              reinterpret_cast<const float4*>(a.vscratch + ((size_t)k * a.T + job.start + m) * a.rpad + c0);
+          const float4 u0 = __ldcg(src), u1 = __ldcg(src + 1);
+          acc[0] += u0.x; acc[1] += u0.y; acc[2] += u0.z; acc[3] += u0.w;
+          acc[4] += u1.x; acc[5] += u1.y; acc[6] += u1.z; acc[7] += u1.w;
+        }
+      }
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(acc[2 * i] * job.scale, acc[2 * i + 1] * job.scale);
+        w[i] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(vrow + (size_t)(c0 >> 3) * (kTileRows / 8) * 128) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *slot_ptr;
+  const int row0 = job.start;
+  const bool full_tile = job.count == kTileRows;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const char* img = static_cast<const char*>(job.B_img);
+      for (int i = 0; i < nn; ++i) {
+        const int s = i % kExpandStages, ph = (i / kExpandStages) & 1;
+        if (i >= kExpandStages && !wait_bar(empty(s), ph ^ 1, &abort_flag, a.err)) break;
+        mbar_expect_tx(full(s), kYStage + rp * 256);
+        tma_load_2d(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s));
+        tma_load_2d(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s));
+        bulk_g2s(bs + s * b_stage, img + (size_t)(nc0 + i) * rp * 256, rp * 256, full(s));
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_f32(kTileRows, kBN);
+      constexpr uint32_t kLbo = (kTileRows / 8) * 128u;      // both operands: 16 core matrices per k group
+      for (int i = 0; i < nn; ++i) {
+        const int s = i % kExpandStages, ph = (i / kExpandStages) & 1, b = i & 1, bph = (i >> 1) & 1;
+        if (!wait_bar(full(s), ph, &abort_flag, a.err)) break;
+        if (i >= 2 && !wait_bar(tempty(b), bph ^ 1, &abort_flag, a.err)) break;
+        tc_fence_after();
+        for (int kk = 0; kk < rp / 16; ++kk) {
+          const uint64_t da = smem_desc(vs + kk * 2 * kLbo, kLbo, 128, 0);
+          const uint64_t db = smem_desc(bs + s * b_stage + kk * 2 * kLbo, kLbo, 128, 0);
+          mma_bf16_ss(tmem_base + b * kBN, da, db, idesc, kk != 0);
+        }
+        mma_commit(tfull(b));
+      }
+    }
+  } else {
+    const int e = tid - 64;
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(a.sites.Y[si]);
+    bool ok = true;
+    for (int i = 0; i < nn && ok; ++i) {
+      const int s = i % kExpandStages, ph = (i / kExpandStages) & 1, b = i & 1, bph = (i >> 1) & 1;
+      ok = wait_bar(tfull(b), bph, &abort_flag, a.err) && wait_bar(full(s), ph, &abort_flag, a.err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      unsigned char* ytile = smem_raw + (ys - base) + (size_t)s * kYStage;
+#pragma unroll 2
+      for (int c16 = 0; c16 < kBN / 16; ++c16) {
+        uint32_t d[16];
+        tmem_ld16(tmem_base + b * kBN + ((uint32_t)(q * 32) << 16) + c16 * 16, d);
+        tmem_wait_ld();
+        if (m < job.count) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int cg = c16 * 2 + h, box = cg >> 3, c = cg & 7;
+            uint4* p = reinterpret_cast<uint4*>(ytile + (size_t)box * (kYStage / 2) + (size_t)m * 128 + ((c ^ (m & 7)) << 4));
+            uint4 y = *p;
+            add8(y, d + 8 * h);
+            *p = y;
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty(b));
+      fence_proxy_async_smem();
+      named_barrier(1, 128);
+      if (full_tile) {
+        if (e == 0) {
+          tma_store_2d(&a.ymap[si], (nc0 + i) * kBN, row0, ys + s * kYStage);
+          tma_store_2d(&a.ymap[si], (nc0 + i) * kBN + 64, row0, ys + s * kYStage + kYStage / 2);
+          bulk_commit_group();
+          bulk_wait_group_read0();
+          mbar_arrive(empty(s));
+        }
+      } else {
+        // a tile with fewer than 128 rows: write only its own rows
+        for (int idx = e; idx < job.count * 16; idx += 128) {
+          const int rr = idx >> 4, cg = idx & 15, box = cg >> 3, c = cg & 7;
+          const uint4 y = *reinterpret_cast<const uint4*>(ytile + (size_t)box * (kYStage / 2) + (size_t)rr * 128 +
+                                                          ((c ^ (rr & 7)) << 4));
+          *reinterpret_cast<uint4*>(Y + (size_t)(row0 + rr) * d2 + (size_t)(nc0 + i) * kBN + cg * 8) = y;
+        }
+        named_barrier(1, 128);
+        if (e == 0) mbar_arrive(empty(s));
+      }
+    }
+    if (e == 0) bulk_wait_group0();
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, kCols);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// registration-time operand images
+// ------------------------------------------------------------------------------------------------------
+// A image: for every 64-wide k chunk a block of rp x 64 bf16 as 8 x 16-byte core-matrix rows;
+// core matrix (j / 8, k / 8) sits at ((k / 8) * (rp / 8) + j / 8) * 128 bytes.  One thread per 16 bytes.
+__global__ void pack_a_image_kernel(const __nv_bfloat16* __restrict__ At, uint4* __restrict__ img, int d1, int r, int rp) {
+  const size_t n_pieces = (size_t)(d1 / 8) * rp;
+  for (size_t p = blockIdx.x * (size_t)blockDim.x + threadIdx.x; p < n_pieces; p += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(p % rp);
+    const int k8 = (int)(p / rp);                 // which group of 8 k values
+    const int kc = k8 / 8, ki = k8 % 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (j < r) v = *reinterpret_cast<const uint4*>(At + (size_t)j * d1 + (size_t)k8 * 8);
+    const size_t off16 = (size_t)kc * (rp * 8) + ((size_t)ki * (rp / 8) + j / 8) * 8 + (j % 8);
+    img[off16] = v;
+  }
+}
+
+// B image: for every 128-wide n chunk a block of 128 x rp bf16 (n rows, k contiguous);
+// core matrix (n / 8, k / 8) sits at ((k / 8) * 16 + n / 8) * 128 bytes.  One thread per 16 bytes.
+__global__ void pack_b_image_kernel(const __nv_bfloat16* __restrict__ B, uint4* __restrict__ img, int d2, int r, int rp) {
+  const size_t n_pieces = (size_t)d2 * (rp / 8);
+  for (size_t p = blockIdx.x * (size_t)blockDim.x + threadIdx.x; p < n_pieces; p += (size_t)gridDim.x * blockDim.x) {
+    const int n = (int)(p % d2);
+    const int ki = (int)(p / d2);
+    const int nc = n / kBN, nl = n % kBN;
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int k0 = ki * 8 + 2 * i;
+      const unsigned short lo = k0 < r ? __bfloat16_as_ushort(B[(size_t)k0 * d2 + n]) : 0;
+      const unsigned short hi = k0 + 1 < r ? __bfloat16_as_ushort(B[(size_t)(k0 + 1) * d2 + n]) : 0;
+      w[i] = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+    const size_t off16 = (size_t)nc * (rp * 16) + ((size_t)ki * 16 + nl / 8) * 8 + (nl % 8);
+    img[off16] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows][cols] bf16 row-major, tiles of 128 rows x 64 columns, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)kTileRows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool prefill_images_supported(const milora_ctx* ctx, int d1, int d2, int rank) {
+  return ctx->desc.dtype == MILORA_BF16 && d1 % kBK == 0 && d2 % kBN == 0 && rank >= 1 && rank <= kRPadMax;
+}
+
+size_t prefill_image_bytes(int d, int rank) { return (size_t)d * ((rank + 15) & ~15) * 2; }
+
+milora_status launch_pack_images(milora_ctx* ctx, const void* At, const void* B, void* At_img, void* B_img, int d1, int d2,
+                                 int rank, cudaStream_t s) {
+  const int rp = (rank + 15) & ~15;
+  const size_t pa = (size_t)(d1 / 8) * rp, pb = (size_t)d2 * (rp / 8);
+  pack_a_image_kernel<<<(unsigned)std::min<size_t>((pa + 255) / 256, 4096), 256, 0, s>>>(
+      static_cast<const __nv_bfloat16*>(At), static_cast<uint4*>(At_img), d1, rank, rp);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  pack_b_image_kernel<<<(unsigned)std::min<size_t>((pb + 255) / 256, 4096), 256, 0, s>>>(
+      static_cast<const __nv_bfloat16*>(B), static_cast<uint4*>(B_img), d2, rank, rp);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                        cudaStream_t s) {
+  (void)layer;
+  if (ctx->desc.dtype != MILORA_BF16) return MILORA_E_SHAPE;
+  const int T = g->T;
+  const int rpad = (ctx->desc.max_rank + 15) & ~15;
+  if (rpad > kRPadMax || T < kTileRows) return MILORA_E_SHAPE;
+  for (int i = 0; i < sites.n; ++i) {
+    const ApplySite& st = sites.site[i];
+    if (st.d1 % kBK || st.d2 % kBN) return MILORA_E_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (reinterpret_cast<uintptr_t>(st.Y) & 15)) return MILORA_E_SHAPE;
+  }
+  const size_t shrink_smem = (size_t)kShrinkStages * (kXStage + rpad * 128) + 256;
+  const size_t expand_smem = (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + 256;
+  if (shrink_smem > 220 * 1024 || expand_smem > 220 * 1024) return MILORA_E_SHAPE;
+
+  const size_t need = (size_t)kKSplit * T * rpad;
+  if (need > ctx->vscratch_floats) {
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+    if (ctx->d_vscratch) MILORA_CUDA(ctx, cudaFree(ctx->d_vscratch));
+    ctx->d_vscratch = nullptr;
+    ctx->vscratch_floats = 0;
+    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_vscratch, need * sizeof(float)));
+    ctx->vscratch_floats = need;
+  }
+
+  ShrinkArgs sa;
+  ExpandArgs ea;
+  PrefillSites ps;
+  ps.n = sites.n;
+  for (int i = 0; i < kMaxSites; ++i) { ps.module[i] = -1; ps.d1[i] = ps.d2[i] = 0; ps.Y[i] = nullptr; }
+  for (int i = 0; i < sites.n; ++i) {
+    const ApplySite& st = sites.site[i];
+    ps.module[i] = st.module; ps.d1[i] = st.d1; ps.d2[i] = st.d2; ps.Y[i] = st.Y;
+    if (!make_map(&sa.xmap[i], st.X, T, st.d1) || !make_map(&ea.ymap[i], st.Y, T, st.d2)) return MILORA_E_SHAPE;
+  }
+  for (int i = sites.n; i < kMaxSites; ++i) { sa.xmap[i] = sa.xmap[0]; ea.ymap[i] = ea.ymap[0]; }
+  const milora_group_layout_t lay = group_layout(g->n_seq, g->T);
+  sa.sites = ps; sa.err = ctx->d_err; sa.ws = g->ws_dev; sa.lay = lay; sa.vscratch = ctx->d_vscratch; sa.T = T; sa.rpad = rpad;
+  ea.sites = ps; ea.err = ctx->d_err; ea.ws = g->ws_dev; ea.lay = lay; ea.vscratch = ctx->d_vscratch; ea.T = T; ea.rpad = rpad;
+
+  MILORA_CUDA(ctx, cudaFuncSetAttribute(prefill_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shrink_smem));
+  MILORA_CUDA(ctx, cudaFuncSetAttribute(prefill_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)expand_smem));
+  const size_t grid_s = (size_t)lay.max_tiles * kKSplit, grid_e = (size_t)lay.max_tiles * kNSplit;
+  if (grid_s > 0x7fffffffull || grid_e > 0x7fffffffull) return MILORA_E_CAPACITY;
+  prefill_shrink_kernel<<<(unsigned)grid_s, kShrinkThreads, shrink_smem, s>>>(sa);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  prefill_expand_kernel<<<(unsigned)grid_e, kExpandThreads, expand_smem, s>>>(ea);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
+}  // namespace milora

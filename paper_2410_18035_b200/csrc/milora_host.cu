@@ -238,21 +238,35 @@ milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, in
   size_t idx = adapter_index(tenant, layer, module, ctx->desc.n_layers);
   size_t bytes_a = ((size_t)rank * d1 * ctx->elem + 255) & ~size_t(255);
   size_t bytes_b = ((size_t)rank * d2 * ctx->elem + 255) & ~size_t(255);
+  // tensor-core operand images (bf16 contexts, dimensions that fit the tiled kernels)
+  const bool images = prefill_images_supported(ctx, d1, d2, rank);
+  size_t bytes_ai = images ? (prefill_image_bytes(d1, rank) + 255) & ~size_t(255) : 0;
+  size_t bytes_bi = images ? (prefill_image_bytes(d2, rank) + 255) & ~size_t(255) : 0;
+  const size_t total = bytes_a + bytes_b + bytes_ai + bytes_bi;
   AdapterEntry& ent = ctx->h_adapters[idx];
   void* store = const_cast<void*>(ent.At);
-  if (!store || ctx->adapter_bytes[idx] != bytes_a + bytes_b) {
+  if (!store || ctx->adapter_bytes[idx] != total) {
     cudaError_t e;
-    store = ctx->arena.alloc(bytes_a + bytes_b, &e);
+    store = ctx->arena.alloc(total, &e);
     if (!store) return cuda_fail(ctx, e, "adapter pool cudaMalloc");
-    ctx->adapter_bytes[idx] = bytes_a + bytes_b;
+    ctx->adapter_bytes[idx] = total;
   }
   void* At = store;
   void* Bs = static_cast<char*>(store) + bytes_a;
+  void* Ai = images ? static_cast<char*>(store) + bytes_a + bytes_b : nullptr;
+  void* Bi = images ? static_cast<char*>(store) + bytes_a + bytes_b + bytes_ai : nullptr;
   milora_status st = launch_repack_adapter(ctx, A_dev, B_dev, At, Bs, d1, d2, rank, as_stream(stream));
   if (st != MILORA_OK) return st;
+  if (images) {
+    st = launch_pack_images(ctx, At, Bs, Ai, Bi, d1, d2, rank, as_stream(stream));
+    if (st != MILORA_OK) return st;
+  }
   ent.At = At;
   ent.B = Bs;
+  ent.At_img = Ai;
+  ent.B_img = Bi;
   ent.rank = rank;
+  ent.rank_pad = (rank + 15) & ~15;
   ent.scale = scale;
   mark(ctx->adapters_dirty_lo, ctx->adapters_dirty_hi, idx);
   return MILORA_OK;
@@ -455,9 +469,10 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
   cudaStream_t s = as_stream(stream);
   milora_status st = sync_tables(ctx, s);
   if (st != MILORA_OK) return st;
-  if (!dense && ctx->desc.dtype == MILORA_BF16) {
-    st = launch_apply_decode_bf16(ctx, layer, sites, groups, s);
-    if (st != MILORA_E_SHAPE) return st;     // MILORA_E_SHAPE: this batch does not fit the cluster kernel
+  if (ctx->desc.dtype == MILORA_BF16) {
+    st = dense ? launch_apply_prefill_bf16(ctx, layer, sites, groups, s)
+               : launch_apply_decode_bf16(ctx, layer, sites, groups, s);
+    if (st != MILORA_E_SHAPE) return st;     // MILORA_E_SHAPE: this batch does not fit the specialised kernel
   }
   return launch_apply_generic(ctx, layer, sites, groups, dense, s);
 }

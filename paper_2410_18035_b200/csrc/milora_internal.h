@@ -167,4 +167,13 @@ milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites&
 milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
                                        cudaStream_t s);
 
+// bf16 prefill path: tcgen05 shrink and expand kernels over the dense tiles (same MILORA_E_SHAPE convention),
+// and the registration-time packing of the operand images they read.
+milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                        cudaStream_t s);
+bool prefill_images_supported(const milora_ctx* ctx, int d1, int d2, int rank);
+size_t prefill_image_bytes(int d, int rank);
+milora_status launch_pack_images(milora_ctx* ctx, const void* At, const void* B, void* At_img, void* B_img, int d1, int d2,
+                                 int rank, cudaStream_t s);
+
 }  // namespace milora

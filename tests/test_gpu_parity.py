@@ -132,7 +132,8 @@ RAGGED = [1, 33, 130, 257, 31, 32, 7, 129]
 
 
 @pytest.mark.parametrize("dtype,d,d_ff,d_kv,r", [("f32", 256, 688, 256, 8), ("bf16", 512, 1376, 128, 16),
-                                                 ("bf16", 256, 688, 256, 40)])
+                                                 ("bf16", 256, 688, 256, 40), ("bf16", 1024, 2816, 256, 16),
+                                                 ("bf16", 512, 1408, 512, 32), ("bf16", 512, 1408, 128, 64)])
 def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r):
     """Sequences of 1..257 rows (both work lists, ragged tile tails) mixed with decode rows; tenants repeat so
     that several sequences share a bucket; one slot is closed and one tenant has no adapters."""
