@@ -180,14 +180,13 @@ class Step:
         rec(1)
         ml.group(0, 1, self.cu_p, self.slots_p, len(self.prefill_ids), self.T_p, self.ws_p)
         rec(2)
-        for m in range(7):
-            ml.apply_prefill(0, m, self.Xp[m], self.Yp[m], self.g_p)
+        ml.apply_prefill_multi(0, self.mods, self.Xp, self.Yp, self.g_p)     # all 7 call sites, one call
         rec(3)
         ml.group(0, 1, self.cu_d, self.slots_d, len(self.decode_ids), self.T_d, self.ws_d)
         rec(4)
         ml.apply_decode_multi(0, self.mods, self.Xd, self.Yd, self.g_d)      # all 7 call sites, one launch
         rec(5)
-        self.n_launches = 1 + 1 + 7 + 1 + 1
+        self.n_launches = 1 + 1 + 2 + 1 + 1
         return self.n_launches
 
 
@@ -254,7 +253,7 @@ def run_ours(args, rank, world, device):
     dom = max(shares, key=shares.get)
     per_kernel = {
         "router": {"ms": route_ms, "launches": 1, "bytes": work["router_bytes"]},
-        "prefill_apply": {"ms": prefill_ms, "launches": 7, "bytes": work["prefill_bytes"]},
+        "prefill_apply": {"ms": prefill_ms, "launches": 2, "bytes": work["prefill_bytes"]},
         "decode_apply": {"ms": decode_ms, "launches": 1, "bytes": work["decode_bytes"]},
     }
     rooflines = {}

@@ -90,7 +90,6 @@ __device__ __forceinline__ uint32_t tmem_cols_for(int rp) { return rp <= 32 ? 32
 // ------------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __grid_constant__ ShrinkArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ int abort_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kKSplit, ks = blockIdx.x % kKSplit;
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
@@ -118,10 +117,11 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
   const uint32_t accb = bars + 16u * kShrinkStages;
   const uint32_t slot = accb + 8u;
   volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  volatile int* abort_ptr = reinterpret_cast<volatile int*>(smem_raw + (slot + 4 - base));
   const uint32_t ncols = tmem_cols_for(rp);
 
   if (tid == 0) {
-    abort_flag = 0;
+    *abort_ptr = 0;
     for (int i = 0; i < kShrinkStages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
     mbar_init(accb, 1);
     fence_barrier_init();
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
       const char* img = static_cast<const char*>(job.At_img);
       for (int i = 0; i < nk; ++i) {
         const int s = i % kShrinkStages, ph = (i / kShrinkStages) & 1;
-        if (i >= kShrinkStages && !wait_bar(empty(s), ph ^ 1, &abort_flag, a.err)) break;
+        if (i >= kShrinkStages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
         mbar_expect_tx(full(s), kXStage + rp * 128);
         tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
         bulk_g2s(as + s * a_stage, img + (size_t)(kc0 + i) * rp * 128, rp * 128, full(s));
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
       bool ok = true;
       for (int i = 0; i < nk && ok; ++i) {
         const int s = i % kShrinkStages, ph = (i / kShrinkStages) & 1;
-        ok = wait_bar(full(s), ph, &abort_flag, a.err);
+        ok = wait_bar(full(s), ph, abort_ptr, a.err);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
 
   // ---- epilogue: fp32 partial product to the scratch ----
   bool ok = true;
-  if (nk > 0) ok = wait_bar(accb, 0, &abort_flag, a.err);
+  if (nk > 0) ok = wait_bar(accb, 0, abort_ptr, a.err);
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
   const int m = warp * 32 + lane;
@@ -212,7 +212,6 @@ __device__ __forceinline__ void add8(uint4& y, const uint32_t* d) {
 
 __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __grid_constant__ ExpandArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ int abort_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kNSplit, ns = blockIdx.x % kNSplit;
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
@@ -243,10 +242,11 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
   auto tempty = [&](int i) { return bars + 8u * (2 * kExpandStages + 2 + i); };
   const uint32_t slot = bars + 8u * (2 * kExpandStages + 4);
   volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  volatile int* abort_ptr = reinterpret_cast<volatile int*>(smem_raw + (slot + 4 - base));
   constexpr uint32_t kCols = 2 * kBN;
 
   if (tid == 0) {
-    abort_flag = 0;
+    *abort_ptr = 0;
     for (int i = 0; i < kExpandStages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
     fence_barrier_init();
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
       const char* img = static_cast<const char*>(job.B_img);
       for (int i = 0; i < nn; ++i) {
         const int s = i % kExpandStages, ph = (i / kExpandStages) & 1;
-        if (i >= kExpandStages && !wait_bar(empty(s), ph ^ 1, &abort_flag, a.err)) break;
+        if (i >= kExpandStages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
         mbar_expect_tx(full(s), kYStage + rp * 256);
         tma_load_2d(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s));
         tma_load_2d(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s));
@@ -309,8 +309,8 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
       constexpr uint32_t kLbo = (kTileRows / 8) * 128u;      // both operands: 16 core matrices per k group
       for (int i = 0; i < nn; ++i) {
         const int s = i % kExpandStages, ph = (i / kExpandStages) & 1, b = i & 1, bph = (i >> 1) & 1;
-        if (!wait_bar(full(s), ph, &abort_flag, a.err)) break;
-        if (i >= 2 && !wait_bar(tempty(b), bph ^ 1, &abort_flag, a.err)) break;
+        if (!wait_bar(full(s), ph, abort_ptr, a.err)) break;
+        if (i >= 2 && !wait_bar(tempty(b), bph ^ 1, abort_ptr, a.err)) break;
         tc_fence_after();
         for (int kk = 0; kk < rp / 16; ++kk) {
           const uint64_t da = smem_desc(vs + kk * 2 * kLbo, kLbo, 128, 0);
@@ -326,23 +326,33 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
     bool ok = true;
     for (int i = 0; i < nn && ok; ++i) {
       const int s = i % kExpandStages, ph = (i / kExpandStages) & 1, b = i & 1, bph = (i >> 1) & 1;
-      ok = wait_bar(tfull(b), bph, &abort_flag, a.err) && wait_bar(full(s), ph, &abort_flag, a.err);
+      ok = wait_bar(tfull(b), bph, abort_ptr, a.err) && wait_bar(full(s), ph, abort_ptr, a.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       unsigned char* ytile = smem_raw + (ys - base) + (size_t)s * kYStage;
-#pragma unroll 2
-      for (int c16 = 0; c16 < kBN / 16; ++c16) {
-        uint32_t d[16];
-        tmem_ld16(tmem_base + b * kBN + ((uint32_t)(q * 32) << 16) + c16 * 16, d);
+      // 64 columns (one 128-byte swizzle box of y) per round: two tensor-memory loads in flight, one wait
+#pragma unroll 1
+      for (int box = 0; box < kBN / 64; ++box) {
+        uint32_t d0[32], d1v[32];
+        const uint32_t taddr = tmem_base + b * kBN + ((uint32_t)(q * 32) << 16) + box * 64;
+        tmem_ld32(taddr, d0);
+        tmem_ld32(taddr + 32, d1v);
         tmem_wait_ld();
         if (m < job.count) {
+          unsigned char* yrow = ytile + (size_t)box * (kYStage / 2) + (size_t)m * 128;
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int cg = c16 * 2 + h, box = cg >> 3, c = cg & 7;
-            uint4* p = reinterpret_cast<uint4*>(ytile + (size_t)box * (kYStage / 2) + (size_t)m * 128 + ((c ^ (m & 7)) << 4));
+          for (int c = 0; c < 4; ++c) {
+            uint4* p = reinterpret_cast<uint4*>(yrow + ((c ^ (m & 7)) << 4));
             uint4 y = *p;
-            add8(y, d + 8 * h);
+            add8(y, d0 + 8 * c);
+            *p = y;
+          }
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint4* p = reinterpret_cast<uint4*>(yrow + (((c + 4) ^ (m & 7)) << 4));
+            uint4 y = *p;
+            add8(y, d1v + 8 * c);
             *p = y;
           }
         }
@@ -480,8 +490,8 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
     if (st.d1 % kBK || st.d2 % kBN) return MILORA_E_SHAPE;
     if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (reinterpret_cast<uintptr_t>(st.Y) & 15)) return MILORA_E_SHAPE;
   }
-  const size_t shrink_smem = (size_t)kShrinkStages * (kXStage + rpad * 128) + 256;
-  const size_t expand_smem = (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + 256;
+  const size_t shrink_smem = (size_t)kShrinkStages * (kXStage + rpad * 128) + 128;
+  const size_t expand_smem = (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + 128;
   if (shrink_smem > 220 * 1024 || expand_smem > 220 * 1024) return MILORA_E_SHAPE;
 
   const size_t need = (size_t)kKSplit * T * rpad;
