@@ -188,13 +188,11 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
 
   // ---- 4. perm: token q of the sorted order ------------------------------------------------
   int32_t* perm = ws + a.lay.perm;
-  for (int q = tid; q < n_active; q += kGThreads) {
-    int lo = 0, hi = n_act_seq;           // last j with tok_off[j] <= q
-    while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if (tok_off[mid] <= q) lo = mid; else hi = mid;
-    }
-    perm[q] = seq_lo[comp[lo] & (kMaxSeq - 1)] + (q - tok_off[lo]);
+  // one warp per sorted sequence: its rows are consecutive, so the writes are coalesced
+  for (int j = tid >> 5; j < n_act_seq; j += kGThreads / 32) {
+    const int i = comp[j] & (kMaxSeq - 1);
+    const int lo = seq_lo[i], len = seq_len[i], off = tok_off[j];
+    for (int t = tid & 31; t < len; t += 32) perm[off + t] = lo + t;
   }
 
   // ---- 5. gather jobs: chunks of kGatherRows short rows per segment ---------------------------

@@ -89,6 +89,41 @@ __device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][8] */) {
   }
 }
 
+// Column reduction over `nr` rows for the 16-byte column group at `col` (row stride d): sum, max, or sum
+// weighted by w[t].  Eight independent 128-bit loads are in flight per thread; rows are combined in order.
+enum { kRedSum = 0, kRedMax = 1, kRedWeighted = 2 };
+template <typename T, int MODE>
+__device__ __forceinline__ void reduce_rows(const T* col, int d, int nr, const float* w, float (&acc)[VecOf<T>::N]) {
+  constexpr int V = VecOf<T>::N;
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] = MODE == kRedMax ? -FLT_MAX : 0.f;
+  int t = 0;
+  for (; t + 8 <= nr; t += 8) {
+    float v[8][V];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) VecOf<T>::load(col + (size_t)(t + k) * d, v[k]);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        if (MODE == kRedMax) acc[i] = fmaxf(acc[i], v[k][i]);
+        else if (MODE == kRedWeighted) acc[i] = fmaf(w[t + k], v[k][i], acc[i]);
+        else acc[i] += v[k][i];
+      }
+    }
+  }
+  for (; t < nr; ++t) {
+    float v[V];
+    VecOf<T>::load(col + (size_t)t * d, v);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      if (MODE == kRedMax) acc[i] = fmaxf(acc[i], v[i]);
+      else if (MODE == kRedWeighted) acc[i] = fmaf(w[t], v[i], acc[i]);
+      else acc[i] += v[i];
+    }
+  }
+}
+
 struct RouteArgs {
   DeviceTables tab;
   const void* H;
@@ -226,35 +261,10 @@ __global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
       const int c0 = (cb * kThreads + tid) * V;
       if (c0 < d) {
         float acc[V];
-        const bool is_max = pool == MILORA_POOL_MAX;
-#pragma unroll
-        for (int i = 0; i < V; ++i) acc[i] = is_max ? -FLT_MAX : 0.f;
         const T* col = H + (size_t)r0 * d + c0;
-        int t = 0;
-        for (; t + 8 <= nr; t += 8) {
-          float v[8][V];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) VecOf<T>::load(col + (size_t)(t + k) * d, v[k]);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-#pragma unroll
-            for (int i = 0; i < V; ++i) {
-              if (is_max) acc[i] = fmaxf(acc[i], v[k][i]);
-              else if (sa) acc[i] = fmaf(u_sm[t + k], v[k][i], acc[i]);
-              else acc[i] += v[k][i];
-            }
-          }
-        }
-        for (; t < nr; ++t) {
-          float v[V];
-          VecOf<T>::load(col + (size_t)t * d, v);
-#pragma unroll
-          for (int i = 0; i < V; ++i) {
-            if (is_max) acc[i] = fmaxf(acc[i], v[i]);
-            else if (sa) acc[i] = fmaf(u_sm[t], v[i], acc[i]);
-            else acc[i] += v[i];
-          }
-        }
+        if (pool == MILORA_POOL_MAX) reduce_rows<T, kRedMax>(col, d, nr, u_sm, acc);
+        else if (sa) reduce_rows<T, kRedWeighted>(col, d, nr, u_sm, acc);
+        else reduce_rows<T, kRedSum>(col, d, nr, u_sm, acc);
 #pragma unroll
         for (int i = 0; i < V; i += 4)
           *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
