@@ -3,16 +3,22 @@
 // written to the int32 route table.
 //
 // The kernel is bound by reading H (e * n_p * d bytes per prompt).  Work is cut into items of
-// kRows consecutive rows x one block of columns; every item writes fp32 partial column sums to
-// scratch, and the CTA that completes a prompt last (an atomic counter per prompt, no waiting)
-// combines the partials in chunk order, so the result does not depend on scheduling.
+// kRows consecutive rows x one block of kThreads 16-byte column groups; every thread streams its
+// column group with eight 128-bit loads in flight and every item writes fp32 partial column sums to
+// scratch.  CTAs take their first item by index and further items from an atomic counter (fetched
+// one item ahead, so its latency is hidden), so all SMs stay busy whatever the prompt lengths.
+// Nothing is synchronised per item: a CTA remembers which prompts it contributed to and, when it has
+// run out of items, publishes its counts with one fence; the CTA whose count completes a prompt
+// combines that prompt's partials in chunk order (nobody waits), so the result does not depend on
+// scheduling.
 #include <cfloat>
 
 #include "milora_internal.h"
 
-// Scratch of milora_route_static: partial column sums and chunk statistics, followed by one completion
-// counter per prompt.  It lives in the library image, so every GPU that loads the library holds it
-// (16 MiB + 16 KiB) until the process exits, and every call of that entry point shares it.
+// Scratch of milora_route_static: partial column sums and chunk statistics, followed by the scheduling
+// words and one completion counter per prompt.  It lives in the library image, so every GPU that loads
+// the library holds it (16 MiB + 16 KiB) until the process exits, and every call of that entry point
+// shares it.
 constexpr size_t kStaticPartialFloats = size_t(4) << 20;
 constexpr size_t kStaticCounters = 4096;
 static __device__ __align__(256) float g_route_static_scratch[kStaticPartialFloats + kStaticCounters];
@@ -20,8 +26,10 @@ static __device__ __align__(256) float g_route_static_scratch[kStaticPartialFloa
 namespace milora {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 128;
+constexpr int kWarps = kThreads / 32;
 constexpr int kRows = 64;
+constexpr int kSchedWords = 2;     // [0] next dynamic item, [1] CTAs that have finished
 
 template <typename T> struct VecOf;
 template <> struct VecOf<float> {
@@ -44,9 +52,6 @@ template <> struct VecOf<__nv_bfloat16> {
   }
 };
 
-__device__ inline float to_float(float v) { return v; }
-__device__ inline float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
-
 __device__ inline float activate(float h, const RouterEntry& r) {
   switch (r.act) {
     case MILORA_ACT_TANH: return tanhf(h);
@@ -65,9 +70,9 @@ __device__ inline float activate(float h, const RouterEntry& r) {
   }
 }
 
-// Sum over the block in a fixed order: lanes by xor-shuffle, then warp 0 adds the warp totals in order.
+// Sum over the block in a fixed order: lanes by xor-shuffle, then every thread adds the warp totals in order.
 template <int NV>
-__device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][8] */) {
+__device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][kWarps] */) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
@@ -77,51 +82,66 @@ __device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][8] */) {
   __syncthreads();
   if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) smem[i * 8 + warp] = v[i];
+    for (int i = 0; i < NV; ++i) smem[i * kWarps + warp] = v[i];
   }
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) s += smem[i * 8 + w];
+    for (int w = 0; w < kWarps; ++w) s += smem[i * kWarps + w];
     v[i] = s;
   }
 }
 
+// 128-bit streaming load that the compiler keeps in program order with the other loads of a batch.
+__device__ __forceinline__ uint4 ldg16_stream(const void* p) {
+  uint4 q;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
+               : "l"(p));
+  return q;
+}
+__device__ __forceinline__ void unpack16(const uint4& q, float (&v)[4]) {
+  v[0] = __uint_as_float(q.x); v[1] = __uint_as_float(q.y); v[2] = __uint_as_float(q.z); v[3] = __uint_as_float(q.w);
+}
+__device__ __forceinline__ void unpack16(const uint4& q, float (&v)[8]) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
 // Column reduction over `nr` rows for the 16-byte column group at `col` (row stride d): sum, max, or sum
-// weighted by w[t].  Eight independent 128-bit loads are in flight per thread; rows are combined in order.
+// weighted by w[t].  Rows are fetched in batches of kDepth independent 128-bit loads and combined in order.
 enum { kRedSum = 0, kRedMax = 1, kRedWeighted = 2 };
+constexpr int kDepth = 8;
 template <typename T, int MODE>
 __device__ __forceinline__ void reduce_rows(const T* col, int d, int nr, const float* w, float (&acc)[VecOf<T>::N]) {
   constexpr int V = VecOf<T>::N;
 #pragma unroll
   for (int i = 0; i < V; ++i) acc[i] = MODE == kRedMax ? -FLT_MAX : 0.f;
-  int t = 0;
-  for (; t + 8 <= nr; t += 8) {
-    float v[8][V];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) VecOf<T>::load(col + (size_t)(t + k) * d, v[k]);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-#pragma unroll
-      for (int i = 0; i < V; ++i) {
-        if (MODE == kRedMax) acc[i] = fmaxf(acc[i], v[k][i]);
-        else if (MODE == kRedWeighted) acc[i] = fmaf(w[t + k], v[k][i], acc[i]);
-        else acc[i] += v[k][i];
-      }
-    }
-  }
-  for (; t < nr; ++t) {
+  auto consume = [&](const uint4& q, int t) {
     float v[V];
-    VecOf<T>::load(col + (size_t)t * d, v);
+    unpack16(q, v);
 #pragma unroll
     for (int i = 0; i < V; ++i) {
       if (MODE == kRedMax) acc[i] = fmaxf(acc[i], v[i]);
       else if (MODE == kRedWeighted) acc[i] = fmaf(w[t], v[i], acc[i]);
       else acc[i] += v[i];
     }
+  };
+  int t = 0;
+  for (; t + kDepth <= nr; t += kDepth) {
+    uint4 q[kDepth];
+#pragma unroll
+    for (int k = 0; k < kDepth; ++k) q[k] = ldg16_stream(col + (size_t)(t + k) * d);
+#pragma unroll
+    for (int k = 0; k < kDepth; ++k) consume(q[k], t + k);
   }
+  for (; t < nr; ++t) consume(ldg16_stream(col + (size_t)t * d), t);
 }
 
 struct RouteArgs {
@@ -133,9 +153,124 @@ struct RouteArgs {
   float* probs_out;
   float* partial;     // [total_chunks][d]
   float* stats;       // [total_chunks][2]  (self-attention pooler: chunk max, chunk sum of exp)
-  int32_t* counters;  // [P], zero on entry, zero again on exit
+  int32_t* sched;     // kSchedWords scheduling words, then one completion counter per prompt; zero on entry and exit
   int layer, P, d, n_colblk;
 };
+
+constexpr int kMaxTouched = 32;   // prompts a CTA may contribute to before it has to publish its counts
+
+// Combine the partials of prompt p (all of its items are complete and visible) and write its route.
+template <typename T>
+__device__ void finalize_prompt(const RouteArgs& a, int p, int chunk0, int n_chunks, float* red) {
+  constexpr int V = VecOf<T>::N;
+  const int tid = threadIdx.x, d = a.d;
+  const int slot = a.seq_slot[p];
+  const bool slot_ok = slot >= 0 && slot < a.tab.max_requests;
+  const int tenant = slot_ok ? a.tab.slot_tenant[slot] : -1;
+  const RouterEntry* rp = (tenant >= 0 && tenant < a.tab.max_tenants)
+                              ? &a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer] : nullptr;
+  if (!rp || rp->W == nullptr || rp->pool < 0) {
+    // closed slot or no router for this tenant at this layer: the request stays "not routed"
+    if (tid == 0) {
+      if (slot_ok) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
+      else atomicOr(a.tab.err, ERR_BAD_SLOT);
+      a.sched[kSchedWords + p] = 0;
+    }
+    __syncthreads();
+    return;
+  }
+  const RouterEntry& r = *rp;
+  const int pool = r.pool;
+  const bool sa = pool == MILORA_POOL_SELFATTN;
+  const int n_p = a.cu[p + 1] - a.cu[p];
+  if (pool == MILORA_POOL_LAST) { chunk0 += n_chunks - 1; n_chunks = 1; }   // only the chunk with the last row counts
+  const float* part0 = a.partial + (size_t)chunk0 * d;
+  const float* st0 = a.stats + 2 * (size_t)chunk0;
+  float gmax = -FLT_MAX, denom = 1.f;
+  if (sa) {
+    for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, __ldcg(st0 + 2 * c));
+    denom = 0.f;
+    for (int c = 0; c < n_chunks; ++c) denom += expf(__ldcg(st0 + 2 * c) - gmax) * __ldcg(st0 + 2 * c + 1);
+  }
+  const T* W = static_cast<const T*>(r.W);
+  float z[MILORA_NMOD];
+#pragma unroll
+  for (int j = 0; j < MILORA_NMOD; ++j) z[j] = 0.f;
+  for (int c0 = tid * V; c0 < d; c0 += kThreads * V) {
+    float h[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) h[i] = pool == MILORA_POOL_MAX ? -FLT_MAX : 0.f;
+    // chunks are fetched eight at a time (all loads of a batch independent) and combined in chunk order
+    for (int cbase = 0; cbase < n_chunks; cbase += 8) {
+      float4 q[8][V / 4];
+      float wgt[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int c = min(cbase + k, n_chunks - 1);
+        wgt[k] = sa ? __ldcg(st0 + 2 * c) : 0.f;
+#pragma unroll
+        for (int i = 0; i < V / 4; ++i)
+          q[k][i] = __ldcg(reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0 + 4 * i));
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (cbase + k < n_chunks) {
+          const float wk = sa ? expf(wgt[k] - gmax) : 1.f;
+#pragma unroll
+          for (int i = 0; i < V / 4; ++i) {
+            const float4 u = q[k][i];
+            float* hh = h + 4 * i;
+            if (pool == MILORA_POOL_MAX) {
+              hh[0] = fmaxf(hh[0], u.x); hh[1] = fmaxf(hh[1], u.y); hh[2] = fmaxf(hh[2], u.z); hh[3] = fmaxf(hh[3], u.w);
+            } else if (sa) {
+              hh[0] = fmaf(wk, u.x, hh[0]); hh[1] = fmaf(wk, u.y, hh[1]); hh[2] = fmaf(wk, u.z, hh[2]); hh[3] = fmaf(wk, u.w, hh[3]);
+            } else {
+              hh[0] += u.x; hh[1] += u.y; hh[2] += u.z; hh[3] += u.w;
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      float hv = h[i];
+      if (pool == MILORA_POOL_MEAN) hv = hv / (float)n_p;
+      else if (sa) hv = hv / denom;
+      h[i] = activate(hv, r);
+    }
+#pragma unroll
+    for (int j = 0; j < MILORA_NMOD; ++j) {
+      float wv[V];
+      VecOf<T>::load(W + (size_t)j * d + c0, wv);
+#pragma unroll
+      for (int i = 0; i < V; ++i) z[j] = fmaf(h[i], wv[i], z[j]);
+    }
+  }
+  block_sum<MILORA_NMOD>(z, red);
+  if (tid == 0) {
+    float zmax = -FLT_MAX;
+    int best = 0;
+#pragma unroll
+    for (int j = 0; j < MILORA_NMOD; ++j) {
+      z[j] += r.bias[j];
+      if (z[j] > zmax) { zmax = z[j]; best = j; }   // strict: ties keep the lower index
+    }
+    float e[MILORA_NMOD], sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < MILORA_NMOD; ++j) { e[j] = expf(z[j] - zmax); sum += e[j]; }
+    a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = best;
+    if (a.logits_out) {
+#pragma unroll
+      for (int j = 0; j < MILORA_NMOD; ++j) a.logits_out[(size_t)p * MILORA_NMOD + j] = z[j];
+    }
+    if (a.probs_out) {
+#pragma unroll
+      for (int j = 0; j < MILORA_NMOD; ++j) a.probs_out[(size_t)p * MILORA_NMOD + j] = e[j] / sum;
+    }
+    a.sched[kSchedWords + p] = 0;
+  }
+  __syncthreads();
+}
 
 // Dynamic shared memory: item_start[P+1], chunk_base[P+1].
 template <typename T>
@@ -143,50 +278,44 @@ __global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
   extern __shared__ int32_t sm_i[];
   int32_t* item_start = sm_i;
   int32_t* chunk_base = sm_i + (a.P + 1);
-  __shared__ float red[8 * 8];
+  __shared__ float red[MILORA_NMOD * kWarps];
   __shared__ float u_sm[kRows];
   __shared__ int32_t carry[2];
-  __shared__ int32_t is_last;
+  __shared__ int32_t wsum[2][kWarps];
+  __shared__ int32_t next_item, n_touched, n_done;
+  __shared__ int32_t touched_p[kMaxTouched], touched_n[kMaxTouched], done_p[kMaxTouched];
   constexpr int V = VecOf<T>::N;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = a.d;
   const T* H = static_cast<const T*>(a.H);
+  int32_t* counters = a.sched + kSchedWords;
 
   // ---- per-CTA prefix over prompts: how many items and scratch rows each prompt owns ----
-  if (tid == 0) { carry[0] = 0; carry[1] = 0; }
+  if (tid == 0) { carry[0] = 0; carry[1] = 0; n_touched = 0; n_done = 0; }
   __syncthreads();
   for (int base = 0; base < a.P; base += kThreads) {
-    int p = base + tid;
+    const int p = base + tid;
     int items = 0, chunks = 0;
     if (p < a.P) {
-      int slot = a.seq_slot[p];
-      int n_p = a.cu[p + 1] - a.cu[p];
-      bool ok = slot >= 0 && slot < a.tab.max_requests && n_p > 0;
-      int tenant = ok ? a.tab.slot_tenant[slot] : -1;
-      ok = ok && tenant >= 0 && tenant < a.tab.max_tenants;
-      if (ok) {
-        const RouterEntry& r = a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer];
-        ok = r.W != nullptr && r.pool >= 0;
-        if (ok) {
-          if (r.pool == MILORA_POOL_LAST) n_p = 1;
-          chunks = (n_p + kRows - 1) / kRows;
-          items = chunks * (r.pool == MILORA_POOL_SELFATTN ? 1 : a.n_colblk);
-        }
-      }
-      if (!ok && blockIdx.x == 0) {
+      // The item count depends on the prompt length alone (one dependent load); items that turn out to have
+      // nothing to do (another pooler, a closed slot) return at once and the prompt is still finalized.
+      const int n_p = a.cu[p + 1] - a.cu[p];
+      if (n_p > 0) {
+        chunks = (n_p + kRows - 1) / kRows;
+        items = chunks * a.n_colblk;
+      } else if (blockIdx.x == 0) {
+        const int slot = a.seq_slot[p];      // an empty prompt has no items: mark it "not routed" here
         if (slot >= 0 && slot < a.tab.max_requests) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
         else atomicOr(a.tab.err, ERR_BAD_SLOT);
       }
     }
-    // inclusive scan of (items, chunks) over the 256 prompts of this round
+    // inclusive scan of (items, chunks) over the prompts of this round
     int si = items, sc = chunks;
-    const int lane = tid & 31, warp = tid >> 5;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       int ti = __shfl_up_sync(0xffffffffu, si, o), tc = __shfl_up_sync(0xffffffffu, sc, o);
       if (lane >= o) { si += ti; sc += tc; }
     }
-    __shared__ int32_t wsum[2][8];
     if (lane == 31) { wsum[0][warp] = si; wsum[1][warp] = sc; }
     __syncthreads();
     int offi = carry[0], offc = carry[1];
@@ -200,7 +329,33 @@ __global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
   __syncthreads();
   const int total_items = item_start[a.P];
 
-  for (int it = blockIdx.x; it < total_items; it += gridDim.x) {
+  // Publish the per-prompt item counts of this CTA; the CTA that completes a prompt's count finalizes it.
+  auto publish = [&]() {
+    __threadfence();                 // this CTA's partial sums are visible before its counts are
+    __syncthreads();
+    const int nt = n_touched;
+    for (int i = tid; i < nt; i += kThreads) {
+      const int p = touched_p[i];
+      const int n_items = item_start[p + 1] - item_start[p];
+      if (atomicAdd(counters + p, touched_n[i]) + touched_n[i] == n_items) done_p[atomicAdd(&n_done, 1)] = p;
+    }
+    __syncthreads();
+    const int nd = n_done;
+    if (nd > 0) __threadfence();     // the other CTAs' partial sums are visible before they are read
+    for (int i = 0; i < nd; ++i) {
+      const int p = done_p[i];
+      finalize_prompt<T>(a, p, chunk_base[p], chunk_base[p + 1] - chunk_base[p], red);
+    }
+    __syncthreads();
+    if (tid == 0) { n_touched = 0; n_done = 0; }
+    __syncthreads();
+  };
+
+  int it = blockIdx.x;
+  while (it < total_items) {
+    // ask for the next item now; the answer is needed only when this item is done
+    int fetched = 0;
+    if (tid == 0) fetched = (int)gridDim.x + atomicAdd(a.sched, 1);
     // prompt of this item: last p with item_start[p] <= it
     int lo = 0, hi = a.P;
     while (hi - lo > 1) {
@@ -209,27 +364,32 @@ __global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
     }
     const int p = lo;
     const int slot = a.seq_slot[p];
-    const int tenant = a.tab.slot_tenant[slot];
-    const RouterEntry& r = a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer];
-    const int pool = r.pool;
-    int row_lo = a.cu[p], row_hi = a.cu[p + 1];
-    const int n_p = row_hi - row_lo;
-    if (pool == MILORA_POOL_LAST) row_lo = row_hi - 1;
-    const int n_chunks = chunk_base[p + 1] - chunk_base[p];
+    const int tenant = (slot >= 0 && slot < a.tab.max_requests) ? a.tab.slot_tenant[slot] : -1;
+    const RouterEntry* rp = (tenant >= 0 && tenant < a.tab.max_tenants)
+                                ? &a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer] : nullptr;
+    bool work = rp && rp->W != nullptr && rp->pool >= 0;    // the same for every thread of the CTA
+    const RouterEntry& r = *(work ? rp : a.tab.routers);
+    const int pool = work ? r.pool : -1;
+    const int row_lo = a.cu[p], row_hi = a.cu[p + 1];
     const int local = it - item_start[p];
     const bool sa = pool == MILORA_POOL_SELFATTN;
-    const int rc = sa ? local : local / a.n_colblk;
-    const int cb0 = sa ? 0 : local % a.n_colblk;
-    const int cb1 = sa ? a.n_colblk : cb0 + 1;
-    const int r0 = row_lo + rc * kRows;
-    const int nr = min(kRows, row_hi - r0);
+    const int rc = local / a.n_colblk, cb = local % a.n_colblk;
+    int r0 = row_lo + rc * kRows;
+    int nr = min(kRows, row_hi - r0);
+    if (pool == MILORA_POOL_LAST) {          // only the last row is pooled: the prompt's last chunk holds it
+      work = work && rc == chunk_base[p + 1] - chunk_base[p] - 1;
+      r0 = row_hi - 1;
+      nr = 1;
+    }
+    if (sa) work = work && cb == 0;          // the self-attention pooler needs whole rows: one item per chunk
+    const int cb0 = sa ? 0 : cb;
+    const int cb1 = !work ? cb0 : (sa ? a.n_colblk : cb0 + 1);
     float* part = a.partial + (size_t)(chunk_base[p] + rc) * d;
 
-    if (sa) {
+    if (sa && work) {
       // Appendix C: u_t = H[t,:] . w_sa for the rows of this chunk, then exp weights relative to the chunk max.
       const T* wsa = static_cast<const T*>(r.Wsa);
-      const int lane = tid & 31, warp = tid >> 5;
-      for (int t = warp; t < nr; t += kThreads / 32) {
+      for (int t = warp; t < nr; t += kWarps) {
         const T* row = H + (size_t)(r0 + t) * d;
         float acc = 0.f;
         for (int c = lane * V; c < d; c += 32 * V) {
@@ -271,81 +431,26 @@ __global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
       }
     }
 
-    // ---- completion: the CTA that finishes the prompt's last item combines the partials ----
-    __threadfence();
-    __syncthreads();
+    // ---- bookkeeping: remember the contribution, move to the prefetched item ----
     if (tid == 0) {
-      int n_items = item_start[p + 1] - item_start[p];
-      int old = atomicAdd(a.counters + p, 1);
-      is_last = (old == n_items - 1);
+      const int nt = n_touched;
+      if (nt > 0 && touched_p[nt - 1] == p) touched_n[nt - 1] += 1;
+      else { touched_p[nt] = p; touched_n[nt] = 1; n_touched = nt + 1; }
+      next_item = fetched;
     }
     __syncthreads();
-    if (!is_last) continue;
+    it = next_item;
+    if (n_touched == kMaxTouched) publish();
+  }
+  publish();
+
+  // ---- the CTA that leaves last puts the scheduling words back to zero for the next launch ----
+  if (tid == 0) {
     __threadfence();
-    const float* part0 = a.partial + (size_t)chunk_base[p] * d;
-    const float* st0 = a.stats + 2 * (size_t)chunk_base[p];
-    float gmax = -FLT_MAX, denom = 1.f;
-    if (sa) {
-      for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, __ldcg(st0 + 2 * c));
-      denom = 0.f;
-      for (int c = 0; c < n_chunks; ++c) denom += expf(__ldcg(st0 + 2 * c) - gmax) * __ldcg(st0 + 2 * c + 1);
+    if (atomicAdd(a.sched + 1, 1) == (int)gridDim.x - 1) {
+      a.sched[0] = 0;
+      a.sched[1] = 0;
     }
-    const T* W = static_cast<const T*>(r.W);
-    float z[MILORA_NMOD];
-#pragma unroll
-    for (int j = 0; j < MILORA_NMOD; ++j) z[j] = 0.f;
-    for (int c0 = tid * 4; c0 < d; c0 += kThreads * 4) {
-      float h[4];
-      if (pool == MILORA_POOL_MAX) {
-        h[0] = h[1] = h[2] = h[3] = -FLT_MAX;
-      } else {
-        h[0] = h[1] = h[2] = h[3] = 0.f;
-      }
-      for (int c = 0; c < n_chunks; ++c) {
-        float4 q = __ldcg(reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0));
-        if (pool == MILORA_POOL_MAX) {
-          h[0] = fmaxf(h[0], q.x); h[1] = fmaxf(h[1], q.y); h[2] = fmaxf(h[2], q.z); h[3] = fmaxf(h[3], q.w);
-        } else if (sa) {
-          float w = expf(__ldcg(st0 + 2 * c) - gmax);
-          h[0] = fmaf(w, q.x, h[0]); h[1] = fmaf(w, q.y, h[1]); h[2] = fmaf(w, q.z, h[2]); h[3] = fmaf(w, q.w, h[3]);
-        } else {
-          h[0] += q.x; h[1] += q.y; h[2] += q.z; h[3] += q.w;
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float hv = h[i];
-        if (pool == MILORA_POOL_MEAN) hv = hv / (float)n_p;
-        else if (sa) hv = hv / denom;
-        float g = activate(hv, r);
-#pragma unroll
-        for (int j = 0; j < MILORA_NMOD; ++j) z[j] = fmaf(g, to_float(W[(size_t)j * d + c0 + i]), z[j]);
-      }
-    }
-    block_sum<MILORA_NMOD>(z, red);
-    if (tid == 0) {
-      float zmax = -FLT_MAX;
-      int best = 0;
-#pragma unroll
-      for (int j = 0; j < MILORA_NMOD; ++j) {
-        z[j] += r.bias[j];
-        if (z[j] > zmax) { zmax = z[j]; best = j; }   // strict: ties keep the lower index
-      }
-      float e[MILORA_NMOD], sum = 0.f;
-#pragma unroll
-      for (int j = 0; j < MILORA_NMOD; ++j) { e[j] = expf(z[j] - zmax); sum += e[j]; }
-      a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = best;
-      if (a.logits_out) {
-#pragma unroll
-        for (int j = 0; j < MILORA_NMOD; ++j) a.logits_out[(size_t)p * MILORA_NMOD + j] = z[j];
-      }
-      if (a.probs_out) {
-#pragma unroll
-        for (int j = 0; j < MILORA_NMOD; ++j) a.probs_out[(size_t)p * MILORA_NMOD + j] = e[j] / sum;
-      }
-      a.counters[p] = 0;
-    }
-    __syncthreads();
   }
 }
 
@@ -375,6 +480,46 @@ milora_status transpose(milora_ctx* ctx, const void* in, void* out, int rows, in
   return MILORA_OK;
 }
 
+struct RoutePlan {
+  int n_colblk;
+  size_t max_chunks, scratch_floats, max_items;
+};
+
+RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
+  RoutePlan pl;
+  const int d = ctx->desc.d_model;
+  const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
+  pl.n_colblk = (d + kThreads * V - 1) / (kThreads * V);
+  pl.max_chunks = (size_t)T_total / kRows + P;
+  pl.scratch_floats = pl.max_chunks * d + 2 * pl.max_chunks;
+  pl.max_items = pl.max_chunks * pl.n_colblk;
+  return pl;
+}
+
+// `scratch` holds plan.scratch_floats floats; `sched` holds kSchedWords + P zeroed int32.
+milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const void* H, const int32_t* cu,
+                        const int32_t* seq_slot, int P, float* logits_out, float* probs_out, float* scratch, int32_t* sched,
+                        cudaStream_t s) {
+  RouteArgs a;
+  a.tab = device_tables(ctx);
+  a.H = H; a.cu = cu; a.seq_slot = seq_slot;
+  a.logits_out = logits_out; a.probs_out = probs_out;
+  a.partial = scratch;
+  a.stats = scratch + pl.max_chunks * ctx->desc.d_model;
+  a.sched = sched;
+  a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_colblk = pl.n_colblk;
+  const size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
+  int grid = (int)std::min<size_t>(pl.max_items, (size_t)ctx->sm_count * 8);
+  if (grid < 1) grid = 1;
+  if (ctx->desc.dtype == MILORA_F32) {
+    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
+  } else {
+    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
+  }
+  MILORA_CUDA(ctx, cudaGetLastError());
+  return MILORA_OK;
+}
+
 }  // namespace
 
 milora_status launch_repack_adapter(milora_ctx* ctx, const void* A, const void* B, void* At, void* Bout, int d1, int d2,
@@ -393,48 +538,26 @@ milora_status launch_repack_router(milora_ctx* ctx, const void* Wr, void* Wt, in
 
 milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int32_t* cu, const int32_t* seq_slot, int P,
                            int T_total, float* logits_out, float* probs_out, cudaStream_t s) {
-  const int d = ctx->desc.d_model;
-  const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
-  const int n_colblk = (d + kThreads * V - 1) / (kThreads * V);
-  const size_t max_chunks = (size_t)T_total / kRows + P;
-  const size_t need = max_chunks * d + 2 * max_chunks;
-  if (need > ctx->scratch_floats) {
+  const RoutePlan pl = plan_route(ctx, P, T_total);
+  if (pl.scratch_floats > ctx->scratch_floats) {
     MILORA_CUDA(ctx, cudaStreamSynchronize(s));
     if (ctx->d_scratch) MILORA_CUDA(ctx, cudaFree(ctx->d_scratch));
     ctx->d_scratch = nullptr;
     ctx->scratch_floats = 0;
-    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_scratch, need * sizeof(float)));
-    ctx->scratch_floats = need;
+    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_scratch, pl.scratch_floats * sizeof(float)));
+    ctx->scratch_floats = pl.scratch_floats;
   }
-  if ((size_t)P > ctx->n_counters) {
+  if ((size_t)P + kSchedWords > ctx->n_counters) {
     MILORA_CUDA(ctx, cudaStreamSynchronize(s));
     if (ctx->d_counters) MILORA_CUDA(ctx, cudaFree(ctx->d_counters));
     ctx->d_counters = nullptr;
     ctx->n_counters = 0;
-    size_t n = std::max<size_t>(P, 1024);
+    size_t n = std::max<size_t>(P, 1024) + kSchedWords;
     MILORA_CUDA(ctx, cudaMalloc(&ctx->d_counters, n * sizeof(int32_t)));
     MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_counters, 0, n * sizeof(int32_t), s));
     ctx->n_counters = n;
   }
-  RouteArgs a;
-  a.tab = device_tables(ctx);
-  a.H = H; a.cu = cu; a.seq_slot = seq_slot;
-  a.logits_out = logits_out; a.probs_out = probs_out;
-  a.partial = ctx->d_scratch;
-  a.stats = ctx->d_scratch + max_chunks * d;
-  a.counters = ctx->d_counters;
-  a.layer = layer; a.P = P; a.d = d; a.n_colblk = n_colblk;
-  size_t max_items = max_chunks * n_colblk;
-  int grid = (int)std::min<size_t>(max_items, (size_t)ctx->sm_count * 4);
-  if (grid < 1) grid = 1;
-  size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
-  if (ctx->desc.dtype == MILORA_F32) {
-    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
-  } else {
-    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
-  }
-  MILORA_CUDA(ctx, cudaGetLastError());
-  return MILORA_OK;
+  return run_route(ctx, pl, layer, H, cu, seq_slot, P, logits_out, probs_out, ctx->d_scratch, ctx->d_counters, s);
 }
 
 // Same kernel as launch_route, but the scratch is the file-scope device array above, so that nothing is
@@ -444,12 +567,9 @@ milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, con
                                   int P, int T_total, float* logits_out, float* probs_out, cudaStream_t s) {
   constexpr int kMaxDevices = 64;
   static float* scratch_of_device[kMaxDevices] = {nullptr};
-  const int d = ctx->desc.d_model;
-  const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
-  const int n_colblk = (d + kThreads * V - 1) / (kThreads * V);
-  const size_t max_chunks = (size_t)T_total / kRows + P;
-  const size_t need = max_chunks * d + 2 * max_chunks;
-  if (need > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
+  const RoutePlan pl = plan_route(ctx, P, T_total);
+  // the last kSchedWords floats of the partial area serve as the scheduling words, right in front of the counters
+  if (pl.scratch_floats + kSchedWords > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
   int dev = -1;
   MILORA_CUDA(ctx, cudaGetDevice(&dev));
   if (dev != ctx->device) return MILORA_E_STATE;     // the context's device must be current
@@ -460,28 +580,10 @@ milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, con
     scratch_of_device[dev] = ptr;
   }
   float* scratch = scratch_of_device[dev];
-  int32_t* counters = reinterpret_cast<int32_t*>(scratch + kStaticPartialFloats);
-  // The array keeps whatever the previous call left; only the counters have to start at zero.
-  MILORA_CUDA(ctx, cudaMemsetAsync(counters, 0, (size_t)P * sizeof(int32_t), s));
-  RouteArgs a;
-  a.tab = device_tables(ctx);
-  a.H = H; a.cu = cu; a.seq_slot = seq_slot;
-  a.logits_out = logits_out; a.probs_out = probs_out;
-  a.partial = scratch;
-  a.stats = scratch + max_chunks * d;
-  a.counters = counters;
-  a.layer = layer; a.P = P; a.d = d; a.n_colblk = n_colblk;
-  size_t max_items = max_chunks * n_colblk;
-  int grid = (int)std::min<size_t>(max_items, (size_t)ctx->sm_count * 4);
-  if (grid < 1) grid = 1;
-  size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
-  if (ctx->desc.dtype == MILORA_F32) {
-    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
-  } else {
-    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
-  }
-  MILORA_CUDA(ctx, cudaGetLastError());
-  return MILORA_OK;
+  int32_t* sched = reinterpret_cast<int32_t*>(scratch + kStaticPartialFloats - kSchedWords);
+  // The array keeps whatever the previous call left; the scheduling words and the counters have to start at zero.
+  MILORA_CUDA(ctx, cudaMemsetAsync(sched, 0, ((size_t)P + kSchedWords) * sizeof(int32_t), s));
+  return run_route(ctx, pl, layer, H, cu, seq_slot, P, logits_out, probs_out, scratch, sched, s);
 }
 
 }  // namespace milora
