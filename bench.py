@@ -294,27 +294,43 @@ def run_ours(args, rank, world, device):
 
 
 def run_e2e(step, args, world, device, tokens_per_step):
-    """Same step, but every step's inputs start in pinned host memory and the outputs end there."""
+    """Same step through milora_step_host: every input starts in pinned HOST memory, the C ABI copies it
+    in, runs the path and copies every output back; all of it is inside the timed region."""
+    ml = step.lw.ml
     steps = max(1, min(args.steps, 3))
-    host_in = [step.H] + step.Xp + step.Yp + step.Xd + step.Yd
-    pinned = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in host_in]
-    for p, t in zip(pinned, host_in):
+
+    def pin(t):
+        p = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
         p.copy_(t)
-    outs = step.Yp + step.Yd
-    pinned_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
-    h2d = sum(t.numel() * t.element_size() for t in host_in)
-    d2h = sum(t.numel() * t.element_size() for t in outs)
+        return p
+
+    Hh = pin(step.H)
+    cu_p, slots_p = pin(step.cu_p), pin(step.slots_p)
+    cu_d, slots_d = pin(step.cu_d), pin(step.slots_d)
+    Xp = {m: pin(step.Xp[m]) for m in range(7)}
+    Yp = {m: pin(step.Yp[m]) for m in range(7)}
+    Xd = {m: pin(step.Xd[m]) for m in range(7)}
+    Yd = {m: pin(step.Yd[m]) for m in range(7)}
+    # prefill part (routes the prompts, applies on the prompt rows) and decode part (applies on the decode rows)
+    st_p = ml.make_host_step(0, cu_p, slots_p, Hh, cu_p, slots_p, step.T_p, Xp, Yp)
+    st_d = ml.make_host_step(0, None, None, None, cu_d, slots_d, step.T_d, Xd, Yd)
+    ws = torch.empty(max(ml.step_host_workspace(st_p), ml.step_host_workspace(st_d)) + 256, dtype=torch.uint8,
+                     device=device)
+    off = (-ws.data_ptr()) % 256
+    ws = ws[off:]
+    nb = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+    h2d = nb([Hh, cu_p, slots_p, cu_p, slots_p, cu_d, slots_d]) + nb(Xp.values()) + nb(Yp.values()) + nb(Xd.values()) + nb(Yd.values())
+    d2h = nb(Yp.values()) + nb(Yd.values())
+    ml.step_host(st_p, ws)
+    ml.step_host(st_d, ws)
     torch.cuda.synchronize(device)
     if world > 1:
         torch.distributed.barrier()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(steps):
-        for p, t in zip(pinned, host_in):
-            t.copy_(p, non_blocking=True)
-        step.run()
-        for p, t in zip(pinned_out, outs):
-            p.copy_(t, non_blocking=True)
+        ml.step_host(st_p, ws)
+        ml.step_host(st_d, ws)
     t1.record()
     torch.cuda.synchronize(device)
     ms = t0.elapsed_time(t1)
@@ -372,7 +388,7 @@ def cpu_threads():
         return 1
 
 
-def cpu_baseline(w, args, n_prompts=16):
+def cpu_baseline(w, args, n_prompts=64):
     tokens, dt = oracle_sample_step(w, n_prompts)
     return {"value": tokens / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
             "sample": f"first {n_prompts} of {len(w.prefill_ids)} prompts (all their tokens) and the same "
@@ -406,7 +422,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2")

@@ -226,6 +226,35 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
                                          const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                          void* stream);
 
+/* ---- one step from host buffers ------------------------------------------------------------------
+ * The whole path for one layer with every input in HOST memory (pinned memory makes the copies
+ * asynchronous): copy in, route the prompts (Eq. 2-3), group the step's sequences, apply Eq. 1 on
+ * every listed module for prompt rows and decode rows, copy the outputs back.  Everything is enqueued
+ * on `stream`; the host buffers may be reused once the stream has been synchronised.
+ *   n_prompts prompts to route: rows [cu_prompts_host[p], cu_prompts_host[p+1]) of H_host
+ *             ([cu_prompts_host[n_prompts]][d_model]), slots prompt_slot_host[p]; n_prompts = 0 skips routing;
+ *   n_seq sequences of T rows in total (cu_seq_host[n_seq+1], seq_slot_host[n_seq]) form the step;
+ *   X_host[m] / Y_host[m] are the [T][d1(m)] inputs and [T][d2(m)] outputs of module m; a NULL pair skips m.
+ * workspace_dev is caller-owned device memory of at least milora_step_host_workspace() bytes,
+ * 256-byte aligned; the library allocates nothing here except what milora_route may grow. */
+typedef struct {
+  int layer;
+  int n_prompts;
+  const int32_t* cu_prompts_host;
+  const int32_t* prompt_slot_host;
+  const void* H_host;
+  int n_seq;
+  int T;
+  const int32_t* cu_seq_host;
+  const int32_t* seq_slot_host;
+  const void* X_host[MILORA_NMOD];
+  void* Y_host[MILORA_NMOD];
+} milora_host_step;
+
+milora_status milora_step_host_workspace(const milora_ctx* ctx, const milora_host_step* step, size_t* bytes);
+milora_status milora_step_host(milora_ctx* ctx, const milora_host_step* step, void* workspace_dev,
+                               size_t workspace_bytes, void* stream);
+
 /* Waits for `stream`, then reads and clears the device error flag.  *device_flag_out is 0 when no
  * kernel skipped anything; the return value is MILORA_E_DEVICE_INDEX otherwise. */
 milora_status milora_poll_error(milora_ctx* ctx, int* device_flag_out, void* stream);

@@ -43,6 +43,13 @@ class Groups(C.Structure):
     _fields_ = [("ws_dev", C.c_void_p), ("n_seq", C.c_int), ("T", C.c_int)]
 
 
+class HostStep(C.Structure):
+    _fields_ = [("layer", C.c_int), ("n_prompts", C.c_int), ("cu_prompts_host", C.c_void_p),
+                ("prompt_slot_host", C.c_void_p), ("H_host", C.c_void_p), ("n_seq", C.c_int), ("T", C.c_int),
+                ("cu_seq_host", C.c_void_p), ("seq_slot_host", C.c_void_p), ("X_host", C.c_void_p * 7),
+                ("Y_host", C.c_void_p * 7)]
+
+
 # name -> (restype, argtypes); every symbol include/milora.h declares
 _VP, _I, _F = C.c_void_p, C.c_int, C.c_float
 SIGNATURES = {
@@ -67,6 +74,8 @@ SIGNATURES = {
     "milora_apply_prefill": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_decode_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
     "milora_apply_prefill_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
+    "milora_step_host_workspace": (_I, [_VP, C.POINTER(HostStep), C.POINTER(C.c_size_t)]),
+    "milora_step_host": (_I, [_VP, C.POINTER(HostStep), _VP, C.c_size_t, _VP]),
     "milora_poll_error": (_I, [_VP, C.POINTER(_I), _VP]),
 }
 
@@ -296,6 +305,51 @@ class Milora:
 
     def apply_prefill_multi(self, layer, modules, Xs, Ys, groups: Groups, stream=None):
         self._multi(self.lib.milora_apply_prefill_multi, "milora_apply_prefill_multi", layer, modules, Xs, Ys, groups, stream)
+
+    # -- one step from host buffers ------------------------------------------------------
+    def make_host_step(self, layer, cu_prompts, prompt_slot, H, cu_seq, seq_slot, T, Xs, Ys) -> HostStep:
+        """Descriptor of milora_step_host.  All tensors are HOST tensors (pinned for asynchronous copies):
+        cu_prompts / prompt_slot / H describe the prompts to route (None: no routing); cu_seq / seq_slot the
+        step's sequences; Xs / Ys are dicts module -> [T, d1] / [T, d2] host tensors.  The caller keeps the
+        tensors alive until the stream has been synchronised."""
+        def host(t, dtype, name):
+            if t is None:
+                return None
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dtype:
+                raise ValueError(f"{name} must be a contiguous host tensor of dtype {dtype}")
+            return t
+        st = HostStep()
+        st.layer = layer
+        st.n_prompts = 0 if prompt_slot is None else prompt_slot.numel()
+        st.cu_prompts_host = _ptr(host(cu_prompts, torch.int32, "cu_prompts"))
+        st.prompt_slot_host = _ptr(host(prompt_slot, torch.int32, "prompt_slot"))
+        st.H_host = _ptr(host(H, self.torch_dtype, "H"))
+        st.n_seq = 0 if seq_slot is None else seq_slot.numel()
+        st.T = T
+        st.cu_seq_host = _ptr(host(cu_seq, torch.int32, "cu_seq"))
+        st.seq_slot_host = _ptr(host(seq_slot, torch.int32, "seq_slot"))
+        for m in range(N_MOD):
+            x, y = Xs.get(m), Ys.get(m)
+            if (x is None) != (y is None):
+                raise ValueError("X and Y must be given together")
+            if x is not None:
+                d1, d2 = self.module_dims(m)
+                if tuple(x.shape) != (T, d1) or tuple(y.shape) != (T, d2):
+                    raise ValueError(f"host step: module {m} needs X [{T},{d1}] and Y [{T},{d2}]")
+            st.X_host[m] = _ptr(host(x, self.torch_dtype, "X"))
+            st.Y_host[m] = _ptr(host(y, self.torch_dtype, "Y"))
+        return st
+
+    def step_host_workspace(self, step: HostStep) -> int:
+        n = C.c_size_t(0)
+        self._check(self.lib.milora_step_host_workspace(self.h, C.byref(step), C.byref(n)), "milora_step_host_workspace")
+        return n.value
+
+    def step_host(self, step: HostStep, workspace, stream=None):
+        if not workspace.is_cuda or workspace.dtype != torch.uint8:
+            raise ValueError("workspace must be a CUDA uint8 tensor")
+        self._check(self.lib.milora_step_host(self.h, C.byref(step), workspace.data_ptr(), workspace.numel(),
+                                              _stream(stream)), "milora_step_host")
 
     def poll_error(self, stream=None) -> int:
         flag = C.c_int(0)

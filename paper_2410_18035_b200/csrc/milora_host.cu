@@ -499,6 +499,118 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
   return apply_common(ctx, layer, n_sites, modules, X_dev, Y_dev, groups, true, stream);
 }
 
+// ---- one step from host buffers ---------------------------------------------------------------------
+namespace {
+struct HostStepPlan {
+  size_t H, cu_p, slot_p, cu_s, slot_s, ws, X[MILORA_NMOD], Y[MILORA_NMOD], total;
+  size_t ws_stride;
+  int T_p;
+};
+size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
+
+milora_status plan_host_step(const milora_ctx* ctx, const milora_host_step* st, HostStepPlan* pl) {
+  if (!ctx || !st || !pl) return MILORA_E_ARG;
+  if (st->layer < 0 || st->layer >= ctx->desc.n_layers) return MILORA_E_ARG;
+  if (st->n_prompts < 0 || st->n_seq < 0 || st->T < 0) return MILORA_E_ARG;
+  if (st->n_prompts > kMaxSeq || st->n_seq > kMaxSeq) return MILORA_E_CAPACITY;
+  if (st->n_prompts > 0 && (!st->cu_prompts_host || !st->prompt_slot_host)) return MILORA_E_ARG;
+  if (st->n_seq > 0 && (!st->cu_seq_host || !st->seq_slot_host)) return MILORA_E_ARG;
+  pl->T_p = st->n_prompts > 0 ? st->cu_prompts_host[st->n_prompts] : 0;
+  if (pl->T_p < 0 || (pl->T_p > 0 && !st->H_host)) return MILORA_E_ARG;
+  size_t o = 0;
+  pl->H = o; o += up256((size_t)pl->T_p * ctx->desc.d_model * ctx->elem);
+  pl->cu_p = o; o += up256((size_t)(st->n_prompts + 1) * 4);
+  pl->slot_p = o; o += up256((size_t)st->n_prompts * 4 + 4);
+  pl->cu_s = o; o += up256((size_t)(st->n_seq + 1) * 4);
+  pl->slot_s = o; o += up256((size_t)st->n_seq * 4 + 4);
+  pl->ws_stride = group_layout(st->n_seq, st->T).total;
+  pl->ws = o; o += up256(pl->ws_stride * 4);
+  for (int m = 0; m < MILORA_NMOD; ++m) {
+    pl->X[m] = pl->Y[m] = 0;
+    if ((st->X_host[m] == nullptr) != (st->Y_host[m] == nullptr)) return MILORA_E_ARG;
+    if (!st->X_host[m]) continue;
+    int d1, d2;
+    module_dims(ctx->desc, m, &d1, &d2);
+    pl->X[m] = o; o += up256((size_t)st->T * d1 * ctx->elem);
+    pl->Y[m] = o; o += up256((size_t)st->T * d2 * ctx->elem);
+  }
+  pl->total = o;
+  return MILORA_OK;
+}
+}  // namespace
+
+milora_status milora_step_host_workspace(const milora_ctx* ctx, const milora_host_step* step, size_t* bytes) {
+  if (!bytes) return MILORA_E_ARG;
+  HostStepPlan pl;
+  milora_status st = plan_host_step(ctx, step, &pl);
+  if (st != MILORA_OK) return st;
+  *bytes = pl.total;
+  return MILORA_OK;
+}
+
+milora_status milora_step_host(milora_ctx* ctx, const milora_host_step* step, void* workspace_dev,
+                               size_t workspace_bytes, void* stream) {
+  HostStepPlan pl;
+  milora_status st = plan_host_step(ctx, step, &pl);
+  if (st != MILORA_OK) return st;
+  if (!workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) & 255) || workspace_bytes < pl.total)
+    return MILORA_E_ARG;
+  char* w = static_cast<char*>(workspace_dev);
+  cudaStream_t s = as_stream(stream);
+  const size_t e = ctx->elem;
+  auto h2d = [&](size_t off, const void* src, size_t bytes) -> cudaError_t {
+    return bytes ? cudaMemcpyAsync(w + off, src, bytes, cudaMemcpyHostToDevice, s) : cudaSuccess;
+  };
+  // inputs
+  MILORA_CUDA(ctx, h2d(pl.H, step->H_host, (size_t)pl.T_p * ctx->desc.d_model * e));
+  if (step->n_prompts > 0) {
+    MILORA_CUDA(ctx, h2d(pl.cu_p, step->cu_prompts_host, (size_t)(step->n_prompts + 1) * 4));
+    MILORA_CUDA(ctx, h2d(pl.slot_p, step->prompt_slot_host, (size_t)step->n_prompts * 4));
+  }
+  if (step->n_seq > 0) {
+    MILORA_CUDA(ctx, h2d(pl.cu_s, step->cu_seq_host, (size_t)(step->n_seq + 1) * 4));
+    MILORA_CUDA(ctx, h2d(pl.slot_s, step->seq_slot_host, (size_t)step->n_seq * 4));
+  }
+  int modules[MILORA_NMOD], n_sites = 0;
+  const void* X[MILORA_NMOD];
+  void* Y[MILORA_NMOD];
+  for (int m = 0; m < MILORA_NMOD; ++m) {
+    if (!step->X_host[m]) continue;
+    int d1, d2;
+    module_dims(ctx->desc, m, &d1, &d2);
+    MILORA_CUDA(ctx, h2d(pl.X[m], step->X_host[m], (size_t)step->T * d1 * e));
+    MILORA_CUDA(ctx, h2d(pl.Y[m], step->Y_host[m], (size_t)step->T * d2 * e));
+    modules[n_sites] = m;
+    X[n_sites] = w + pl.X[m];
+    Y[n_sites] = w + pl.Y[m];
+    ++n_sites;
+  }
+  // the path
+  if (step->n_prompts > 0 && pl.T_p > 0) {
+    st = milora_route(ctx, step->layer, w + pl.H, reinterpret_cast<const int32_t*>(w + pl.cu_p),
+                      reinterpret_cast<const int32_t*>(w + pl.slot_p), step->n_prompts, pl.T_p, nullptr, nullptr, stream);
+    if (st != MILORA_OK) return st;
+  }
+  if (step->n_seq > 0 && step->T > 0 && n_sites > 0) {
+    int32_t* ws = reinterpret_cast<int32_t*>(w + pl.ws);
+    st = milora_group(ctx, step->layer, 1, reinterpret_cast<const int32_t*>(w + pl.cu_s),
+                      reinterpret_cast<const int32_t*>(w + pl.slot_s), step->n_seq, step->T, ws, pl.ws_stride, stream);
+    if (st != MILORA_OK) return st;
+    milora_groups g{ws, step->n_seq, step->T};
+    st = milora_apply_prefill_multi(ctx, step->layer, n_sites, modules, X, Y, &g, stream);
+    if (st != MILORA_OK) return st;
+    st = milora_apply_decode_multi(ctx, step->layer, n_sites, modules, X, Y, &g, stream);
+    if (st != MILORA_OK) return st;
+    // outputs
+    for (int i = 0; i < n_sites; ++i) {
+      int d1, d2;
+      module_dims(ctx->desc, modules[i], &d1, &d2);
+      MILORA_CUDA(ctx, cudaMemcpyAsync(step->Y_host[modules[i]], Y[i], (size_t)step->T * d2 * e, cudaMemcpyDeviceToHost, s));
+    }
+  }
+  return MILORA_OK;
+}
+
 milora_status milora_poll_error(milora_ctx* ctx, int* device_flag_out, void* stream) {
   if (!ctx || !device_flag_out) return MILORA_E_ARG;
   cudaStream_t s = as_stream(stream);

@@ -264,3 +264,45 @@ def test_host_validation_reports_errors_before_launch():
     ml.route_table_write(2, [[3, -1]])
     assert ml.route_table_read(2, 1).tolist() == [[3, -1]]
     ml.close()
+
+
+def test_step_from_host_buffers_matches_oracle():
+    """milora_step_host: inputs in pinned host memory, outputs back in host memory, one call per step."""
+    base = get_workload("c1")
+    lens = np.array([130, 40, 7, 64, 1, 1, 1], dtype=np.int32)
+    w = scaled_workload(base, name="host_step", dtype="bf16", d_model=512, d_ff=1408, d_kv=128, rank=16, n_tenants=3,
+                        request_tenant=np.array([0, 1, 2, 0, 1, 2, 0], dtype=np.int32), prompt_len=lens,
+                        prefill_ids=np.arange(4), decode_ids=np.arange(4, 7), has_base_weights=False, n_layers=1)
+    lw = _loaded(w)
+    ml = lw.ml
+    prefill, decode = [0, 1, 2, 3], [4, 5, 6]
+    # the decode requests were routed earlier from their own prompts
+    lw.route(0, decode)
+    cu, slots, T = lw.seq_arrays(prefill, decode)
+    pin = lambda t: t.cpu().pin_memory()
+    cu_p = pin(torch.from_numpy(w.cu_seqlens(prefill)))
+    slot_p = pin(torch.tensor(prefill, dtype=torch.int32))
+    H = pin(w.hidden_batch(0, prefill))
+    Xs = {m: pin(w.module_input(0, m, T, 3)) for m in range(7)}
+    Ybs = {m: w.base_output(0, m, T, 3) for m in range(7)}
+    Ys = {m: pin(Ybs[m].clone()) for m in range(7)}
+    step = ml.make_host_step(0, cu_p, slot_p, H, pin(cu), pin(slots), T, Xs, Ys)
+    ws = torch.empty(ml.step_host_workspace(step) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    ml.step_host(step, ws)
+    torch.cuda.synchronize()
+    assert ml.poll_error() == 0
+    table = ml.route_table_read(0, w.n_requests).numpy()
+    tmp = np.full((w.n_requests, 1), -1, dtype=np.int32)
+    _, margins = R.route_requests(w, 0, prefill, tmp)
+    compare_routes(table[prefill, 0], tmp[prefill, 0], margins)
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu.cpu().numpy()))
+    for m in range(7):
+        y_o = R.apply_site(w, 0, m, Xs[m], Ybs[m], token_slot, table[:, 0])
+        assert_apply_close(Ys[m], y_o, Ybs[m], "bf16", what=f"host step module {m}")
+    # a workspace that is too small is refused before anything is enqueued
+    from paper_2410_18035_b200 import MiloraError
+    with pytest.raises(MiloraError) as e:
+        ml.step_host(step, ws[:1024])
+    assert e.value.status == 1
+    lw.close()
