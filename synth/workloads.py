@@ -237,3 +237,10 @@ def scaled_workload(base: Workload, **overrides) -> Workload:
     d = {f.name: getattr(base, f.name) for f in dataclasses.fields(base) if f.name != "_cache"}
     d.update(overrides)
     return Workload(**d)
+
+
+def shard_by_tenant(request_tenant, world_size: int):
+    """Requests of each rank when tenants are placed round-robin (tenant % world_size): every adapter lives on
+    exactly one rank and a request follows its tenant, so no rank ever needs another rank's data."""
+    t = np.asarray(request_tenant)
+    return [np.nonzero(t % world_size == r)[0] for r in range(world_size)]

@@ -1,0 +1,79 @@
+"""The N > 1 path on CPU ranks (gloo, world size 2): requests are sharded by tenant, every rank works on its own
+shard with no data-path collective, and the only communication is the barrier and the MAX of the step times."""
+import os
+import socket
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import reference_run as R
+    from synth import get_workload
+    from synth.workloads import shard_by_tenant
+
+    w = get_workload("c1")
+    mine = shard_by_tenant(w.request_tenant, world)[rank]
+    table = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+    for layer in range(w.n_layers):
+        R.route_requests(w, layer, mine, table)
+    # timing protocol of the benchmark: barrier, then the slowest rank defines the step time
+    dist.barrier()
+    t = torch.tensor([1.0 + rank], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    # gather the shards' route rows (a test-side check only; the data path itself never communicates)
+    rows = [torch.zeros((w.n_requests, w.n_layers), dtype=torch.int32) for _ in range(world)]
+    dist.all_gather(rows, torch.from_numpy(table))
+    if rank == 0:
+        np.save(os.path.join(out_dir, "gathered.npy"), np.stack([r.numpy() for r in rows]))
+        np.save(os.path.join(out_dir, "tmax.npy"), t.numpy())
+    dist.destroy_process_group()
+
+
+def test_tenant_sharding_over_two_gloo_ranks(tmp_path):
+    from oracle import reference_run as R
+    from synth import get_workload
+    from synth.workloads import shard_by_tenant
+
+    world = 2
+    mp.spawn(_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    gathered = np.load(tmp_path / "gathered.npy")
+    w = get_workload("c1")
+    full, _ = R.full_route_table(w)
+    shards = shard_by_tenant(w.request_tenant, world)
+    # the shards partition the requests, every tenant sits on exactly one rank
+    assert sorted(np.concatenate(shards).tolist()) == list(range(w.n_requests))
+    for r in range(world):
+        assert set(w.request_tenant[shards[r]] % world) <= {r}
+        assert np.array_equal(gathered[r][shards[r]], full[shards[r]])          # same decisions as one process
+        other = np.setdiff1d(np.arange(w.n_requests), shards[r])
+        assert np.all(gathered[r][other] == -1)                                # and nothing outside the shard
+    assert np.load(tmp_path / "tmax.npy")[0] == 2.0                            # MAX over ranks
+
+
+def test_shard_by_tenant_structure():
+    from synth import get_workload
+    from synth.workloads import shard_by_tenant
+    w = get_workload("c4")
+    for world in (1, 2, 4, 8):
+        shards = shard_by_tenant(w.request_tenant, world)
+        assert sum(len(s) for s in shards) == w.n_requests
+        tenants = [set(w.request_tenant[s].tolist()) for s in shards]
+        for a in range(world):
+            for b in range(a + 1, world):
+                assert not (tenants[a] & tenants[b])
