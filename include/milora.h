@@ -130,7 +130,8 @@ milora_status milora_request_close(milora_ctx* ctx, int slot);
  * when not NULL, logits_out_dev [P][7] fp32 (g(h) W_r + bias) and probs_out_dev [P][7] fp32 (their
  * softmax).
  * Prompts whose slot is closed or whose tenant has no router at this layer get route -1.
- * One fused launch; deterministic (fixed reduction order).  The first call, and any call with more
+ * Two launches (streaming partial reduction, then one CTA per prompt); deterministic (fixed reduction
+ * order, no atomics on data).  The first call, and any call with more
  * rows than every earlier one, grows an internal scratch buffer (cudaMalloc after a stream sync). */
 milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const int32_t* cu_seqlens_dev,
                            const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
@@ -142,15 +143,15 @@ milora_status milora_route(milora_ctx* ctx, int layer, const void* H_dev, const 
  * whose memory pool already owns the whole device, inside a region where the allocator is frozen, or on
  * a latency path where the implicit device synchronisation of cudaMalloc/cudaFree is not acceptable.
  * This entry point takes the same arguments and gives the same results, but keeps its scratch (partial
- * column sums and per-prompt completion counters) in a fixed array inside the library image:
+ * column sums and one scheduling word) in a fixed array inside the library image:
  *   - the array is 16 MiB + 16 KiB and is held by every GPU that loads the library until the process
  *     exits;
- *   - a call needs (T_total / 64 + P) * (d_model + 2) floats of it and P counters; a call that needs
+ *   - a call needs (T_total / 64 + P) * (d_model + 2) floats of it; a call that needs
  *     more than 4 Mi floats, or has P > 4096, is rejected with MILORA_E_CAPACITY before any launch;
  *   - the first call on a device looks up the array's device address (cudaGetSymbolAddress); the
  *     context's device must be current (else MILORA_E_STATE), and this first call should be made
  *     before any stream capture begins;
- *   - all calls, from every context on that device, share the array: the counters are cleared on
+ *   - all calls, from every context on that device, share the array: its scheduling word is cleared on
  *     `stream` at the start of each call, but two calls that overlap on the GPU (different streams)
  *     race on it, so keep calls of this entry point ordered on one stream;
  *   - it calls no cudaMalloc, cudaFree or other allocating routine.  Pending table updates made by

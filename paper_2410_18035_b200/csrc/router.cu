@@ -1,22 +1,20 @@
-// Prompt-aware router (Section 3.3, Eq. 2-3; Appendix C; Eq. 7), one fused launch per layer:
+// Prompt-aware router (Section 3.3, Eq. 2-3; Appendix C; Eq. 7):
 // pooling over the prompt's rows -> activation g -> 7 dot products with W_r -> softmax -> argmax,
 // written to the int32 route table.
 //
-// The kernel is bound by reading H (e * n_p * d bytes per prompt).  Work is cut into items of
-// kRows consecutive rows x one block of kThreads 16-byte column groups; every thread streams its
-// column group with eight 128-bit loads in flight and every item writes fp32 partial column sums to
-// scratch.  CTAs take their first item by index and further items from an atomic counter (fetched
-// one item ahead, so its latency is hidden), so all SMs stay busy whatever the prompt lengths.
-// Nothing is synchronised per item: a CTA remembers which prompts it contributed to and, when it has
-// run out of items, publishes its counts with one fence; the CTA whose count completes a prompt
-// combines that prompt's partials in chunk order (nobody waits), so the result does not depend on
-// scheduling.
+// Two launches.  Pass 1 is bound by reading H (e * n_p * d bytes per prompt): a unit is one 64-row chunk of a
+// prompt x one strip of 32 sixteen-byte column groups and belongs to ONE WARP, which streams its rows with
+// eight independent 128-bit loads per batch, accumulates in fp32 in row order and writes the partial column
+// sums to scratch.  Warps take their first unit by index and later ones from an atomic counter (fetched one
+// unit ahead); they never synchronise with each other, so every SM has dozens of independent load chains in
+// flight.  Pass 2 (one CTA per prompt) adds the partials in chunk order, applies g, does the 7 dot products,
+// softmax and argmax.  No fences, no spin-waits; the result does not depend on scheduling.
 #include <cfloat>
 
 #include "milora_internal.h"
 
 // Scratch of milora_route_static: partial column sums and chunk statistics, followed by the scheduling
-// words and one completion counter per prompt.  It lives in the library image, so every GPU that loads
+// word.  It lives in the library image, so every GPU that loads
 // the library holds it (16 MiB + 16 KiB) until the process exits, and every call of that entry point
 // shares it.
 constexpr size_t kStaticPartialFloats = size_t(4) << 20;
@@ -26,10 +24,9 @@ static __device__ __align__(256) float g_route_static_scratch[kStaticPartialFloa
 namespace milora {
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kRows = 64;
-constexpr int kSchedWords = 2;     // [0] next dynamic item, [1] CTAs that have finished
 
 template <typename T> struct VecOf;
 template <> struct VecOf<float> {
@@ -153,44 +150,200 @@ struct RouteArgs {
   float* probs_out;
   float* partial;     // [total_chunks][d]
   float* stats;       // [total_chunks][2]  (self-attention pooler: chunk max, chunk sum of exp)
-  int32_t* sched;     // kSchedWords scheduling words, then one completion counter per prompt; zero on entry and exit
-  int layer, P, d, n_colblk;
+  int32_t* sched;     // next dynamic unit; zero on entry, put back to zero by pass 2
+  int layer, P, d, n_strips;
 };
 
-constexpr int kMaxTouched = 32;   // prompts a CTA may contribute to before it has to publish its counts
-
-// Combine the partials of prompt p (all of its items are complete and visible) and write its route.
-template <typename T>
-__device__ void finalize_prompt(const RouteArgs& a, int p, int chunk0, int n_chunks, float* red) {
-  constexpr int V = VecOf<T>::N;
-  const int tid = threadIdx.x, d = a.d;
+// Router entry of prompt p, or nullptr when its slot is closed / its tenant has no router at this layer.
+__device__ __forceinline__ const RouterEntry* router_of(const RouteArgs& a, int p, int* slot_out) {
   const int slot = a.seq_slot[p];
-  const bool slot_ok = slot >= 0 && slot < a.tab.max_requests;
-  const int tenant = slot_ok ? a.tab.slot_tenant[slot] : -1;
-  const RouterEntry* rp = (tenant >= 0 && tenant < a.tab.max_tenants)
-                              ? &a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer] : nullptr;
-  if (!rp || rp->W == nullptr || rp->pool < 0) {
-    // closed slot or no router for this tenant at this layer: the request stays "not routed"
-    if (tid == 0) {
-      if (slot_ok) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
-      else atomicOr(a.tab.err, ERR_BAD_SLOT);
-      a.sched[kSchedWords + p] = 0;
+  *slot_out = slot;
+  if (slot < 0 || slot >= a.tab.max_requests) return nullptr;
+  const int tenant = a.tab.slot_tenant[slot];
+  if (tenant < 0 || tenant >= a.tab.max_tenants) return nullptr;
+  const RouterEntry* r = &a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer];
+  return (r->W != nullptr && r->pool >= 0) ? r : nullptr;
+}
+
+// ---- pass 1: partial column reductions -------------------------------------------------------------
+// A unit is one 64-row chunk of a prompt x one strip of 32 sixteen-byte column groups, handled by ONE
+// WARP; warps walk the units with a fixed stride and never synchronise with each other, so an SM always
+// has dozens of independent load chains in flight.  Dynamic shared memory: chunk_start[P+1], pool[P].
+template <typename T>
+__global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
+  extern __shared__ int32_t sm_i[];
+  int32_t* chunk_start = sm_i;
+  int32_t* pool_sm = sm_i + (a.P + 1);
+  __shared__ int32_t carry;
+  __shared__ int32_t wsum[kWarps];
+  __shared__ float u_all[kWarps][kRows];
+  constexpr int V = VecOf<T>::N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int d = a.d;
+  const T* H = static_cast<const T*>(a.H);
+
+  // per-CTA prefix over prompts: chunks per prompt (from the lengths) and the pooler of each prompt
+  if (tid == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < a.P; base += kThreads) {
+    const int p = base + tid;
+    int chunks = 0;
+    if (p < a.P) {
+      const int n_p = a.cu[p + 1] - a.cu[p];
+      if (n_p > 0) chunks = (n_p + kRows - 1) / kRows;
+      int slot;
+      const RouterEntry* r = router_of(a, p, &slot);
+      pool_sm[p] = r ? r->pool : -1;
     }
+    int sc = chunks;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int tc = __shfl_up_sync(0xffffffffu, sc, o);
+      if (lane >= o) sc += tc;
+    }
+    if (lane == 31) wsum[warp] = sc;
     __syncthreads();
+    int off = carry;
+    for (int w = 0; w < warp; ++w) off += wsum[w];
+    if (p < a.P) chunk_start[p] = off + sc - chunks;
+    __syncthreads();
+    if (tid == kThreads - 1) carry = off + sc;
+    __syncthreads();
+  }
+  if (tid == 0) chunk_start[a.P] = carry;
+  __syncthreads();
+  const int total_units = chunk_start[a.P] * a.n_strips;
+  float* u_sm = u_all[warp];
+
+  const int warps_total = gridDim.x * kWarps;
+  int u_next = blockIdx.x * kWarps + warp;
+  while (u_next < total_units) {
+    const int u = u_next;
+    {
+      // ask for the following unit now; the answer is only needed when this one is done
+      int fetched = 0;
+      if (lane == 0) fetched = warps_total + atomicAdd(a.sched, 1);
+      u_next = __shfl_sync(0xffffffffu, fetched, 0);
+    }
+    const int cg = u / a.n_strips, strip = u % a.n_strips;
+    int lo = 0, hi = a.P;                       // prompt of this chunk: last p with chunk_start[p] <= cg
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (chunk_start[mid] <= cg) lo = mid; else hi = mid;
+    }
+    const int p = lo;
+    const int pool = pool_sm[p];
+    if (pool < 0) continue;
+    const int rc = cg - chunk_start[p];
+    const int row_lo = a.cu[p], row_hi = a.cu[p + 1];
+    int r0 = row_lo + rc * kRows;
+    int nr = min(kRows, row_hi - r0);
+    if (pool == MILORA_POOL_LAST) {             // only the prompt's last row is pooled; its last chunk holds it
+      if (rc != chunk_start[p + 1] - chunk_start[p] - 1) continue;
+      r0 = row_hi - 1;
+      nr = 1;
+    }
+    float* part = a.partial + (size_t)cg * d;
+    if (pool == MILORA_POOL_SELFATTN) {
+      // Appendix C needs whole rows: the warp of strip 0 does the chunk alone.  u_t = H[t,:] . w_sa, exp weights
+      // relative to the chunk max, then the weighted column sums strip by strip.
+      if (strip != 0) continue;
+      int slot;
+      const RouterEntry* r = router_of(a, p, &slot);
+      const T* wsa = static_cast<const T*>(r->Wsa);
+      for (int t = 0; t < nr; ++t) {
+        const T* row = H + (size_t)(r0 + t) * d;
+        float acc = 0.f;
+        for (int c = lane * V; c < d; c += 32 * V) {
+          float hv[V], wv[V];
+          VecOf<T>::load(row + c, hv);
+          VecOf<T>::load(wsa + c, wv);
+#pragma unroll
+          for (int i = 0; i < V; ++i) acc = fmaf(hv[i], wv[i], acc);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) u_sm[t] = acc;
+      }
+      __syncwarp();
+      float m = -FLT_MAX;
+      for (int t = 0; t < nr; ++t) m = fmaxf(m, u_sm[t]);
+      __syncwarp();
+      for (int t = lane; t < nr; t += 32) u_sm[t] = expf(u_sm[t] - m);
+      __syncwarp();
+      float l = 0.f;
+      for (int t = 0; t < nr; ++t) l += u_sm[t];
+      if (lane == 0) {
+        a.stats[2 * (size_t)cg] = m;
+        a.stats[2 * (size_t)cg + 1] = l;
+      }
+      for (int c0 = lane * V; c0 < d; c0 += 32 * V) {
+        float acc[V];
+        reduce_rows<T, kRedWeighted>(H + (size_t)r0 * d + c0, d, nr, u_sm, acc);
+#pragma unroll
+        for (int i = 0; i < V; i += 4)
+          *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+      }
+      __syncwarp();
+      continue;
+    }
+    const int c0 = (strip * 32 + lane) * V;
+    if (c0 < d) {
+      float acc[V];
+      const T* col = H + (size_t)r0 * d + c0;
+      if (pool == MILORA_POOL_MAX) reduce_rows<T, kRedMax>(col, d, nr, u_sm, acc);
+      else reduce_rows<T, kRedSum>(col, d, nr, u_sm, acc);
+#pragma unroll
+      for (int i = 0; i < V; i += 4)
+        *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    }
+  }
+}
+
+// ---- pass 2: one CTA per prompt combines the partials in chunk order and routes -----------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
+  constexpr int V = VecOf<T>::N;
+  __shared__ float red[MILORA_NMOD * kWarps];
+  __shared__ int32_t wsum[kWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int p = blockIdx.x, d = a.d;
+  // first scratch row of this prompt = number of chunks of the prompts before it
+  int mine = 0;
+  for (int q = tid; q < p; q += kThreads) {
+    const int n_q = a.cu[q + 1] - a.cu[q];
+    if (n_q > 0) mine += (n_q + kRows - 1) / kRows;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+  if (lane == 0) wsum[warp] = mine;
+  __syncthreads();
+  int chunk0 = 0;
+  for (int w = 0; w < kWarps; ++w) chunk0 += wsum[w];
+  const int n_p = a.cu[p + 1] - a.cu[p];
+  int n_chunks = n_p > 0 ? (n_p + kRows - 1) / kRows : 0;
+  int slot;
+  const RouterEntry* rp = router_of(a, p, &slot);
+  if (!rp || n_chunks == 0) {
+    // closed slot, no router for this tenant at this layer, or an empty prompt: the request stays "not routed"
+    if (tid == 0) {
+      if (slot >= 0 && slot < a.tab.max_requests) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
+      else atomicOr(a.tab.err, ERR_BAD_SLOT);
+      if (p == 0) *a.sched = 0;
+    }
     return;
   }
   const RouterEntry& r = *rp;
   const int pool = r.pool;
   const bool sa = pool == MILORA_POOL_SELFATTN;
-  const int n_p = a.cu[p + 1] - a.cu[p];
   if (pool == MILORA_POOL_LAST) { chunk0 += n_chunks - 1; n_chunks = 1; }   // only the chunk with the last row counts
   const float* part0 = a.partial + (size_t)chunk0 * d;
   const float* st0 = a.stats + 2 * (size_t)chunk0;
   float gmax = -FLT_MAX, denom = 1.f;
   if (sa) {
-    for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, __ldcg(st0 + 2 * c));
+    for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, st0[2 * c]);
     denom = 0.f;
-    for (int c = 0; c < n_chunks; ++c) denom += expf(__ldcg(st0 + 2 * c) - gmax) * __ldcg(st0 + 2 * c + 1);
+    for (int c = 0; c < n_chunks; ++c) denom += expf(st0[2 * c] - gmax) * st0[2 * c + 1];
   }
   const T* W = static_cast<const T*>(r.W);
   float z[MILORA_NMOD];
@@ -207,10 +360,10 @@ __device__ void finalize_prompt(const RouteArgs& a, int p, int chunk0, int n_chu
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int c = min(cbase + k, n_chunks - 1);
-        wgt[k] = sa ? __ldcg(st0 + 2 * c) : 0.f;
+        wgt[k] = sa ? st0[2 * c] : 0.f;
 #pragma unroll
         for (int i = 0; i < V / 4; ++i)
-          q[k][i] = __ldcg(reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0 + 4 * i));
+          q[k][i] = *reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0 + 4 * i);
       }
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -259,6 +412,7 @@ __device__ void finalize_prompt(const RouteArgs& a, int p, int chunk0, int n_chu
 #pragma unroll
     for (int j = 0; j < MILORA_NMOD; ++j) { e[j] = expf(z[j] - zmax); sum += e[j]; }
     a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = best;
+    if (p == 0) *a.sched = 0;       // pass 1 of the next call starts its unit queue from zero
     if (a.logits_out) {
 #pragma unroll
       for (int j = 0; j < MILORA_NMOD; ++j) a.logits_out[(size_t)p * MILORA_NMOD + j] = z[j];
@@ -266,190 +420,6 @@ __device__ void finalize_prompt(const RouteArgs& a, int p, int chunk0, int n_chu
     if (a.probs_out) {
 #pragma unroll
       for (int j = 0; j < MILORA_NMOD; ++j) a.probs_out[(size_t)p * MILORA_NMOD + j] = e[j] / sum;
-    }
-    a.sched[kSchedWords + p] = 0;
-  }
-  __syncthreads();
-}
-
-// Dynamic shared memory: item_start[P+1], chunk_base[P+1].
-template <typename T>
-__global__ void __launch_bounds__(kThreads) route_kernel(RouteArgs a) {
-  extern __shared__ int32_t sm_i[];
-  int32_t* item_start = sm_i;
-  int32_t* chunk_base = sm_i + (a.P + 1);
-  __shared__ float red[MILORA_NMOD * kWarps];
-  __shared__ float u_sm[kRows];
-  __shared__ int32_t carry[2];
-  __shared__ int32_t wsum[2][kWarps];
-  __shared__ int32_t next_item, n_touched, n_done;
-  __shared__ int32_t touched_p[kMaxTouched], touched_n[kMaxTouched], done_p[kMaxTouched];
-  constexpr int V = VecOf<T>::N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int d = a.d;
-  const T* H = static_cast<const T*>(a.H);
-  int32_t* counters = a.sched + kSchedWords;
-
-  // ---- per-CTA prefix over prompts: how many items and scratch rows each prompt owns ----
-  if (tid == 0) { carry[0] = 0; carry[1] = 0; n_touched = 0; n_done = 0; }
-  __syncthreads();
-  for (int base = 0; base < a.P; base += kThreads) {
-    const int p = base + tid;
-    int items = 0, chunks = 0;
-    if (p < a.P) {
-      // The item count depends on the prompt length alone (one dependent load); items that turn out to have
-      // nothing to do (another pooler, a closed slot) return at once and the prompt is still finalized.
-      const int n_p = a.cu[p + 1] - a.cu[p];
-      if (n_p > 0) {
-        chunks = (n_p + kRows - 1) / kRows;
-        items = chunks * a.n_colblk;
-      } else if (blockIdx.x == 0) {
-        const int slot = a.seq_slot[p];      // an empty prompt has no items: mark it "not routed" here
-        if (slot >= 0 && slot < a.tab.max_requests) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
-        else atomicOr(a.tab.err, ERR_BAD_SLOT);
-      }
-    }
-    // inclusive scan of (items, chunks) over the prompts of this round
-    int si = items, sc = chunks;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int ti = __shfl_up_sync(0xffffffffu, si, o), tc = __shfl_up_sync(0xffffffffu, sc, o);
-      if (lane >= o) { si += ti; sc += tc; }
-    }
-    if (lane == 31) { wsum[0][warp] = si; wsum[1][warp] = sc; }
-    __syncthreads();
-    int offi = carry[0], offc = carry[1];
-    for (int w = 0; w < warp; ++w) { offi += wsum[0][w]; offc += wsum[1][w]; }
-    if (p < a.P) { item_start[p] = offi + si - items; chunk_base[p] = offc + sc - chunks; }
-    __syncthreads();
-    if (tid == kThreads - 1) { carry[0] = offi + si; carry[1] = offc + sc; }
-    __syncthreads();
-  }
-  if (tid == 0) { item_start[a.P] = carry[0]; chunk_base[a.P] = carry[1]; }
-  __syncthreads();
-  const int total_items = item_start[a.P];
-
-  // Publish the per-prompt item counts of this CTA; the CTA that completes a prompt's count finalizes it.
-  auto publish = [&]() {
-    __threadfence();                 // this CTA's partial sums are visible before its counts are
-    __syncthreads();
-    const int nt = n_touched;
-    for (int i = tid; i < nt; i += kThreads) {
-      const int p = touched_p[i];
-      const int n_items = item_start[p + 1] - item_start[p];
-      if (atomicAdd(counters + p, touched_n[i]) + touched_n[i] == n_items) done_p[atomicAdd(&n_done, 1)] = p;
-    }
-    __syncthreads();
-    const int nd = n_done;
-    if (nd > 0) __threadfence();     // the other CTAs' partial sums are visible before they are read
-    for (int i = 0; i < nd; ++i) {
-      const int p = done_p[i];
-      finalize_prompt<T>(a, p, chunk_base[p], chunk_base[p + 1] - chunk_base[p], red);
-    }
-    __syncthreads();
-    if (tid == 0) { n_touched = 0; n_done = 0; }
-    __syncthreads();
-  };
-
-  int it = blockIdx.x;
-  while (it < total_items) {
-    // ask for the next item now; the answer is needed only when this item is done
-    int fetched = 0;
-    if (tid == 0) fetched = (int)gridDim.x + atomicAdd(a.sched, 1);
-    // prompt of this item: last p with item_start[p] <= it
-    int lo = 0, hi = a.P;
-    while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if (item_start[mid] <= it) lo = mid; else hi = mid;
-    }
-    const int p = lo;
-    const int slot = a.seq_slot[p];
-    const int tenant = (slot >= 0 && slot < a.tab.max_requests) ? a.tab.slot_tenant[slot] : -1;
-    const RouterEntry* rp = (tenant >= 0 && tenant < a.tab.max_tenants)
-                                ? &a.tab.routers[(size_t)tenant * a.tab.n_layers + a.layer] : nullptr;
-    bool work = rp && rp->W != nullptr && rp->pool >= 0;    // the same for every thread of the CTA
-    const RouterEntry& r = *(work ? rp : a.tab.routers);
-    const int pool = work ? r.pool : -1;
-    const int row_lo = a.cu[p], row_hi = a.cu[p + 1];
-    const int local = it - item_start[p];
-    const bool sa = pool == MILORA_POOL_SELFATTN;
-    const int rc = local / a.n_colblk, cb = local % a.n_colblk;
-    int r0 = row_lo + rc * kRows;
-    int nr = min(kRows, row_hi - r0);
-    if (pool == MILORA_POOL_LAST) {          // only the last row is pooled: the prompt's last chunk holds it
-      work = work && rc == chunk_base[p + 1] - chunk_base[p] - 1;
-      r0 = row_hi - 1;
-      nr = 1;
-    }
-    if (sa) work = work && cb == 0;          // the self-attention pooler needs whole rows: one item per chunk
-    const int cb0 = sa ? 0 : cb;
-    const int cb1 = !work ? cb0 : (sa ? a.n_colblk : cb0 + 1);
-    float* part = a.partial + (size_t)(chunk_base[p] + rc) * d;
-
-    if (sa && work) {
-      // Appendix C: u_t = H[t,:] . w_sa for the rows of this chunk, then exp weights relative to the chunk max.
-      const T* wsa = static_cast<const T*>(r.Wsa);
-      for (int t = warp; t < nr; t += kWarps) {
-        const T* row = H + (size_t)(r0 + t) * d;
-        float acc = 0.f;
-        for (int c = lane * V; c < d; c += 32 * V) {
-          float hv[V], wv[V];
-          VecOf<T>::load(row + c, hv);
-          VecOf<T>::load(wsa + c, wv);
-#pragma unroll
-          for (int i = 0; i < V; ++i) acc = fmaf(hv[i], wv[i], acc);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) u_sm[t] = acc;
-      }
-      __syncthreads();
-      float m = -FLT_MAX;
-      for (int t = 0; t < nr; ++t) m = fmaxf(m, u_sm[t]);
-      __syncthreads();
-      float l = 0.f;
-      if (tid < nr) u_sm[tid] = expf(u_sm[tid] - m);
-      __syncthreads();
-      for (int t = 0; t < nr; ++t) l += u_sm[t];
-      if (tid == 0) {
-        a.stats[2 * (size_t)(chunk_base[p] + rc)] = m;
-        a.stats[2 * (size_t)(chunk_base[p] + rc) + 1] = l;
-      }
-    }
-
-    for (int cb = cb0; cb < cb1; ++cb) {
-      const int c0 = (cb * kThreads + tid) * V;
-      if (c0 < d) {
-        float acc[V];
-        const T* col = H + (size_t)r0 * d + c0;
-        if (pool == MILORA_POOL_MAX) reduce_rows<T, kRedMax>(col, d, nr, u_sm, acc);
-        else if (sa) reduce_rows<T, kRedWeighted>(col, d, nr, u_sm, acc);
-        else reduce_rows<T, kRedSum>(col, d, nr, u_sm, acc);
-#pragma unroll
-        for (int i = 0; i < V; i += 4)
-          *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
-      }
-    }
-
-    // ---- bookkeeping: remember the contribution, move to the prefetched item ----
-    if (tid == 0) {
-      const int nt = n_touched;
-      if (nt > 0 && touched_p[nt - 1] == p) touched_n[nt - 1] += 1;
-      else { touched_p[nt] = p; touched_n[nt] = 1; n_touched = nt + 1; }
-      next_item = fetched;
-    }
-    __syncthreads();
-    it = next_item;
-    if (n_touched == kMaxTouched) publish();
-  }
-  publish();
-
-  // ---- the CTA that leaves last puts the scheduling words back to zero for the next launch ----
-  if (tid == 0) {
-    __threadfence();
-    if (atomicAdd(a.sched + 1, 1) == (int)gridDim.x - 1) {
-      a.sched[0] = 0;
-      a.sched[1] = 0;
     }
   }
 }
@@ -481,22 +451,22 @@ milora_status transpose(milora_ctx* ctx, const void* in, void* out, int rows, in
 }
 
 struct RoutePlan {
-  int n_colblk;
-  size_t max_chunks, scratch_floats, max_items;
+  int n_strips;
+  size_t max_chunks, scratch_floats, max_units;
 };
 
 RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
   RoutePlan pl;
   const int d = ctx->desc.d_model;
   const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
-  pl.n_colblk = (d + kThreads * V - 1) / (kThreads * V);
+  pl.n_strips = (d + 32 * V - 1) / (32 * V);
   pl.max_chunks = (size_t)T_total / kRows + P;
   pl.scratch_floats = pl.max_chunks * d + 2 * pl.max_chunks;
-  pl.max_items = pl.max_chunks * pl.n_colblk;
+  pl.max_units = pl.max_chunks * pl.n_strips;
   return pl;
 }
 
-// `scratch` holds plan.scratch_floats floats; `sched` holds kSchedWords + P zeroed int32.
+// `scratch` holds plan.scratch_floats floats; `sched` is one zeroed int32.
 milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const void* H, const int32_t* cu,
                         const int32_t* seq_slot, int P, float* logits_out, float* probs_out, float* scratch, int32_t* sched,
                         cudaStream_t s) {
@@ -507,15 +477,22 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   a.partial = scratch;
   a.stats = scratch + pl.max_chunks * ctx->desc.d_model;
   a.sched = sched;
-  a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_colblk = pl.n_colblk;
-  const size_t smem = (size_t)(P + 1) * 2 * sizeof(int32_t);
-  int grid = (int)std::min<size_t>(pl.max_items, (size_t)ctx->sm_count * 8);
+  a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_strips = pl.n_strips;
+  const size_t smem = (size_t)(2 * P + 1) * sizeof(int32_t);
+  const bool f32 = ctx->desc.dtype == MILORA_F32;
+  // pass 1: one wave of resident CTAs (a warp's first unit is assigned by index, so every CTA must start at once)
+  int per_sm = 0;
+  if (f32) MILORA_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pool_partial_kernel<float>, kThreads, smem));
+  else MILORA_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pool_partial_kernel<__nv_bfloat16>, kThreads, smem));
+  if (per_sm < 1) per_sm = 1;
+  int grid = (int)std::min<size_t>((pl.max_units + kWarps - 1) / kWarps, (size_t)ctx->sm_count * per_sm);
   if (grid < 1) grid = 1;
-  if (ctx->desc.dtype == MILORA_F32) {
-    route_kernel<float><<<grid, kThreads, smem, s>>>(a);
-  } else {
-    route_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
-  }
+  if (f32) pool_partial_kernel<float><<<grid, kThreads, smem, s>>>(a);
+  else pool_partial_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
+  MILORA_CUDA(ctx, cudaGetLastError());
+  // pass 2: one CTA per prompt
+  if (f32) route_finalize_kernel<float><<<P, kThreads, 0, s>>>(a);
+  else route_finalize_kernel<__nv_bfloat16><<<P, kThreads, 0, s>>>(a);
   MILORA_CUDA(ctx, cudaGetLastError());
   return MILORA_OK;
 }
@@ -547,12 +524,12 @@ milora_status launch_route(milora_ctx* ctx, int layer, const void* H, const int3
     MILORA_CUDA(ctx, cudaMalloc(&ctx->d_scratch, pl.scratch_floats * sizeof(float)));
     ctx->scratch_floats = pl.scratch_floats;
   }
-  if ((size_t)P + kSchedWords > ctx->n_counters) {
+  if (ctx->n_counters < 1) {
     MILORA_CUDA(ctx, cudaStreamSynchronize(s));
     if (ctx->d_counters) MILORA_CUDA(ctx, cudaFree(ctx->d_counters));
     ctx->d_counters = nullptr;
     ctx->n_counters = 0;
-    size_t n = std::max<size_t>(P, 1024) + kSchedWords;
+    size_t n = 64;
     MILORA_CUDA(ctx, cudaMalloc(&ctx->d_counters, n * sizeof(int32_t)));
     MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_counters, 0, n * sizeof(int32_t), s));
     ctx->n_counters = n;
@@ -568,8 +545,8 @@ milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, con
   constexpr int kMaxDevices = 64;
   static float* scratch_of_device[kMaxDevices] = {nullptr};
   const RoutePlan pl = plan_route(ctx, P, T_total);
-  // the last kSchedWords floats of the partial area serve as the scheduling words, right in front of the counters
-  if (pl.scratch_floats + kSchedWords > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
+  // the scheduling word sits right behind the partial area
+  if (pl.scratch_floats > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
   int dev = -1;
   MILORA_CUDA(ctx, cudaGetDevice(&dev));
   if (dev != ctx->device) return MILORA_E_STATE;     // the context's device must be current
@@ -580,9 +557,9 @@ milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, con
     scratch_of_device[dev] = ptr;
   }
   float* scratch = scratch_of_device[dev];
-  int32_t* sched = reinterpret_cast<int32_t*>(scratch + kStaticPartialFloats - kSchedWords);
-  // The array keeps whatever the previous call left; the scheduling words and the counters have to start at zero.
-  MILORA_CUDA(ctx, cudaMemsetAsync(sched, 0, ((size_t)P + kSchedWords) * sizeof(int32_t), s));
+  int32_t* sched = reinterpret_cast<int32_t*>(scratch + kStaticPartialFloats);
+  // The array keeps whatever the previous call left; only the scheduling word has to start at zero.
+  MILORA_CUDA(ctx, cudaMemsetAsync(sched, 0, sizeof(int32_t), s));
   return run_route(ctx, pl, layer, H, cu, seq_slot, P, logits_out, probs_out, scratch, sched, s);
 }
 
