@@ -14,37 +14,52 @@
 namespace milora {
 namespace {
 
-constexpr int kGThreads = 1024;
+constexpr int kGMaxThreads = 1024;
 constexpr int kSeqBits = 12;  // kMaxSeq = 4096 sequences
 static_assert((1 << kSeqBits) == kMaxSeq, "kSeqBits must match kMaxSeq");
 constexpr int kSmemArrays = 8;
 
-// Exclusive prefix sum over the block of one int per thread; returns the exclusive value, *total gets the sum.
-__device__ inline int block_exscan(int v, int* total, int* wsum /* [33] */) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
+// Exclusive prefix sums over the block of N ints per thread (scanned together: three barriers in all);
+// returns the exclusive values in v, the block totals in total.  wsum holds N x 33 ints.
+template <int N>
+__device__ inline void block_exscan(int (&v)[N], int (&total)[N], int* wsum) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  int inc[N];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  __syncthreads();
-  if (lane == 31) wsum[warp] = inc;
-  __syncthreads();
-  if (warp == 0) {
-    int w = wsum[lane];
-    int winc = w;
+  for (int k = 0; k < N; ++k) {
+    inc[k] = v[k];
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int t = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += t;
+      int t = __shfl_up_sync(0xffffffffu, inc[k], o);
+      if (lane >= o) inc[k] += t;
     }
-    wsum[lane] = winc - w;
-    if (lane == 31) wsum[32] = winc;
   }
   __syncthreads();
-  *total = wsum[32];
-  return wsum[warp] + inc - v;
+  if (lane == 31) {
+#pragma unroll
+    for (int k = 0; k < N; ++k) wsum[k * 33 + warp] = inc[k];
+  }
+  __syncthreads();
+  if (warp == 0) {
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+      int w = lane < nwarps ? wsum[k * 33 + lane] : 0;
+      int winc = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += t;
+      }
+      wsum[k * 33 + lane] = winc - w;
+      if (lane == 31) wsum[k * 33 + 32] = winc;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    total[k] = wsum[k * 33 + 32];
+    v[k] = wsum[k * 33 + warp] + inc[k] - v[k];
+  }
 }
 
 struct GroupArgs {
@@ -59,9 +74,10 @@ struct GroupArgs {
 
 // Shared memory (int32): comp[n_pad], seq_lo[n_pad], seq_len[n_pad], tok_off[n_pad+1], seg_tile[n_pad+1],
 // seg_short[n_pad+1], seg_gather[n_pad+1] (kSmemArrays * n_pad + 8 in total).
-__global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
+__global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   extern __shared__ int32_t sm[];
-  __shared__ int wsum[33];
+  __shared__ int wsum[5 * 33];
+  const int kGThreads = blockDim.x;
   const int n_pad = a.n_pad, n_seq = a.n_seq;
   int32_t* comp = sm;
   int32_t* seq_lo = comp + n_pad;
@@ -105,7 +121,11 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
     comp[i] = c;
   }
   int n_excl;
-  block_exscan(excl, &n_excl, wsum);
+  {
+    int v1[1] = {excl}, t1[1];
+    block_exscan<1>(v1, t1, wsum);
+    n_excl = t1[0];
+  }
 
   // ---- 2. bitonic sort of the composite keys ----------------------------------------------
   for (int k = 2; k <= n_pad; k <<= 1) {
@@ -136,12 +156,10 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
     if (len >= kLongSeq) s_tile += (len + kTileRows - 1) / kTileRows;
     else s_short += len;
   }
-  int n_active, n_seg, n_tiles, n_short, n_act_seq;
-  int o_tok = block_exscan(s_tok, &n_active, wsum);
-  int o_head = block_exscan(s_head, &n_seg, wsum);
-  int o_tile = block_exscan(s_tile, &n_tiles, wsum);
-  int o_short = block_exscan(s_short, &n_short, wsum);
-  block_exscan(s_act, &n_act_seq, wsum);
+  int v5[5] = {s_tok, s_head, s_tile, s_short, s_act}, t5[5];
+  block_exscan<5>(v5, t5, wsum);
+  int o_tok = v5[0], o_head = v5[1], o_tile = v5[2], o_short = v5[3];
+  const int n_active = t5[0], n_seg = t5[1], n_tiles = t5[2], n_short = t5[3], n_act_seq = t5[4];
 
   TileJob* tiles = reinterpret_cast<TileJob*>(ws + a.lay.tiles);
   int32_t* gather_rows = ws + a.lay.gather_rows;
@@ -200,8 +218,13 @@ __global__ void __launch_bounds__(kGThreads) group_kernel(GroupArgs a) {
   const int s0 = min(tid * sper, n_seg), s1 = min(s0 + sper, n_seg);
   int g_cnt = 0;
   for (int s = s0; s < s1; ++s) g_cnt += (seg_short[s + 1] - seg_short[s] + kGatherRows - 1) / kGatherRows;
-  int n_gather;
-  int o_g = block_exscan(g_cnt, &n_gather, wsum);
+  int n_gather, o_g;
+  {
+    int v1[1] = {g_cnt}, t1[1];
+    block_exscan<1>(v1, t1, wsum);
+    o_g = v1[0];
+    n_gather = t1[0];
+  }
   GatherJob* gather = reinterpret_cast<GatherJob*>(ws + a.lay.gather);
   for (int s = s0; s < s1; ++s) {
     seg_gather[s] = o_g;
@@ -262,7 +285,9 @@ milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   if (smem > 48 * 1024) {
     MILORA_CUDA(ctx, cudaFuncSetAttribute(group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
-  group_kernel<<<n_layers, kGThreads, smem, s>>>(a);
+  // few sequences (a decode batch): a smaller block makes every barrier and scan cheaper
+  const int threads = std::max(128, std::min(kGMaxThreads, n_pad));
+  group_kernel<<<n_layers, threads, smem, s>>>(a);
   MILORA_CUDA(ctx, cudaGetLastError());
   return MILORA_OK;
 }
