@@ -121,6 +121,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t crank = cluster_ctarank();
   const int job_idx = blockIdx.x / kC;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n_jobs = a.ws[a.lay.header + H_NGATHER];
   if (job_idx >= n_jobs || job_idx >= a.lay.max_gather) return;          // same decision in the whole cluster
   const GatherJob job = reinterpret_cast<const GatherJob*>(a.ws + a.lay.gather)[job_idx];
@@ -317,8 +319,7 @@ milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySi
   }
   size_t grid = (size_t)a.lay.max_gather * kC;
   if (grid > 0x7fffffffull) return MILORA_E_CAPACITY;
-  decode_bf16_kernel<<<(unsigned)grid, kThreads, smem, s>>>(a);
-  MILORA_CUDA(ctx, cudaGetLastError());
+  MILORA_CUDA(ctx, launch_pdl(decode_bf16_kernel, dim3((unsigned)grid), dim3(kThreads), smem, s, a));
   return MILORA_OK;
 }
 

@@ -66,6 +66,8 @@ __global__ void __launch_bounds__(kThreads) apply_generic_kernel(ApplyArgs a) {
   __shared__ float v_sm[R][kMaxRank];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int job_idx = blockIdx.x / kSub, sub = blockIdx.x % kSub;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n_jobs = a.ws[a.lay.header + (DENSE ? H_NTILES : H_NGATHER)];
   if (job_idx >= n_jobs || job_idx >= (DENSE ? a.lay.max_tiles : a.lay.max_gather)) return;
 
@@ -187,13 +189,13 @@ milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites&
   if (grid < 1) grid = 1;
   if (grid > 0x7fffffffull) return MILORA_E_CAPACITY;
   const bool f32 = ctx->desc.dtype == MILORA_F32;
-  if (dense) {
-    if (f32) apply_generic_kernel<float, true><<<(unsigned)grid, kThreads, 0, s>>>(a);
-    else apply_generic_kernel<__nv_bfloat16, true><<<(unsigned)grid, kThreads, 0, s>>>(a);
-  } else {
-    if (f32) apply_generic_kernel<float, false><<<(unsigned)grid, kThreads, 0, s>>>(a);
-    else apply_generic_kernel<__nv_bfloat16, false><<<(unsigned)grid, kThreads, 0, s>>>(a);
-  }
+  const dim3 g3((unsigned)grid), b3(kThreads);
+  cudaError_t e;
+  if (dense) e = f32 ? launch_pdl(apply_generic_kernel<float, true>, g3, b3, 0, s, a)
+                     : launch_pdl(apply_generic_kernel<__nv_bfloat16, true>, g3, b3, 0, s, a);
+  else e = f32 ? launch_pdl(apply_generic_kernel<float, false>, g3, b3, 0, s, a)
+               : launch_pdl(apply_generic_kernel<__nv_bfloat16, false>, g3, b3, 0, s, a);
+  MILORA_CUDA(ctx, e);
   MILORA_CUDA(ctx, cudaGetLastError());
   return MILORA_OK;
 }

@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kKSplit, ks = blockIdx.x % kKSplit;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
   if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
@@ -214,6 +216,8 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kNSplit, ns = blockIdx.x % kNSplit;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
   if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
@@ -523,10 +527,8 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
   MILORA_CUDA(ctx, cudaFuncSetAttribute(prefill_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)expand_smem));
   const size_t grid_s = (size_t)lay.max_tiles * kKSplit, grid_e = (size_t)lay.max_tiles * kNSplit;
   if (grid_s > 0x7fffffffull || grid_e > 0x7fffffffull) return MILORA_E_CAPACITY;
-  prefill_shrink_kernel<<<(unsigned)grid_s, kShrinkThreads, shrink_smem, s>>>(sa);
-  MILORA_CUDA(ctx, cudaGetLastError());
-  prefill_expand_kernel<<<(unsigned)grid_e, kExpandThreads, expand_smem, s>>>(ea);
-  MILORA_CUDA(ctx, cudaGetLastError());
+  MILORA_CUDA(ctx, launch_pdl(prefill_shrink_kernel, dim3((unsigned)grid_s), dim3(kShrinkThreads), shrink_smem, s, sa));
+  MILORA_CUDA(ctx, launch_pdl(prefill_expand_kernel, dim3((unsigned)grid_e), dim3(kExpandThreads), expand_smem, s, ea));
   return MILORA_OK;
 }
 

@@ -90,6 +90,8 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   const int layer = a.layer_begin + blockIdx.x;
   int32_t* ws = a.ws + (size_t)blockIdx.x * a.ws_stride;
   const int max_tenants = a.tab.max_tenants;
+  pdl_launch_dependents();
+  pdl_wait();
 
   // ---- 1. composite keys, excluded-token count --------------------------------------------
   int excl = 0;
@@ -287,8 +289,7 @@ milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   }
   // few sequences (a decode batch): a smaller block makes every barrier and scan cheaper
   const int threads = std::max(128, std::min(kGMaxThreads, n_pad));
-  group_kernel<<<n_layers, threads, smem, s>>>(a);
-  MILORA_CUDA(ctx, cudaGetLastError());
+  MILORA_CUDA(ctx, launch_pdl(group_kernel, dim3(n_layers), dim3(threads), smem, s, a));
   return MILORA_OK;
 }
 

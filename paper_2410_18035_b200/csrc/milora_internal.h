@@ -137,6 +137,33 @@ DeviceTables device_tables(const milora_ctx* ctx);
 void module_dims(const milora_model_desc& d, int module, int* d1, int* d2);
 milora_group_layout_t group_layout(int n_seq, int T);
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// Every hot-path kernel is launched with the programmatic-stream-serialization attribute: it may start
+// while the kernel before it on the stream is still draining, sets up its shared memory, barriers and
+// tensor memory, and calls pdl_wait() before its first access to global memory (the wait returns once
+// the preceding grid has completed and its writes are visible).  pdl_launch_dependents() at the top lets
+// the kernel after it do the same.  Every CTA calls pdl_wait() before it can return, so completion of a
+// grid implies completion of everything before it on the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class Args>
+inline cudaError_t launch_pdl(void (*kernel)(Args), dim3 grid, dim3 block, size_t smem, cudaStream_t s, const Args& args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args);
+}
+#endif
+
 // kernels (defined in their own .cu files)
 milora_status launch_repack_adapter(milora_ctx* ctx, const void* A, const void* B, void* At, void* Bout, int d1, int d2,
                                     int rank, cudaStream_t s);

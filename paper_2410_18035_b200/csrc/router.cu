@@ -181,6 +181,8 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = a.d;
   const T* H = static_cast<const T*>(a.H);
+  pdl_launch_dependents();
+  pdl_wait();
 
   // per-CTA prefix over prompts: chunks per prompt (from the lengths) and the pooler of each prompt
   if (tid == 0) carry = 0;
@@ -308,6 +310,8 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   __shared__ int32_t wsum[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int p = blockIdx.x, d = a.d;
+  pdl_launch_dependents();
+  pdl_wait();
   // first scratch row of this prompt = number of chunks of the prompts before it
   int mine = 0;
   for (int q = tid; q < p; q += kThreads) {
@@ -487,13 +491,11 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   if (per_sm < 1) per_sm = 1;
   int grid = (int)std::min<size_t>((pl.max_units + kWarps - 1) / kWarps, (size_t)ctx->sm_count * per_sm);
   if (grid < 1) grid = 1;
-  if (f32) pool_partial_kernel<float><<<grid, kThreads, smem, s>>>(a);
-  else pool_partial_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a);
-  MILORA_CUDA(ctx, cudaGetLastError());
+  if (f32) MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<float>, dim3(grid), dim3(kThreads), smem, s, a));
+  else MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), smem, s, a));
   // pass 2: one CTA per prompt
-  if (f32) route_finalize_kernel<float><<<P, kThreads, 0, s>>>(a);
-  else route_finalize_kernel<__nv_bfloat16><<<P, kThreads, 0, s>>>(a);
-  MILORA_CUDA(ctx, cudaGetLastError());
+  if (f32) MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<float>, dim3(P), dim3(kThreads), 0, s, a));
+  else MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<__nv_bfloat16>, dim3(P), dim3(kThreads), 0, s, a));
   return MILORA_OK;
 }
 
