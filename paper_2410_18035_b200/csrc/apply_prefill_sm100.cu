@@ -37,6 +37,7 @@ constexpr int kXStage = kTileRows * kBK * 2;    // 16 KiB
 constexpr int kYStage = kTileRows * kBN * 2;    // 32 KiB (two 64-column TMA boxes)
 constexpr int kShrinkThreads = 128;
 constexpr int kExpandThreads = 192;             // warp 0 copies, warp 1 issues MMAs, warps 2..5 epilogue
+constexpr int kIdentBytes = 16 * 16 * 2;        // expand: identity block that carries y into the accumulator
 
 struct PrefillSites {
   int module[kMaxSites], d1[kMaxSites], d2[kMaxSites];
@@ -92,8 +93,10 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kKSplit, ks = blockIdx.x % kKSplit;
-  pdl_launch_dependents();
+  // The expand kernel starts its copies of y and B before its own wait; it may do so only once
+  // everything ahead of this kernel has completed, so the trigger comes after the wait here.
   pdl_wait();
+  pdl_launch_dependents();
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
   if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
@@ -200,46 +203,48 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
 // ------------------------------------------------------------------------------------------------------
 // expand
 // ------------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void add8(uint4& y, const uint32_t* d) {
-  uint32_t w[4] = {y.x, y.y, y.z, y.w};
+// Eight fp32 accumulator values (y + delta) rounded to bf16.
+__device__ __forceinline__ uint4 pack8(const uint32_t* d) {
+  uint32_t w[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    float lo = __uint_as_float(w[i] << 16) + __uint_as_float(d[2 * i]);
-    float hi = __uint_as_float(w[i] & 0xFFFF0000u) + __uint_as_float(d[2 * i + 1]);
-    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]));
     w[i] = *reinterpret_cast<uint32_t*>(&h);
   }
-  y = make_uint4(w[0], w[1], w[2], w[3]);
+  return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __grid_constant__ ExpandArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile_idx = blockIdx.x / kNSplit, ns = blockIdx.x % kNSplit;
+  // Launched behind the shrink kernel, whose CTAs trigger only after their own wait: the job list, y and
+  // the B images are final when this CTA starts.  Only the partial products of the shrink need pdl_wait().
   pdl_launch_dependents();
-  pdl_wait();
   const int n_tiles = a.ws[a.lay.header + H_NTILES];
-  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
+  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) { pdl_wait(); return; }
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
   const int si = find_site(a.sites, job.module);
-  if (si < 0) return;
+  if (si < 0) { pdl_wait(); return; }
   const int rp = job.rank_pad;
   const uint32_t base = smem_u32(smem_raw);
   if (!job.B_img || rp < 16 || rp > a.rpad || (rp & 15) || (base & 1023) || job.count < 1 || job.count > kTileRows ||
       job.start < 0 || job.start + job.count > a.T) {
     if (tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    pdl_wait();
     return;
   }
   const int d2 = a.sites.d2[si];
   const int nchunks = d2 / kBN, cps = (nchunks + kNSplit - 1) / kNSplit;
   const int nc0 = ns * cps, nc1 = min(nchunks, nc0 + cps), nn = nc1 - nc0;
-  if (nn <= 0) return;
+  if (nn <= 0) { pdl_wait(); return; }
 
   const uint32_t ys = base;
   const uint32_t bs = ys + kExpandStages * kYStage;
   const uint32_t b_stage = (uint32_t)a.rpad * 256u;
   const uint32_t vs = bs + kExpandStages * b_stage;
-  const uint32_t bars = vs + (uint32_t)kTileRows * a.rpad * 2u;
+  const uint32_t ident = vs + (uint32_t)kTileRows * a.rpad * 2u;     // 16 x 16 identity, 512 bytes
+  const uint32_t bars = ident + kIdentBytes;
   auto full = [&](int i) { return bars + 8u * i; };
   auto empty = [&](int i) { return bars + 8u * (kExpandStages + i); };
   auto tfull = [&](int i) { return bars + 8u * (2 * kExpandStages + i); };
@@ -257,12 +262,27 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
     prefetch_tensormap(&a.ymap[si]);
   }
   __syncthreads();
-  if (warp == 0) { tmem_alloc(slot, kCols); tmem_relinquish(); }
+  const int row0 = job.start;
+  auto issue_stage = [&](int i) {       // y tile (two 64-column boxes) and B image chunk of n chunk i
+    const int s = i % kExpandStages;
+    mbar_expect_tx(full(s), kYStage + rp * 256);
+    tma_load_2d(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s));
+    tma_load_2d(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s));
+    bulk_g2s(bs + s * b_stage, static_cast<const char*>(job.B_img) + (size_t)(nc0 + i) * rp * 256, rp * 256, full(s));
+  };
+  if (warp == 0) {
+    tmem_alloc(slot, kCols);
+    tmem_relinquish();
+    // first pass over the ring: these copies do not depend on the shrink kernel
+    if (lane == 0)
+      for (int i = 0; i < nn && i < kExpandStages; ++i) issue_stage(i);
+  }
 
   // epilogue threads also build the A operand: V = s * sum_k V_k, bf16, 8 x 16-byte core-matrix rows
   const int q = warp & 3;               // tensor-memory lane quarter this warp may read
   const int m = q * 32 + lane;          // row of the tile this thread owns
   if (warp >= 2) {
+    pdl_wait();                         // the partial products written by the shrink kernel
     unsigned char* vrow = smem_raw + (vs - base) + (size_t)(m >> 3) * 128 + (size_t)(m & 7) * 16;
     for (int c0 = 0; c0 < rp; c0 += 8) {
       float acc[8];
@@ -286,30 +306,33 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
       }
       *reinterpret_cast<uint4*>(vrow + (size_t)(c0 >> 3) * (kTileRows / 8) * 128) = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    // I_16 as a K-major operand without swizzle: core matrix (n / 8, k / 8) at ((k / 8) * 2 + n / 8) * 128 bytes
+    for (int idx = tid - 64; idx < 256; idx += 128) {
+      const int n = idx >> 4, k = idx & 15;
+      const uint32_t off = (uint32_t)(((k >> 3) * 2 + (n >> 3)) * 128 + (n & 7) * 16 + (k & 7) * 2);
+      *reinterpret_cast<unsigned short*>(smem_raw + (ident - base) + off) = (n == k) ? 0x3F80 : 0;   // bf16 1.0
+    }
     fence_proxy_async_smem();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *slot_ptr;
-  const int row0 = job.start;
   const bool full_tile = job.count == kTileRows;
 
   if (warp == 0) {
     if (lane == 0) {
-      const char* img = static_cast<const char*>(job.B_img);
-      for (int i = 0; i < nn; ++i) {
+      for (int i = kExpandStages; i < nn; ++i) {
         const int s = i % kExpandStages, ph = (i / kExpandStages) & 1;
-        if (i >= kExpandStages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
-        mbar_expect_tx(full(s), kYStage + rp * 256);
-        tma_load_2d(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s));
-        tma_load_2d(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s));
-        bulk_g2s(bs + s * b_stage, img + (size_t)(nc0 + i) * rp * 256, rp * 256, full(s));
+        if (!wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
+        issue_stage(i);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(kTileRows, kBN);
+      const uint32_t idesc_i = idesc_bf16_f32(kTileRows, 16);
+      const uint64_t di = smem_desc(ident, 256, 128, 0);
       constexpr uint32_t kLbo = (kTileRows / 8) * 128u;      // both operands: 16 core matrices per k group
       for (int i = 0; i < nn; ++i) {
         const int s = i % kExpandStages, ph = (i / kExpandStages) & 1, b = i & 1, bph = (i >> 1) & 1;
@@ -320,6 +343,13 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
           const uint64_t da = smem_desc(vs + kk * 2 * kLbo, kLbo, 128, 0);
           const uint64_t db = smem_desc(bs + s * b_stage + kk * 2 * kLbo, kLbo, 128, 0);
           mma_bf16_ss(tmem_base + b * kBN, da, db, idesc, kk != 0);
+        }
+        // y itself joins the accumulator: D[:, 16g .. 16g+16) += Y[:, 16g .. 16g+16) . I_16 (exact in fp32),
+        // so the epilogue only converts and stores.  The y tile is the 128-byte-swizzled K-major A operand.
+#pragma unroll
+        for (int g = 0; g < kBN / 16; ++g) {
+          const uint64_t da = smem_desc(ys + s * kYStage + (g >> 2) * (kYStage / 2) + (g & 3) * 32, 16, 1024, 2);
+          mma_bf16_ss(tmem_base + b * kBN + g * 16, da, di, idesc_i, 1);
         }
         mma_commit(tfull(b));
       }
@@ -346,19 +376,11 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
         if (m < job.count) {
           unsigned char* yrow = ytile + (size_t)box * (kYStage / 2) + (size_t)m * 128;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint4* p = reinterpret_cast<uint4*>(yrow + ((c ^ (m & 7)) << 4));
-            uint4 y = *p;
-            add8(y, d0 + 8 * c);
-            *p = y;
-          }
+          for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint4*>(yrow + ((c ^ (m & 7)) << 4)) = pack8(d0 + 8 * c);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint4* p = reinterpret_cast<uint4*>(yrow + (((c + 4) ^ (m & 7)) << 4));
-            uint4 y = *p;
-            add8(y, d1v + 8 * c);
-            *p = y;
-          }
+          for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint4*>(yrow + (((c + 4) ^ (m & 7)) << 4)) = pack8(d1v + 8 * c);
         }
       }
       tc_fence_before();
@@ -388,6 +410,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
     if (e == 0) bulk_wait_group0();
   }
   __syncwarp();
+  pdl_wait();                           // returns at once here; keeps "every thread waited before it exits" true
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kCols);
@@ -495,7 +518,8 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
     if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (reinterpret_cast<uintptr_t>(st.Y) & 15)) return MILORA_E_SHAPE;
   }
   const size_t shrink_smem = (size_t)kShrinkStages * (kXStage + rpad * 128) + 128;
-  const size_t expand_smem = (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + 128;
+  const size_t expand_smem =
+      (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + kIdentBytes + 128;
   if (shrink_smem > 220 * 1024 || expand_smem > 220 * 1024) return MILORA_E_SHAPE;
 
   const size_t need = (size_t)kKSplit * T * rpad;
