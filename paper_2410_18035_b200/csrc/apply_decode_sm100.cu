@@ -123,9 +123,17 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   const int job_idx = blockIdx.x / kC;
   pdl_launch_dependents();
   pdl_wait();
+  if (job_idx >= a.lay.max_gather) return;                              // same decision in the whole cluster
+  // the job record is fetched together with the job count (the list has max_gather slots, so the read is in bounds)
+  const uint4* jp = reinterpret_cast<const uint4*>(a.ws + a.lay.gather) + (size_t)job_idx * 4;
+  const uint4 j0 = jp[0], j1 = jp[1], j2 = jp[2], j3 = jp[3];
   const int n_jobs = a.ws[a.lay.header + H_NGATHER];
-  if (job_idx >= n_jobs || job_idx >= a.lay.max_gather) return;          // same decision in the whole cluster
-  const GatherJob job = reinterpret_cast<const GatherJob*>(a.ws + a.lay.gather)[job_idx];
+  if (job_idx >= n_jobs) return;
+  GatherJob job;
+  {
+    uint4* dst = reinterpret_cast<uint4*>(&job);
+    dst[0] = j0; dst[1] = j1; dst[2] = j2; dst[3] = j3;
+  }
   int si = -1;
 #pragma unroll
   for (int i = 0; i < kMaxSites; ++i)

@@ -99,13 +99,13 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
     int c = INT_MAX;
     if (i < n_seq) {
       int lo = i, hi = i + 1;
+      const int slot = a.seq_slot[i];          // fetched together with the row range
       if (a.cu) { lo = a.cu[i]; hi = a.cu[i + 1]; }
       bool rows_ok = lo >= 0 && hi >= lo && hi <= a.T;
       if (!rows_ok) atomicOr(a.tab.err, ERR_BAD_ROW);
       int len = rows_ok ? hi - lo : 0;
       seq_lo[i] = lo;
       seq_len[i] = len;
-      int slot = a.seq_slot[i];
       bool ok = slot >= 0 && slot < a.tab.max_requests;
       if (!ok) atomicOr(a.tab.err, ERR_BAD_SLOT);
       int key = -1;
@@ -129,7 +129,23 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
     n_excl = t1[0];
   }
 
-  // ---- 2. bitonic sort of the composite keys ----------------------------------------------
+  // ---- 2. sort of the composite keys ---------------------------------------------------------
+  if (n_pad <= 256 && n_pad <= kGThreads) {
+    // at most one key per thread (a decode batch, a few prompts): rank by counting, three barriers
+    // in place of a sorting network.  Valid keys are unique; the padding is ordered by position.
+    __syncthreads();
+    const int c = tid < n_pad ? comp[tid] : INT_MAX;
+    int rank = 0;
+    if (tid < n_pad) {
+#pragma unroll 8
+      for (int j = 0; j < n_pad; ++j) {
+        const int o = comp[j];
+        rank += (o < c || (o == c && j < tid)) ? 1 : 0;
+      }
+    }
+    __syncthreads();
+    if (tid < n_pad) comp[rank] = c;
+  } else
   for (int k = 2; k <= n_pad; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
       __syncthreads();
