@@ -69,6 +69,10 @@ enum { MILORA_Q = 0, MILORA_K = 1, MILORA_V = 2, MILORA_O = 3, MILORA_GATE = 4, 
 
 enum { MILORA_MAX_RATIONAL_COEF = 16 };
 
+/* How a selected module's LoRA term is weighted (Eq. 3 selects; the paper prints no weighting, so NONE is the
+ * default reading).  PROB multiplies the term of the j-th selected module by its softmax probability. */
+typedef enum { MILORA_GATE_NONE = 0, MILORA_GATE_PROB = 1 } milora_gate;
+
 typedef struct {
   int n_layers;
   int d_model;      /* hidden size d; d_model, d_ff and d_kv must be multiples   */
@@ -78,11 +82,13 @@ typedef struct {
   int max_rank;     /* largest LoRA rank that will be registered (1..256)       */
   int max_tenants;
   int max_requests; /* number of request slots (rows of the route table)        */
+  int top_k;        /* k of Eq. 3 (Top-k): modules selected per request and layer, 1..7; 0 means 1 */
+  int gate;         /* milora_gate                                               */
 } milora_model_desc;
 
 /* Create / destroy.  milora_create allocates the device tables (adapter table, router table,
- * slot table, route table [max_requests][n_layers] initialised to -1) with cudaMalloc on the
- * current device and waits for their initialisation.  milora_destroy frees everything the
+ * slot table, route table [max_requests][n_layers][top_k] initialised to -1, gate table of the same
+ * shape) with cudaMalloc on the current device and waits for their initialisation.  milora_destroy frees everything the
  * library allocated, including adapter copies. */
 milora_status milora_create(const milora_model_desc* desc, milora_ctx** out);
 milora_status milora_destroy(milora_ctx* ctx);
@@ -126,8 +132,9 @@ milora_status milora_request_close(milora_ctx* ctx, int slot);
  * Route P prompts at `layer`.  H_dev holds the prompts' hidden states back to back:
  * rows [cu_seqlens[p], cu_seqlens[p+1]) of a [T_total, d_model] matrix belong to prompt p;
  * T_total = cu_seqlens[P] must be passed by the host.  seq_slot_dev[p] is the request slot of
- * prompt p (P <= 4096).  Writes route[slot][layer] (module id 0..6, ties to the lower index) and,
- * when not NULL, logits_out_dev [P][7] fp32 (g(h) W_r + bias) and probs_out_dev [P][7] fp32 (their
+ * prompt p (P <= 4096).  Writes route[slot][layer][0..top_k) (module ids 0..6 in descending order of
+ * their logits, ties to the lower index; Eq. 3, and the k sweep of Section 4.5), the matching softmax
+ * probabilities to the gate table and, when not NULL, logits_out_dev [P][7] fp32 (g(h) W_r + bias) and probs_out_dev [P][7] fp32 (their
  * softmax).
  * Prompts whose slot is closed or whose tenant has no router at this layer get route -1.
  * Two launches (streaming partial reduction, then one CTA per prompt); deterministic (fixed reduction
@@ -160,23 +167,30 @@ milora_status milora_route_static(milora_ctx* ctx, int layer, const void* H_dev,
                                   const int32_t* seq_slot_dev, int P, int T_total, float* logits_out_dev,
                                   float* probs_out_dev, void* stream);
 
-/* Device pointer to the route table, int32 [max_requests][n_layers], read-only for callers. */
+/* Device pointer to the route table, int32 [max_requests][n_layers][top_k], read-only for callers. */
 milora_status milora_route_table(const milora_ctx* ctx, const int32_t** table_dev);
 
-/* Copy route rows [slot_begin, slot_begin + n_slots) to / from host memory (n_slots * n_layers int32).
+/* Copy route rows [slot_begin, slot_begin + n_slots) to / from host memory (n_slots * n_layers * top_k int32).
  * Both wait for `stream` first and return when the copy is done.  Writing lets a caller restore
  * decisions that were computed earlier (for example after moving a request to another replica);
- * values must be -1 or 0..6. */
+ * values must be -1 or 0..6, and the modules of one (slot, layer) cell distinct. */
 milora_status milora_route_table_read(milora_ctx* ctx, int slot_begin, int n_slots, int32_t* rows_host, void* stream);
 milora_status milora_route_table_write(milora_ctx* ctx, int slot_begin, int n_slots, const int32_t* rows_host,
                                        void* stream);
+/* The same for the gate table (fp32, same shape as the route table): entry j is the softmax probability of
+ * the j-th selected module, written by milora_route.  Only read by the library when gate = MILORA_GATE_PROB. */
+milora_status milora_gate_table_read(milora_ctx* ctx, int slot_begin, int n_slots, float* rows_host, void* stream);
+milora_status milora_gate_table_write(milora_ctx* ctx, int slot_begin, int n_slots, const float* rows_host,
+                                      void* stream);
 
 /* ---- grouping (multi-tenant batches, Section 4.5) ------------------------------------------
  * A step's tokens are n_seq sequences laid out back to back (rows [cu_seqlens[i], cu_seqlens[i+1])
  * of every X / Y matrix; n_seq <= 4096); a decode request is a sequence of length 1 (cu_seqlens_dev
  * == NULL means every sequence has length 1).  For layers [layer_begin, layer_begin + n_layers) the tokens are
- * bucketed by key = route[slot][layer] * max_tenants + tenant(slot).  Sequences whose slot is
- * closed, not routed, or whose tenant has no adapter on the routed module are excluded.
+ * bucketed by key = route[slot][layer][j] * max_tenants + tenant(slot); with top_k > 1 a token belongs to
+ * one bucket per selected module (n_seq * top_k <= 4096).  A sequence whose slot is closed or not routed, or
+ * whose tenant has no adapter on any of its selected modules, is excluded (n_excluded counts its tokens);
+ * n_active counts (token, module) pairs.
  *
  * Output: one int32 block per layer in ws_dev (block l at ws_dev + l * ws_stride), laid out as
  * milora_group_layout describes:

@@ -260,46 +260,55 @@ def group_tokens(token_slot, slot_tenant, route_col, has_adapter, max_tenants: i
 
     token_slot  (T,) request slot of every token
     slot_tenant (R,) tenant of each slot (-1: slot closed)
-    route_col   (R,) routed module of each slot at this layer (-1: not routed)
+    route_col   (R,) routed module of each slot at this layer (-1: not routed), or (R, k) for
+                Top-k routing (Eq. 3; the k sweep of Section 4.5): the k selected modules
     has_adapter callable (tenant, module) -> bool
-    Tokens whose slot is closed, unrouted or without an adapter are excluded.
+    A token belongs to one bucket per selected module on which its tenant has an adapter.
+    Tokens whose slot is closed, unrouted or without any such adapter are excluded.
 
     Returns dict:
-      perm        (T_active,) token indices ordered by (module, tenant, token index)
+      perm        (n_active,) token indices of the (token, module) pairs ordered by
+                  (module, tenant, token index); a token appears once per selected module
       seg_key     (S,) module * max_tenants + tenant of every non-empty bucket, ascending
       seg_offset  (S+1,) bucket boundaries in perm
       mod_offset  (N_mod+1,) bucket-index boundaries per module
       n_excluded  number of excluded tokens
     """
     T = len(token_slot)
-    keys = np.full(T, -1, dtype=np.int64)
+    route_sel = np.asarray(route_col)
+    if route_sel.ndim == 1:
+        route_sel = route_sel[:, None]
+    pairs = []                                   # (key, token) in token order
+    n_excluded = 0
     for t in range(T):
         slot = int(token_slot[t])
         tenant = int(slot_tenant[slot])
-        module = int(route_col[slot])
-        if tenant < 0 or module < 0:
-            continue
-        if not has_adapter(tenant, module):
-            continue
-        keys[t] = module * max_tenants + tenant
-    active = [t for t in range(T) if keys[t] >= 0]
-    active.sort(key=lambda t: keys[t])          # Python's sort is stable
-    perm = np.array(active, dtype=np.int32)
+        found = False
+        if tenant >= 0:
+            for module in (int(v) for v in route_sel[slot]):
+                if module < 0 or not has_adapter(tenant, module):
+                    continue
+                pairs.append((module * max_tenants + tenant, t))
+                found = True
+        if not found:
+            n_excluded += 1
+    pairs.sort(key=lambda kt: kt[0])             # Python's sort is stable
+    perm = np.array([t for _, t in pairs], dtype=np.int32)
     seg_key, seg_offset = [], [0]
-    for i, t in enumerate(active):
-        if i == 0 or keys[t] != keys[active[i - 1]]:
+    for i, (key, _) in enumerate(pairs):
+        if i == 0 or key != pairs[i - 1][0]:
             if i > 0:
                 seg_offset.append(i)
-            seg_key.append(int(keys[t]))
-    if active:
-        seg_offset.append(len(active))
+            seg_key.append(int(key))
+    if pairs:
+        seg_offset.append(len(pairs))
     seg_key = np.array(seg_key, dtype=np.int32)
     seg_offset = np.array(seg_offset, dtype=np.int32)
     mod_offset = np.zeros(N_MOD + 1, dtype=np.int32)
     for m in range(N_MOD):
         mod_offset[m + 1] = mod_offset[m] + int(np.sum(seg_key // max_tenants == m))
     return {"perm": perm, "seg_key": seg_key, "seg_offset": seg_offset,
-            "mod_offset": mod_offset, "n_excluded": T - len(active)}
+            "mod_offset": mod_offset, "n_excluded": n_excluded}
 
 
 # --------------------------------------------------------------------------
@@ -331,7 +340,18 @@ def merged_weight(W, A, B, s: float):
     return _f64(W) + float(s) * (_f64(A) @ _f64(B))
 
 
-def apply_module(y_base, x, token_slot, slot_tenant, route_sel, module: int, adapters):
+def _selection_weight(route_sel, gate, slot: int, module: int):
+    """None if `module` is not among the slot's selected modules, else the weight of its LoRA term:
+    1 (hard selection) or gate[slot][j] for the position j at which it was selected."""
+    sel = [int(v) for v in route_sel[slot]]
+    if module not in sel:
+        return None
+    if gate is None:
+        return 1.0
+    return float(np.asarray(gate, dtype=np.float64).reshape(len(route_sel), -1)[slot][sel.index(module)])
+
+
+def apply_module(y_base, x, token_slot, slot_tenant, route_sel, module: int, adapters, gate=None):
     """Outputs of module `module` for a mixed batch.
 
     y_base     (T, d2) the backbone's x W_m + b_m (an input here)
@@ -339,6 +359,9 @@ def apply_module(y_base, x, token_slot, slot_tenant, route_sel, module: int, ada
     route_sel  (R,) int, or (R, k) int for top-k routing: the module(s) selected
                for each slot at this layer
     adapters   callable (tenant, module) -> (A, B, s) or None
+    gate       optional (R,) / (R, k) weights, gate[slot][j] for the j-th selected module
+               (the paper only selects, so None = weight 1 is the default reading; a
+               probability-weighted mixture passes the router's softmax values here)
     A token receives s (x A) B iff its slot's selection contains `module` and the
     tenant has an adapter there; every other row is returned unchanged.
     """
@@ -350,17 +373,18 @@ def apply_module(y_base, x, token_slot, slot_tenant, route_sel, module: int, ada
     for t in range(y.shape[0]):
         slot = int(token_slot[t])
         tenant = int(slot_tenant[slot])
-        if tenant < 0 or module not in [int(v) for v in route_sel[slot]]:
+        wgt = None if tenant < 0 else _selection_weight(route_sel, gate, slot, module)
+        if wgt is None:
             continue
         ad = adapters(tenant, module)
         if ad is None:
             continue
         A, B, s = ad
-        y[t] = y[t] + lora_delta(x[t:t + 1], A, B, s)[0]
+        y[t] = y[t] + wgt * lora_delta(x[t:t + 1], A, B, s)[0]
     return y
 
 
-def apply_module_sampled(y_base_rows, x_rows, rows, token_slot, slot_tenant, route_sel, module, adapters):
+def apply_module_sampled(y_base_rows, x_rows, rows, token_slot, slot_tenant, route_sel, module, adapters, gate=None):
     """Same as apply_module, restricted to the token indices `rows` (for full-size
     workloads where only sampled outputs are checked).  y_base_rows / x_rows hold
     just those rows, in the order of `rows`."""
@@ -372,13 +396,14 @@ def apply_module_sampled(y_base_rows, x_rows, rows, token_slot, slot_tenant, rou
     for i, t in enumerate(rows):
         slot = int(token_slot[int(t)])
         tenant = int(slot_tenant[slot])
-        if tenant < 0 or module not in [int(v) for v in route_sel[slot]]:
+        wgt = None if tenant < 0 else _selection_weight(route_sel, gate, slot, module)
+        if wgt is None:
             continue
         ad = adapters(tenant, module)
         if ad is None:
             continue
         A, B, s = ad
-        y[i] = y[i] + lora_delta(x[i:i + 1], A, B, s)[0]
+        y[i] = y[i] + wgt * lora_delta(x[i:i + 1], A, B, s)[0]
     return y
 
 

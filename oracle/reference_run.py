@@ -74,13 +74,14 @@ def adapters_of(w, layer: int):
     return get
 
 
-def apply_site(w, layer: int, module: int, x, y_base, token_slot, route_sel, rows=None):
+def apply_site(w, layer: int, module: int, x, y_base, token_slot, route_sel, rows=None, gate=None):
     """Oracle output of one module call site.  With `rows`, x / y_base hold only those rows."""
     slot_tenant = w.request_tenant
     ad = adapters_of(w, layer)
     if rows is None:
-        return O.apply_module(to_f64(y_base), to_f64(x), token_slot, slot_tenant, route_sel, module, ad)
-    return O.apply_module_sampled(to_f64(y_base), to_f64(x), rows, token_slot, slot_tenant, route_sel, module, ad)
+        return O.apply_module(to_f64(y_base), to_f64(x), token_slot, slot_tenant, route_sel, module, ad, gate=gate)
+    return O.apply_module_sampled(to_f64(y_base), to_f64(x), rows, token_slot, slot_tenant, route_sel, module, ad,
+                                  gate=gate)
 
 
 def group_layer(w, token_slot, route_col, max_tenants=None):

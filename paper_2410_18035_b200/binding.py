@@ -16,6 +16,7 @@ POOL_MEAN, POOL_LAST, POOL_MAX, POOL_SELFATTN = 0, 1, 2, 3
 ACT_TANH, ACT_IDENTITY, ACT_RELU, ACT_GELU, ACT_RATIONAL = 0, 1, 2, 3, 4
 MODULES = ("q", "k", "v", "o", "gate", "up", "down")
 N_MOD = 7
+GATE_NONE, GATE_PROB = 0, 1
 
 STATUS_NAMES = {0: "MILORA_OK", 1: "MILORA_E_ARG", 2: "MILORA_E_SHAPE", 3: "MILORA_E_DTYPE",
                 4: "MILORA_E_UNREGISTERED", 5: "MILORA_E_CAPACITY", 6: "MILORA_E_STATE", 7: "MILORA_E_CUDA",
@@ -30,7 +31,8 @@ class MiloraError(RuntimeError):
 
 class ModelDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int), ("d_model", C.c_int), ("d_ff", C.c_int), ("d_kv", C.c_int),
-                ("dtype", C.c_int), ("max_rank", C.c_int), ("max_tenants", C.c_int), ("max_requests", C.c_int)]
+                ("dtype", C.c_int), ("max_rank", C.c_int), ("max_tenants", C.c_int), ("max_requests", C.c_int),
+                ("top_k", C.c_int), ("gate", C.c_int)]
 
 
 class GroupLayout(C.Structure):
@@ -68,6 +70,8 @@ SIGNATURES = {
     "milora_route_table": (_I, [_VP, C.POINTER(_VP)]),
     "milora_route_table_read": (_I, [_VP, _I, _I, _VP, _VP]),
     "milora_route_table_write": (_I, [_VP, _I, _I, _VP, _VP]),
+    "milora_gate_table_read": (_I, [_VP, _I, _I, _VP, _VP]),
+    "milora_gate_table_write": (_I, [_VP, _I, _I, _VP, _VP]),
     "milora_group_layout": (_I, [_VP, _I, _I, C.POINTER(GroupLayout)]),
     "milora_group": (_I, [_VP, _I, _I, _VP, _VP, _I, _I, _VP, C.c_size_t, _VP]),
     "milora_apply_decode": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
@@ -111,14 +115,15 @@ def _stream(stream) -> int:
 class Milora:
     """One library context (see include/milora.h for the meaning of every call)."""
 
-    def __init__(self, n_layers, d_model, d_ff, d_kv, dtype, max_rank, max_tenants, max_requests):
+    def __init__(self, n_layers, d_model, d_ff, d_kv, dtype, max_rank, max_tenants, max_requests, top_k=1, gate=GATE_NONE):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("the MiLoRA library needs a CUDA device; there is no CPU path")
         self.torch_dtype = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype] if isinstance(dtype, str) else dtype
         code = F32 if self.torch_dtype == torch.float32 else BF16
-        self.desc = ModelDesc(n_layers, d_model, d_ff, d_kv, code, max_rank, max_tenants, max_requests)
+        self.desc = ModelDesc(n_layers, d_model, d_ff, d_kv, code, max_rank, max_tenants, max_requests, top_k, gate)
         self.n_layers, self.max_requests, self.max_tenants = n_layers, max_requests, max_tenants
+        self.top_k = max(1, top_k)
         h = C.c_void_p()
         self._check(self.lib.milora_create(C.byref(self.desc), C.byref(h)), "milora_create", ctx=None)
         self.h = h
@@ -231,17 +236,33 @@ class Milora:
         return p.value
 
     def route_table_read(self, slot_begin=0, n_slots=None, stream=None):
+        """[n_slots, n_layers] for top_k = 1, else [n_slots, n_layers, top_k]."""
         n_slots = self.max_requests - slot_begin if n_slots is None else n_slots
-        out = torch.empty((n_slots, self.n_layers), dtype=torch.int32)
+        out = torch.empty((n_slots, self.n_layers, self.top_k), dtype=torch.int32)
         self._check(self.lib.milora_route_table_read(self.h, slot_begin, n_slots, out.data_ptr(), _stream(stream)),
                     "milora_route_table_read")
+        return out[:, :, 0] if self.top_k == 1 else out
+
+    def gate_table_read(self, slot_begin=0, n_slots=None, stream=None):
+        n_slots = self.max_requests - slot_begin if n_slots is None else n_slots
+        out = torch.empty((n_slots, self.n_layers, self.top_k), dtype=torch.float32)
+        self._check(self.lib.milora_gate_table_read(self.h, slot_begin, n_slots, out.data_ptr(), _stream(stream)),
+                    "milora_gate_table_read")
         return out
+
+    def gate_table_write(self, slot_begin, rows, stream=None):
+        rows = torch.as_tensor(rows, dtype=torch.float32).contiguous().cpu()
+        n_slots = rows.shape[0]
+        if rows.numel() != n_slots * self.n_layers * self.top_k:
+            raise ValueError("gate_table_write: rows must be [n_slots, n_layers, top_k]")
+        self._check(self.lib.milora_gate_table_write(self.h, slot_begin, n_slots, rows.data_ptr(), _stream(stream)),
+                    "milora_gate_table_write")
 
     def route_table_write(self, slot_begin, rows, stream=None):
         rows = torch.as_tensor(rows, dtype=torch.int32).contiguous().cpu()
         n_slots = rows.shape[0]
-        if rows.numel() != n_slots * self.n_layers:
-            raise ValueError("route_table_write: rows must be [n_slots, n_layers]")
+        if rows.numel() != n_slots * self.n_layers * self.top_k:
+            raise ValueError("route_table_write: rows must be [n_slots, n_layers] (or [n_slots, n_layers, top_k])")
         self._check(self.lib.milora_route_table_write(self.h, slot_begin, n_slots, rows.data_ptr(), _stream(stream)),
                     "milora_route_table_write")
 

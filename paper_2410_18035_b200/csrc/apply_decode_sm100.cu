@@ -262,7 +262,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
     float s = 0.f;
 #pragma unroll
     for (int c = 0; c < kC; ++c) s += part[((size_t)c * kR + t) * a.rmax + j];
-    v_sm[t * a.rmax + j] = s * job.scale;
+    v_sm[t * a.rmax + j] = s * job.scale * job.gate[t];
   }
   __syncthreads();
 
@@ -309,7 +309,7 @@ milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySi
   a.err = ctx->d_err;
   a.sites = sites;
   a.ws = g->ws_dev;
-  a.lay = group_layout(g->n_seq, g->T);
+  a.lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
   a.T = g->T;
   a.rmax = (ctx->desc.max_rank + 3) & ~3;
   int per2 = 0;

@@ -73,19 +73,25 @@ __global__ void __launch_bounds__(kThreads) apply_generic_kernel(ApplyArgs a) {
 
   const void *At_v, *B_v;
   int r, module, n_rows, rows[R];
-  float scale;
+  float scale, gate[R];
   if (DENSE) {
     const TileJob w = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[job_idx];
     At_v = w.At; B_v = w.B; r = w.rank; scale = w.scale; module = w.module;
     n_rows = min(R, w.count - sub * R);
 #pragma unroll
-    for (int t = 0; t < R; ++t) rows[t] = (t < n_rows) ? w.start + sub * R + t : -1;
+    for (int t = 0; t < R; ++t) {
+      rows[t] = (t < n_rows) ? w.start + sub * R + t : -1;
+      gate[t] = 1.f;                      // a tile's weight is already folded into its scale
+    }
   } else {
     const GatherJob w = reinterpret_cast<const GatherJob*>(a.ws + a.lay.gather)[job_idx];
     At_v = w.At; B_v = w.B; r = w.rank; scale = w.scale; module = w.module;
     n_rows = min(R, w.count);
 #pragma unroll
-    for (int t = 0; t < R; ++t) rows[t] = (t < n_rows) ? w.rows[t] : -1;
+    for (int t = 0; t < R; ++t) {
+      rows[t] = (t < n_rows) ? w.rows[t] : -1;
+      gate[t] = (t < kGatherRows) ? w.gate[t < kGatherRows ? t : 0] : 0.f;
+    }
   }
   if (n_rows <= 0) return;
   int si = -1;
@@ -137,7 +143,7 @@ __global__ void __launch_bounds__(kThreads) apply_generic_kernel(ApplyArgs a) {
     }
     if (lane == 0) {
 #pragma unroll
-      for (int t = 0; t < R; ++t) v_sm[t][j] = acc[t] * scale;
+      for (int t = 0; t < R; ++t) v_sm[t][j] = acc[t] * scale * gate[t];
     }
   }
   __syncthreads();
@@ -182,7 +188,7 @@ milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites&
   a.err = ctx->d_err;
   a.sites = sites;
   a.ws = g->ws_dev;
-  a.lay = group_layout(g->n_seq, g->T);
+  a.lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
   a.T = g->T;
   // one CTA per (job, sub-block) of the largest list this batch can have; the exact count is on the device
   size_t grid = dense ? (size_t)a.lay.max_tiles * (kTileRows / kDenseRows) : (size_t)a.lay.max_gather;

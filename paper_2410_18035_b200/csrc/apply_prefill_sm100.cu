@@ -51,7 +51,7 @@ struct ShrinkArgs {
   int32_t* err;
   const int32_t* ws;
   milora_group_layout_t lay;
-  float* vscratch;     // [kKSplit][T][rpad]
+  float* vscratch;     // [kKSplit][max_tiles * 128][rpad]: indexed by tile, since with top-k routing a row sits in several tiles
   int T, rpad;
 };
 
@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
   const int m = warp * 32 + lane;
-  float* dst = a.vscratch + ((size_t)ks * a.T + job.start + m) * a.rpad;
+  float* dst = a.vscratch + (((size_t)ks * a.lay.max_tiles + tile_idx) * kTileRows + m) * a.rpad;
   for (int c0 = 0; c0 < rp; c0 += 16) {
     uint32_t v[16];
     if (nk > 0 && ok) {
@@ -292,7 +292,8 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
 #pragma unroll
         for (int k = 0; k < kKSplit; ++k) {
           const float4* src =
-              reinterpret_cast<const float4*>(a.vscratch + ((size_t)k * a.T + job.start + m) * a.rpad + c0);
+              reinterpret_cast<const float4*>(
+                  a.vscratch + (((size_t)k * a.lay.max_tiles + tile_idx) * kTileRows + m) * a.rpad + c0);
           const float4 u0 = __ldcg(src), u1 = __ldcg(src + 1);
           acc[0] += u0.x; acc[1] += u0.y; acc[2] += u0.z; acc[3] += u0.w;
           acc[4] += u1.x; acc[5] += u1.y; acc[6] += u1.z; acc[7] += u1.w;
@@ -522,7 +523,8 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
       (size_t)kExpandStages * (kYStage + rpad * 256) + (size_t)kTileRows * rpad * 2 + kIdentBytes + 128;
   if (shrink_smem > 220 * 1024 || expand_smem > 220 * 1024) return MILORA_E_SHAPE;
 
-  const size_t need = (size_t)kKSplit * T * rpad;
+  const milora_group_layout_t lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
+  const size_t need = (size_t)kKSplit * lay.max_tiles * kTileRows * rpad;
   if (need > ctx->vscratch_floats) {
     MILORA_CUDA(ctx, cudaStreamSynchronize(s));
     if (ctx->d_vscratch) MILORA_CUDA(ctx, cudaFree(ctx->d_vscratch));
@@ -543,7 +545,6 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
     if (!make_map(&sa.xmap[i], st.X, T, st.d1) || !make_map(&ea.ymap[i], st.Y, T, st.d2)) return MILORA_E_SHAPE;
   }
   for (int i = sites.n; i < kMaxSites; ++i) { sa.xmap[i] = sa.xmap[0]; ea.ymap[i] = ea.ymap[0]; }
-  const milora_group_layout_t lay = group_layout(g->n_seq, g->T);
   sa.sites = ps; sa.err = ctx->d_err; sa.ws = g->ws_dev; sa.lay = lay; sa.vscratch = ctx->d_vscratch; sa.T = T; sa.rpad = rpad;
   ea.sites = ps; ea.err = ctx->d_err; ea.ws = g->ws_dev; ea.lay = lay; ea.vscratch = ctx->d_vscratch; ea.T = T; ea.rpad = rpad;
 

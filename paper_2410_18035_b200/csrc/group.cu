@@ -1,12 +1,12 @@
 // Token grouping for multi-tenant batches: bucket a step's tokens by (module, tenant) for one layer
 // and build the work lists of the apply kernels.
 //
-// A step is given as sequences of consecutive rows, and the key of a token depends only on its
-// sequence's request slot, so the sort runs over sequences (at most kMaxSeq), not over tokens:
-// one CTA per layer sorts the composite keys (key << 12 | sequence index), which are unique, with
-// a bitonic network in shared memory; equal keys then sit next to each other in sequence order,
-// which is row order.  Everything after that is prefix sums.  Integer work only; the result is
-// the same as a stable sort of the tokens by key.
+// A step is given as sequences of consecutive rows, and the keys of a token depend only on its
+// sequence's request slot, so the sort runs over (sequence, selected module) entries (at most kMaxSeq;
+// top_k entries per sequence), not over tokens: one CTA per layer sorts the composite keys
+// (key << 12 | entry index), which are unique, in shared memory; equal keys then sit next to each other
+// in sequence order, which is row order.  Everything after that is prefix sums.  Integer work only; the
+// result is the same as a stable sort of the (token, module) pairs by key.
 #include <climits>
 
 #include "milora_internal.h"
@@ -17,7 +17,7 @@ namespace {
 constexpr int kGMaxThreads = 1024;
 constexpr int kSeqBits = 12;  // kMaxSeq = 4096 sequences
 static_assert((1 << kSeqBits) == kMaxSeq, "kSeqBits must match kMaxSeq");
-constexpr int kSmemArrays = 8;
+constexpr int kSmemArrays = 9;
 
 // Exclusive prefix sums over the block of N ints per thread (scanned together: three barriers in all);
 // returns the exclusive values in v, the block totals in total.  wsum holds N x 33 ints.
@@ -69,11 +69,11 @@ struct GroupArgs {
   int32_t* ws;
   size_t ws_stride;
   milora_group_layout_t lay;
-  int layer_begin, n_seq, n_pad, T;
+  int layer_begin, n_seq, n_ent, n_pad, T;
 };
 
-// Shared memory (int32): comp[n_pad], seq_lo[n_pad], seq_len[n_pad], tok_off[n_pad+1], seg_tile[n_pad+1],
-// seg_short[n_pad+1], seg_gather[n_pad+1] (kSmemArrays * n_pad + 8 in total).
+// Shared memory (int32): comp[n_pad], seq_lo[n_pad], seq_len[n_pad], ent_gate[n_pad] (fp32), tok_off[n_pad+1],
+// seg_tile[n_pad+1], seg_short[n_pad+1], seg_gather[n_pad+1] (kSmemArrays * n_pad + 8 in total).
 __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   extern __shared__ int32_t sm[];
   __shared__ int wsum[5 * 33];
@@ -82,7 +82,8 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   int32_t* comp = sm;
   int32_t* seq_lo = comp + n_pad;
   int32_t* seq_len = seq_lo + n_pad;
-  int32_t* tok_off = seq_len + n_pad;
+  float* ent_gate = reinterpret_cast<float*>(seq_len + n_pad);
+  int32_t* tok_off = seq_len + 2 * n_pad;
   int32_t* seg_tile = tok_off + n_pad + 1;
   int32_t* seg_short = seg_tile + n_pad + 1;
   int32_t* seg_gather = seg_short + n_pad + 1;
@@ -90,37 +91,47 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   const int layer = a.layer_begin + blockIdx.x;
   int32_t* ws = a.ws + (size_t)blockIdx.x * a.ws_stride;
   const int max_tenants = a.tab.max_tenants;
+  const int K = a.tab.top_k, n_ent = a.n_ent;
   pdl_launch_dependents();
   pdl_wait();
 
-  // ---- 1. composite keys, excluded-token count --------------------------------------------
+  // ---- 1. composite keys of the (sequence, selected module) entries, excluded-token count ------
+  for (int e = n_ent + tid; e < n_pad; e += kGThreads) comp[e] = INT_MAX;
   int excl = 0;
-  for (int i = tid; i < n_pad; i += kGThreads) {
-    int c = INT_MAX;
-    if (i < n_seq) {
-      int lo = i, hi = i + 1;
-      const int slot = a.seq_slot[i];          // fetched together with the row range
-      if (a.cu) { lo = a.cu[i]; hi = a.cu[i + 1]; }
-      bool rows_ok = lo >= 0 && hi >= lo && hi <= a.T;
-      if (!rows_ok) atomicOr(a.tab.err, ERR_BAD_ROW);
-      int len = rows_ok ? hi - lo : 0;
-      seq_lo[i] = lo;
-      seq_len[i] = len;
-      bool ok = slot >= 0 && slot < a.tab.max_requests;
-      if (!ok) atomicOr(a.tab.err, ERR_BAD_SLOT);
-      int key = -1;
-      if (ok && len > 0) {
-        int tenant = a.tab.slot_tenant[slot];
-        int module = a.tab.route[(size_t)slot * a.tab.n_layers + layer];
-        if (tenant >= 0 && tenant < max_tenants && module >= 0 && module < MILORA_NMOD) {
+  for (int i = tid; i < n_seq; i += kGThreads) {
+    int lo = i, hi = i + 1;
+    const int slot = a.seq_slot[i];          // fetched together with the row range
+    if (a.cu) { lo = a.cu[i]; hi = a.cu[i + 1]; }
+    bool rows_ok = lo >= 0 && hi >= lo && hi <= a.T;
+    if (!rows_ok) atomicOr(a.tab.err, ERR_BAD_ROW);
+    int len = rows_ok ? hi - lo : 0;
+    seq_lo[i] = lo;
+    seq_len[i] = len;
+    bool ok = slot >= 0 && slot < a.tab.max_requests;
+    if (!ok) atomicOr(a.tab.err, ERR_BAD_SLOT);
+    int tenant = -1;
+    if (ok && len > 0) tenant = a.tab.slot_tenant[slot];
+    const bool tenant_ok = tenant >= 0 && tenant < max_tenants;
+    bool any = false;
+    for (int j = 0; j < K; ++j) {
+      int c = INT_MAX;
+      float gt = 1.f;
+      if (tenant_ok) {
+        const size_t cell = ((size_t)slot * a.tab.n_layers + layer) * K + j;
+        const int module = a.tab.route[cell];
+        if (module >= 0 && module < MILORA_NMOD) {
           const AdapterEntry& e = a.tab.adapters[adapter_index(tenant, layer, module, a.tab.n_layers)];
-          if (e.rank > 0) key = module * max_tenants + tenant;
+          if (e.rank > 0) {
+            c = ((module * max_tenants + tenant) << kSeqBits) | (i * K + j);
+            any = true;
+            if (a.tab.gating) gt = a.tab.gate[cell];
+          }
         }
       }
-      if (key >= 0) c = (key << kSeqBits) | i;
-      else excl += len;
+      comp[i * K + j] = c;
+      ent_gate[i * K + j] = gt;
     }
-    comp[i] = c;
+    if (!any) excl += len;
   }
   int n_excl;
   {
@@ -167,7 +178,7 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   for (int j = j0; j < j1; ++j) {
     int c = comp[j];
     if (c == INT_MAX) break;
-    int len = seq_len[c & (kMaxSeq - 1)];
+    int len = seq_len[(c & (kMaxSeq - 1)) / K];
     s_act += 1;
     s_tok += len;
     s_head += (j == 0 || (comp[j - 1] >> kSeqBits) != (c >> kSeqBits)) ? 1 : 0;
@@ -180,14 +191,15 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   const int n_active = t5[0], n_seg = t5[1], n_tiles = t5[2], n_short = t5[3], n_act_seq = t5[4];
 
   TileJob* tiles = reinterpret_cast<TileJob*>(ws + a.lay.tiles);
-  int32_t* gather_rows = ws + a.lay.gather_rows;
+  int32_t* gather_rows = ws + a.lay.gather_rows;       // row, entry index of every gathered (token, module) pair
   int32_t* seg_key = ws + a.lay.seg_key;
   int32_t* seg_offset = ws + a.lay.seg_offset;
   for (int j = j0; j < j1; ++j) {
     int c = comp[j];
     if (c == INT_MAX) break;
     int key = c >> kSeqBits;
-    int lo = seq_lo[c & (kMaxSeq - 1)], len = seq_len[c & (kMaxSeq - 1)];
+    const int ent = c & (kMaxSeq - 1);
+    int lo = seq_lo[ent / K], len = seq_len[ent / K];
     bool head = (j == 0 || (comp[j - 1] >> kSeqBits) != key);
     if (head) {
       seg_key[o_head] = key;
@@ -204,14 +216,18 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
       const AdapterEntry e = a.tab.adapters[adapter_index(key % max_tenants, layer, module, a.tab.n_layers)];
       TileJob w;
       w.At = e.At; w.B = e.B; w.At_img = e.At_img; w.B_img = e.B_img;
-      w.rank = e.rank; w.scale = e.scale; w.module = module; w.seg = seg; w.rank_pad = e.rank_pad; w.pad = 0;
+      w.rank = e.rank; w.scale = e.scale * ent_gate[ent]; w.module = module; w.seg = seg; w.rank_pad = e.rank_pad; w.pad = 0;
       for (int r = 0; r < len; r += kTileRows) {
         w.start = lo + r;
         w.count = min(kTileRows, len - r);
         tiles[o_tile++] = w;
       }
     } else {
-      for (int r = 0; r < len; ++r) gather_rows[o_short++] = lo + r;
+      for (int r = 0; r < len; ++r) {
+        gather_rows[2 * o_short] = lo + r;
+        gather_rows[2 * o_short + 1] = ent;
+        ++o_short;
+      }
     }
   }
   if (tid == 0) {
@@ -226,7 +242,7 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   int32_t* perm = ws + a.lay.perm;
   // one warp per sorted sequence: its rows are consecutive, so the writes are coalesced
   for (int j = tid >> 5; j < n_act_seq; j += kGThreads / 32) {
-    const int i = comp[j] & (kMaxSeq - 1);
+    const int i = (comp[j] & (kMaxSeq - 1)) / K;
     const int lo = seq_lo[i], len = seq_len[i], off = tok_off[j];
     for (int t = tid & 31; t < len; t += 32) perm[off + t] = lo + t;
   }
@@ -252,11 +268,14 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
     const int module = key / max_tenants;
     const AdapterEntry ent = a.tab.adapters[adapter_index(key % max_tenants, layer, module, a.tab.n_layers)];
     GatherJob w;
-    w.At = ent.At; w.B = ent.B; w.rank = ent.rank; w.scale = ent.scale; w.module = module; w.seg = s; w.pad = 0;
+    w.At = ent.At; w.B = ent.B; w.rank = ent.rank; w.scale = ent.scale; w.module = module;
     for (int r = b; r < e; r += kGatherRows) {
       w.count = min(kGatherRows, e - r);
 #pragma unroll
-      for (int t = 0; t < kGatherRows; ++t) w.rows[t] = (t < w.count) ? gather_rows[r + t] : -1;
+      for (int t = 0; t < kGatherRows; ++t) {
+        w.rows[t] = (t < w.count) ? gather_rows[2 * (r + t)] : -1;
+        w.gate[t] = (t < w.count) ? ent_gate[gather_rows[2 * (r + t) + 1]] : 0.f;
+      }
       gather[o_g++] = w;
     }
   }
@@ -294,10 +313,11 @@ milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   GroupArgs a;
   a.tab = device_tables(ctx);
   a.cu = cu; a.seq_slot = seq_slot; a.ws = ws; a.ws_stride = ws_stride;
-  a.lay = group_layout(n_seq, T);
+  a.lay = group_layout(n_seq, T, top_k_of(ctx));
   a.layer_begin = layer_begin; a.n_seq = n_seq; a.T = T;
+  a.n_ent = n_seq * top_k_of(ctx);
   int n_pad = 2;
-  while (n_pad < n_seq) n_pad <<= 1;
+  while (n_pad < a.n_ent) n_pad <<= 1;
   a.n_pad = n_pad;
   size_t smem = ((size_t)n_pad * kSmemArrays + 8) * sizeof(int32_t);
   if (smem > 48 * 1024) {

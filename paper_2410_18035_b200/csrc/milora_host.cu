@@ -52,20 +52,23 @@ void module_dims(const milora_model_desc& d, int module, int* d1, int* d2) {
 
 static size_t round4(size_t v) { return (v + 3) & ~size_t(3); }
 
-milora_group_layout_t group_layout(int n_seq, int T) {
+// Sizes for `top_k` selected modules per sequence: a token may sit in up to top_k buckets.
+milora_group_layout_t group_layout(int n_seq, int T, int top_k) {
   milora_group_layout_t L;
   size_t o = 0;
+  const size_t k = top_k < 1 ? 1 : (size_t)top_k;
+  const size_t n_ent = (size_t)n_seq * k, TT = (size_t)T * k;
   L.header = o; o += kHeaderInts;
   L.mod_offset = o; o += 8;
   L.mod_tile_offset = o; o += 8;
   L.mod_gather_offset = o; o += 8;
-  L.seg_key = o; o += round4((size_t)n_seq);
-  L.seg_offset = o; o += round4((size_t)n_seq + 1);
-  L.perm = o; o += round4((size_t)T);
-  L.max_tiles = T / kTileRows + n_seq;
+  L.seg_key = o; o += round4(n_ent);
+  L.seg_offset = o; o += round4(n_ent + 1);
+  L.perm = o; o += round4(TT);
+  L.max_tiles = (int)(TT / kTileRows + n_ent);
   L.tiles = o; o += (size_t)L.max_tiles * kJobInts;
-  L.gather_rows = o; o += round4((size_t)T);
-  L.max_gather = T / kGatherRows + n_seq + 1;
+  L.gather_rows = o; o += round4(2 * TT);      // row and sequence of every gathered (token, module) pair
+  L.max_gather = (int)(TT / kGatherRows + n_ent + 1);
   L.gather = o; o += (size_t)L.max_gather * kJobInts;
   L.total = round4(o);
   return L;
@@ -77,6 +80,9 @@ DeviceTables device_tables(const milora_ctx* ctx) {
   t.routers = ctx->d_routers;
   t.slot_tenant = ctx->d_slot_tenant;
   t.route = ctx->d_route;
+  t.gate = ctx->d_gate;
+  t.top_k = top_k_of(ctx);
+  t.gating = ctx->desc.gate;
   t.err = ctx->d_err;
   t.n_layers = ctx->desc.n_layers;
   t.max_tenants = ctx->desc.max_tenants;
@@ -151,11 +157,14 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   if (desc->max_rank < 1 || desc->max_rank > 256) return MILORA_E_CAPACITY;
   if (desc->max_tenants < 1 || desc->max_requests < 1) return MILORA_E_CAPACITY;
   if ((long long)desc->max_tenants * MILORA_NMOD > (1ll << 30)) return MILORA_E_CAPACITY;
+  if (desc->top_k < 0 || desc->top_k > MILORA_NMOD) return MILORA_E_ARG;
+  if (desc->gate != MILORA_GATE_NONE && desc->gate != MILORA_GATE_PROB) return MILORA_E_ARG;
   milora_ctx* ctx = new (std::nothrow) milora_ctx();
   if (!ctx) return MILORA_E_CAPACITY;
   ctx->desc = *desc;
   ctx->elem = desc->dtype == MILORA_F32 ? 4 : 2;
   ctx->d_adapters = nullptr; ctx->d_routers = nullptr; ctx->d_slot_tenant = nullptr; ctx->d_route = nullptr;
+  ctx->d_gate = nullptr;
   ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
   ctx->d_vscratch = nullptr; ctx->vscratch_floats = 0;
   ctx->n_counters = 0;
@@ -183,7 +192,7 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->adapters_dirty_lo = 0; ctx->adapters_dirty_hi = n_ad;
   ctx->routers_dirty_lo = 0; ctx->routers_dirty_hi = n_rt;
   ctx->slots_dirty_lo = 0; ctx->slots_dirty_hi = desc->max_requests;
-  size_t route_bytes = (size_t)desc->max_requests * desc->n_layers * sizeof(int32_t);
+  size_t route_bytes = (size_t)desc->max_requests * desc->n_layers * top_k_of(ctx) * sizeof(int32_t);
 #define CREATE_CUDA(call)                                            \
   do {                                                               \
     cudaError_t e__ = (call);                                        \
@@ -193,8 +202,10 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   CREATE_CUDA(cudaMalloc(&ctx->d_routers, n_rt * sizeof(RouterEntry)));
   CREATE_CUDA(cudaMalloc(&ctx->d_slot_tenant, desc->max_requests * sizeof(int32_t)));
   CREATE_CUDA(cudaMalloc(&ctx->d_route, route_bytes));
+  CREATE_CUDA(cudaMalloc(&ctx->d_gate, route_bytes));
   CREATE_CUDA(cudaMalloc(&ctx->d_err, 256));
   CREATE_CUDA(cudaMemset(ctx->d_route, 0xFF, route_bytes));
+  CREATE_CUDA(cudaMemset(ctx->d_gate, 0, route_bytes));
   CREATE_CUDA(cudaMemset(ctx->d_err, 0, 256));
   st = sync_tables(ctx, nullptr);
   if (st != MILORA_OK) return fail(st);
@@ -210,6 +221,7 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_routers);
   cudaFree(ctx->d_slot_tenant);
   cudaFree(ctx->d_route);
+  cudaFree(ctx->d_gate);
   cudaFree(ctx->d_err);
   cudaFree(ctx->d_scratch);
   cudaFree(ctx->d_counters);
@@ -344,8 +356,8 @@ milora_status milora_request_open(milora_ctx* ctx, int slot, int tenant) {
   if (ctx->h_slot_tenant[slot] >= 0) return MILORA_E_STATE;
   // The route row of a freshly opened slot must read "not routed".
   // The slot is closed, so no kernel in flight reads this row; the reset is finished before returning.
-  MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_route + (size_t)slot * ctx->desc.n_layers, 0xFF,
-                                   (size_t)ctx->desc.n_layers * sizeof(int32_t), nullptr));
+  const size_t row = (size_t)ctx->desc.n_layers * top_k_of(ctx);
+  MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_route + (size_t)slot * row, 0xFF, row * sizeof(int32_t), nullptr));
   MILORA_CUDA(ctx, cudaStreamSynchronize(nullptr));
   ctx->h_slot_tenant[slot] = tenant;
   mark(ctx->slots_dirty_lo, ctx->slots_dirty_hi, (size_t)slot);
@@ -400,9 +412,34 @@ milora_status milora_route_table_read(milora_ctx* ctx, int slot_begin, int n_slo
     return MILORA_E_ARG;
   if (n_slots == 0) return MILORA_OK;
   cudaStream_t s = as_stream(stream);
-  size_t L = ctx->desc.n_layers;
+  size_t L = (size_t)ctx->desc.n_layers * top_k_of(ctx);
   MILORA_CUDA(ctx, cudaMemcpyAsync(rows_host, ctx->d_route + (size_t)slot_begin * L, (size_t)n_slots * L * sizeof(int32_t),
                                    cudaMemcpyDeviceToHost, s));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  return MILORA_OK;
+}
+
+milora_status milora_gate_table_read(milora_ctx* ctx, int slot_begin, int n_slots, float* rows_host, void* stream) {
+  if (!ctx || !rows_host || slot_begin < 0 || n_slots < 0 || slot_begin + n_slots > ctx->desc.max_requests)
+    return MILORA_E_ARG;
+  if (n_slots == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  size_t L = (size_t)ctx->desc.n_layers * top_k_of(ctx);
+  MILORA_CUDA(ctx, cudaMemcpyAsync(rows_host, ctx->d_gate + (size_t)slot_begin * L, (size_t)n_slots * L * sizeof(float),
+                                   cudaMemcpyDeviceToHost, s));
+  MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  return MILORA_OK;
+}
+
+milora_status milora_gate_table_write(milora_ctx* ctx, int slot_begin, int n_slots, const float* rows_host,
+                                      void* stream) {
+  if (!ctx || !rows_host || slot_begin < 0 || n_slots < 0 || slot_begin + n_slots > ctx->desc.max_requests)
+    return MILORA_E_ARG;
+  if (n_slots == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  size_t L = (size_t)ctx->desc.n_layers * top_k_of(ctx);
+  MILORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_gate + (size_t)slot_begin * L, rows_host, (size_t)n_slots * L * sizeof(float),
+                                   cudaMemcpyHostToDevice, s));
   MILORA_CUDA(ctx, cudaStreamSynchronize(s));
   return MILORA_OK;
 }
@@ -411,9 +448,22 @@ milora_status milora_route_table_write(milora_ctx* ctx, int slot_begin, int n_sl
                                        void* stream) {
   if (!ctx || !rows_host || slot_begin < 0 || n_slots < 0 || slot_begin + n_slots > ctx->desc.max_requests)
     return MILORA_E_ARG;
-  size_t L = ctx->desc.n_layers;
+  size_t L = (size_t)ctx->desc.n_layers * top_k_of(ctx);
   for (size_t i = 0; i < (size_t)n_slots * L; ++i)
     if (rows_host[i] < -1 || rows_host[i] >= MILORA_NMOD) return MILORA_E_ARG;
+  {
+    // the modules selected for one (slot, layer) must be distinct: a module is applied at most once
+    const size_t K = top_k_of(ctx);
+    for (size_t c = 0; c < (size_t)n_slots * ctx->desc.n_layers; ++c) {
+      unsigned seen = 0;
+      for (size_t j = 0; j < K; ++j) {
+        const int m = rows_host[c * K + j];
+        if (m < 0) continue;
+        if ((seen >> m) & 1u) return MILORA_E_ARG;
+        seen |= 1u << m;
+      }
+    }
+  }
   if (n_slots == 0) return MILORA_OK;
   cudaStream_t s = as_stream(stream);
   MILORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_route + (size_t)slot_begin * L, rows_host, (size_t)n_slots * L * sizeof(int32_t),
@@ -424,8 +474,8 @@ milora_status milora_route_table_write(milora_ctx* ctx, int slot_begin, int n_sl
 
 milora_status milora_group_layout(const milora_ctx* ctx, int n_seq, int T, milora_group_layout_t* out) {
   if (!ctx || !out || n_seq < 0 || T < 0) return MILORA_E_ARG;
-  if (n_seq > kMaxSeq) return MILORA_E_CAPACITY;
-  *out = group_layout(n_seq, T);
+  if ((long long)n_seq * top_k_of(ctx) > kMaxSeq) return MILORA_E_CAPACITY;
+  *out = group_layout(n_seq, T, top_k_of(ctx));
   return MILORA_OK;
 }
 
@@ -435,9 +485,9 @@ milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   if (!ctx || !ws_dev) return MILORA_E_ARG;
   if (layer_begin < 0 || n_layers < 1 || layer_begin + n_layers > ctx->desc.n_layers) return MILORA_E_ARG;
   if (n_seq < 0 || T < 0 || (n_seq > 0 && !seq_slot_dev)) return MILORA_E_ARG;
-  if (n_seq > kMaxSeq) return MILORA_E_CAPACITY;
+  if ((long long)n_seq * top_k_of(ctx) > kMaxSeq) return MILORA_E_CAPACITY;
   if (!cu_seqlens_dev && T != n_seq) return MILORA_E_ARG;
-  milora_group_layout_t L = group_layout(n_seq, T);
+  milora_group_layout_t L = group_layout(n_seq, T, top_k_of(ctx));
   if (ws_stride < L.total || (ws_stride & 3) || (reinterpret_cast<uintptr_t>(ws_dev) & 15)) return MILORA_E_ARG;
   cudaStream_t s = as_stream(stream);
   milora_status st = sync_tables(ctx, s);
@@ -451,7 +501,8 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
   if (!ctx || !groups || !modules || !X_dev || !Y_dev) return MILORA_E_ARG;
   if (layer < 0 || layer >= ctx->desc.n_layers) return MILORA_E_ARG;
   if (n_sites < 1 || n_sites > kMaxSites) return MILORA_E_ARG;
-  if (!groups->ws_dev || groups->n_seq < 0 || groups->T < 0 || groups->n_seq > kMaxSeq) return MILORA_E_ARG;
+  if (!groups->ws_dev || groups->n_seq < 0 || groups->T < 0 || (long long)groups->n_seq * top_k_of(ctx) > kMaxSeq)
+    return MILORA_E_ARG;
   ApplySites sites;
   sites.n = n_sites;
   unsigned seen = 0;
@@ -523,7 +574,8 @@ milora_status plan_host_step(const milora_ctx* ctx, const milora_host_step* st, 
   pl->slot_p = o; o += up256((size_t)st->n_prompts * 4 + 4);
   pl->cu_s = o; o += up256((size_t)(st->n_seq + 1) * 4);
   pl->slot_s = o; o += up256((size_t)st->n_seq * 4 + 4);
-  pl->ws_stride = group_layout(st->n_seq, st->T).total;
+  if ((long long)st->n_seq * top_k_of(ctx) > kMaxSeq) return MILORA_E_CAPACITY;
+  pl->ws_stride = group_layout(st->n_seq, st->T, top_k_of(ctx)).total;
   pl->ws = o; o += up256(pl->ws_stride * 4);
   for (int m = 0; m < MILORA_NMOD; ++m) {
     pl->X[m] = pl->Y[m] = 0;

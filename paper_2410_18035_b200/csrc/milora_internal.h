@@ -54,9 +54,9 @@ struct GatherJob {       // up to kGatherRows rows anywhere in X / Y that share 
   const void* B;
   int32_t rank;
   float scale;
-  int32_t module, count, seg, pad;
+  int32_t module, count;
   int32_t rows[kGatherRows];
-  int32_t pad2[2];
+  float gate[kGatherRows];   // per-row weight of the LoRA term (1 unless probability gating is on)
 };
 struct TileJob {         // `count` consecutive rows starting at `start`
   const void* At;
@@ -76,9 +76,11 @@ struct DeviceTables {
   const AdapterEntry* adapters;   // [max_tenants][n_layers][7]
   const RouterEntry* routers;     // [max_tenants][n_layers]
   const int32_t* slot_tenant;     // [max_requests], -1 = closed
-  int32_t* route;                 // [max_requests][n_layers]
+  int32_t* route;                 // [max_requests][n_layers][top_k]
+  float* gate;                    // same shape: softmax probability of each selected module
   int32_t* err;                   // single flag word
   int n_layers, max_tenants, max_requests;
+  int top_k, gating;
 };
 
 __host__ __device__ inline size_t adapter_index(int tenant, int layer, int module, int n_layers) {
@@ -111,6 +113,7 @@ struct milora_ctx {
   milora::RouterEntry* d_routers;
   int32_t* d_slot_tenant;
   int32_t* d_route;
+  float* d_gate;
   int32_t* d_err;
   float* d_scratch;                             // router partial sums
   size_t scratch_floats;
@@ -135,7 +138,8 @@ milora_status cuda_fail(milora_ctx* ctx, cudaError_t e, const char* where);
 milora_status sync_tables(milora_ctx* ctx, cudaStream_t stream);
 DeviceTables device_tables(const milora_ctx* ctx);
 void module_dims(const milora_model_desc& d, int module, int* d1, int* d2);
-milora_group_layout_t group_layout(int n_seq, int T);
+milora_group_layout_t group_layout(int n_seq, int T, int top_k);
+inline int top_k_of(const milora_ctx* ctx) { return ctx->desc.top_k < 1 ? 1 : ctx->desc.top_k; }
 
 // ---- programmatic dependent launch ---------------------------------------------------------------
 // Every hot-path kernel is launched with the programmatic-stream-serialization attribute: it may start

@@ -331,8 +331,12 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   if (!rp || n_chunks == 0) {
     // closed slot, no router for this tenant at this layer, or an empty prompt: the request stays "not routed"
     if (tid == 0) {
-      if (slot >= 0 && slot < a.tab.max_requests) a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = -1;
-      else atomicOr(a.tab.err, ERR_BAD_SLOT);
+      if (slot >= 0 && slot < a.tab.max_requests) {
+        for (int j = 0; j < a.tab.top_k; ++j)
+          a.tab.route[((size_t)slot * a.tab.n_layers + a.layer) * a.tab.top_k + j] = -1;
+      } else {
+        atomicOr(a.tab.err, ERR_BAD_SLOT);
+      }
       if (p == 0) *a.sched = 0;
     }
     return;
@@ -406,16 +410,28 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   block_sum<MILORA_NMOD>(z, red);
   if (tid == 0) {
     float zmax = -FLT_MAX;
-    int best = 0;
 #pragma unroll
     for (int j = 0; j < MILORA_NMOD; ++j) {
       z[j] += r.bias[j];
-      if (z[j] > zmax) { zmax = z[j]; best = j; }   // strict: ties keep the lower index
+      zmax = fmaxf(zmax, z[j]);
     }
     float e[MILORA_NMOD], sum = 0.f;
 #pragma unroll
     for (int j = 0; j < MILORA_NMOD; ++j) { e[j] = expf(z[j] - zmax); sum += e[j]; }
-    a.tab.route[(size_t)slot * a.tab.n_layers + a.layer] = best;
+    // Eq. 3, Top-k: the k largest in descending order; the comparison is strict, so ties keep the lower index
+    const size_t cell = ((size_t)slot * a.tab.n_layers + a.layer) * a.tab.top_k;
+    unsigned taken = 0;
+    for (int q = 0; q < a.tab.top_k; ++q) {
+      int best = -1;
+      float bz = 0.f, be = 0.f;
+#pragma unroll
+      for (int j = 0; j < MILORA_NMOD; ++j) {
+        if (!((taken >> j) & 1u) && (best < 0 || z[j] > bz)) { best = j; bz = z[j]; be = e[j]; }
+      }
+      taken |= 1u << best;
+      a.tab.route[cell + q] = best;
+      a.tab.gate[cell + q] = be / sum;
+    }
     if (p == 0) *a.sched = 0;       // pass 1 of the next call starts its unit queue from zero
     if (a.logits_out) {
 #pragma unroll

@@ -19,14 +19,14 @@ class LoadedWorkload:
     """
 
     def __init__(self, w, device="cuda", layers=None, tenants=None, pool=POOL_MEAN, act=ACT_TANH, with_bias=False,
-                 max_requests=None, register_adapters=True):
+                 max_requests=None, register_adapters=True, top_k=1, gate=0):
         self.w = w
         self.device = torch.device(device)
         self.layers = list(range(w.n_layers)) if layers is None else list(layers)
         self.tenants = [int(t) for t in (w.active_tenants() if tenants is None else tenants)]
         self.pool, self.act, self.with_bias = pool, act, with_bias
         self.ml = Milora(len(self.layers), w.d_model, w.d_ff, w.d_kv, w.dtype, w.rank, w.n_tenants,
-                         max_requests or w.n_requests)
+                         max_requests or w.n_requests, top_k=top_k, gate=gate)
         for tenant in self.tenants:
             for li, layer in enumerate(self.layers):
                 self.register_router(tenant, li, layer)

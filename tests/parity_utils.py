@@ -85,15 +85,16 @@ def read_group_block(ml, ws_layer: torch.Tensor, n_seq: int, T: int):
     # (seg, start, count, module) per dense tile
     out["tiles"] = np.stack([tiles[:, 12], tiles[:, 13], tiles[:, 11], tiles[:, 10]], axis=1) if n_tiles else np.zeros((0, 4), int)
     out["tile_rank"] = tiles[:, 8].copy()
-    # (seg, count, module, rows[4]) per gather job
-    out["gather"] = [(int(g[8]), int(g[7]), int(g[6]), [int(v) for v in g[10:14]]) for g in gather]
+    # (count, module, rows[4]) per gather job, and the per-row weights (fp32 bit patterns in ints 12..15)
+    out["gather"] = [(int(g[7]), int(g[6]), [int(v) for v in g[8:12]]) for g in gather]
+    out["gather_gate"] = gather[:, 12:16].copy().view(np.float32) if n_gather else np.zeros((0, 4), np.float32)
     out["gather_rank"] = gather[:, 4].copy()
     return out
 
 
 def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_rows=4):
     """perm / seg_key / seg_offset / mod_offset / n_excluded are compared bit for bit; the work lists must
-    cover every active row exactly once, dense tiles with consecutive rows of long sequences only."""
+    cover every active (row, module) pair exactly once, dense tiles with consecutive rows of long sequences only."""
     assert g_gpu["n_excluded"] == g_oracle["n_excluded"]
     assert g_gpu["n_seg"] == len(g_oracle["seg_key"])
     assert np.array_equal(g_gpu["perm"], g_oracle["perm"])
@@ -105,29 +106,32 @@ def assert_groups_equal(g_gpu, g_oracle, cu, long_seq=32, tile_rows=128, gather_
     cu = np.asarray(cu)
     seq_of_row = np.repeat(np.arange(len(cu) - 1), np.diff(cu))
     seq_len = np.diff(cu)
+    max_tenants = g_oracle["max_tenants"]
     covered = []
-    seg_of_row = {}
+    seg_of_pair = {}
     for s in range(g_gpu["n_seg"]):
+        module = int(g_gpu["seg_key"][s]) // max_tenants
         for q in range(g_gpu["seg_offset"][s], g_gpu["seg_offset"][s + 1]):
-            seg_of_row[int(g_gpu["perm"][q])] = s
+            seg_of_pair[(int(g_gpu["perm"][q]), module)] = s
     for seg, start, count, module in g_gpu["tiles"]:
         assert 1 <= count <= tile_rows
         rows = list(range(start, start + count))
         assert len({seq_of_row[r] for r in rows}) == 1 and seq_len[seq_of_row[start]] >= long_seq
-        assert all(seg_of_row[r] == seg for r in rows)
-        assert module == g_gpu["seg_key"][seg] // (g_oracle["max_tenants"])
-        covered += rows
-    for seg, count, module, job_rows in g_gpu["gather"]:
+        assert all(seg_of_pair[(r, int(module))] == seg for r in rows)
+        assert module == g_gpu["seg_key"][seg] // max_tenants
+        covered += [(r, int(module)) for r in rows]
+    for count, module, job_rows in g_gpu["gather"]:
         assert 1 <= count <= gather_rows
         rows = job_rows[:count]
         assert all(r == -1 for r in job_rows[count:])
-        assert all(seg_of_row[r] == seg and seq_len[seq_of_row[r]] < long_seq for r in rows)
-        assert module == g_gpu["seg_key"][seg] // (g_oracle["max_tenants"])
-        covered += rows
-    assert sorted(covered) == sorted(int(r) for r in g_gpu["perm"]), "work lists do not cover the active rows exactly once"
+        assert len({seg_of_pair[(r, module)] for r in rows}) == 1, "rows of a gather job share one bucket"
+        assert all(seq_len[seq_of_row[r]] < long_seq for r in rows)
+        covered += [(r, module) for r in rows]
+    assert sorted(covered) == sorted(seg_of_pair.keys()), "work lists do not cover the active pairs exactly once"
+    assert len(covered) == len(g_gpu["perm"])
     for m in range(7):
         t0, t1 = g_gpu["mod_tile_offset"][m], g_gpu["mod_tile_offset"][m + 1]
         assert all(row[3] == m for row in g_gpu["tiles"][t0:t1])
         q0, q1 = g_gpu["mod_gather_offset"][m], g_gpu["mod_gather_offset"][m + 1]
-        assert all(job[2] == m for job in g_gpu["gather"][q0:q1])
+        assert all(job[1] == m for job in g_gpu["gather"][q0:q1])
     assert g_gpu["mod_tile_offset"][7] == g_gpu["n_tiles"] and g_gpu["mod_gather_offset"][7] == g_gpu["n_gather"]

@@ -42,8 +42,9 @@ def _route_all_layers(lw, ids, **okw):
     return table_g, table_o, excused
 
 
-def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False):
-    """group + apply (prefill and decode lists) on one step; compares grouping and all 7 module outputs."""
+def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, gate=None):
+    """group + apply (prefill and decode lists) on one step; compares grouping and all 7 module outputs.
+    table is [R, L] (top-1) or [R, L, k]; gate, when given, holds the [R, L, k] weights of the selected modules."""
     w, ml = lw.w, lw.ml
     layer = lw.layers[li]
     cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
@@ -75,7 +76,8 @@ def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False):
     torch.cuda.synchronize()
     worst = 0.0
     for m in range(7):
-        y_o = R.apply_site(w, layer, m, Xs[m].cpu(), Ybs[m].cpu(), token_slot, table[:, li])
+        y_o = R.apply_site(w, layer, m, Xs[m].cpu(), Ybs[m].cpu(), token_slot, table[:, li],
+                           gate=None if gate is None else gate[:, li])
         worst = max(worst, assert_apply_close(Ys[m], y_o, Ybs[m], w.dtype, what=f"{w.name} layer {layer} module {m}"))
     assert ml.poll_error() == 0
     return worst
@@ -158,6 +160,62 @@ def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r):
     w.request_tenant = w.request_tenant.copy()
     w.request_tenant[3] = -1
     _step_parity(lw, 0, prefill, decode, table, tag=9)
+    lw.close()
+
+
+@pytest.mark.parametrize("dtype,d,d_ff,d_kv,r,k,gate", [("f32", 256, 688, 256, 8, 3, 0), ("bf16", 512, 1408, 128, 16, 3, 0),
+                                                        ("bf16", 512, 1408, 512, 32, 2, 1), ("f32", 256, 688, 256, 8, 7, 1),
+                                                        ("bf16", 256, 688, 256, 40, 3, 1)])
+def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
+    """Eq. 3 with k > 1 (Section 4.5 sweeps k): the route table holds the k best modules in order, every token
+    is bucketed once per selected module and receives each selected module's LoRA term, optionally weighted by
+    the router probability."""
+    base = get_workload("c1")
+    n = len(RAGGED) + 6
+    lens = np.array(RAGGED + [16] * 6, dtype=np.int32)
+    tenants = np.array([0, 1, 2, 0, 1, 3, 2, 0, 0, 1, 1, 2, 3, 0], dtype=np.int32)
+    w = scaled_workload(base, name=f"topk_{dtype}", dtype=dtype, d_model=d, d_ff=d_ff, d_kv=d_kv, rank=r,
+                        n_tenants=5, request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(len(RAGGED)),
+                        decode_ids=np.arange(len(RAGGED), n), has_base_weights=False, n_layers=2)
+    lw = _loaded(w, tenants=[0, 1, 2, 3], top_k=k, gate=gate)
+    ids = list(range(n))
+    P = len(ids)
+    logits = torch.zeros((P, 7), dtype=torch.float32, device="cuda")
+    probs_o = np.zeros((w.n_requests, 2, 7))
+    excused = 0
+    for li in range(2):
+        lw.route(li, ids, logits=logits)
+        tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+        topk_o = np.full((w.n_requests, w.n_layers, k), -1, dtype=np.int32)
+        lo, _ = R.route_requests(w, li, ids, tmp, k=k, topk_table=topk_o)
+        probs_o[ids, li] = O.softmax(lo)
+        table_g = lw.ml.route_table_read(0, w.n_requests).numpy().reshape(w.n_requests, 2, k)
+        for p, i in enumerate(ids):
+            assert len(set(table_g[i, li].tolist())) == k
+            if not np.array_equal(table_g[i, li], topk_o[i, li]):
+                zs = np.sort(lo[p])[::-1]
+                gaps = zs[:k] - zs[1:k + 1] if k < 7 else zs[:6] - zs[1:7]
+                assert gaps.min() < 1e-3, f"top-k mismatch at request {i}: {table_g[i, li]} vs {topk_o[i, li]}"
+                excused += 1
+    assert excused <= 2
+    table = lw.ml.route_table_read(0, w.n_requests).numpy().reshape(w.n_requests, 2, k).copy()
+    gates_g = lw.ml.gate_table_read(0, w.n_requests).numpy()
+    gates_o = np.take_along_axis(probs_o, table.astype(np.int64), axis=2)
+    np.testing.assert_allclose(gates_g, gates_o, atol=2e-4)
+    gate_arg = gates_o if gate else None
+    prefill, decode = list(range(len(RAGGED))), list(range(len(RAGGED), n))
+    for li in range(2):
+        _step_parity(lw, li, prefill, decode, table, tag=11, gate=gate_arg)
+        _step_parity(lw, li, prefill[::-1], decode, table, tag=12, use_multi=True, gate=gate_arg)
+    # restoring a table by hand: duplicates inside a cell are refused
+    from paper_2410_18035_b200 import MiloraError
+    if k >= 2:
+        bad = table[:1].copy()
+        bad[0, 0, 1] = bad[0, 0, 0]
+        with pytest.raises(MiloraError):
+            lw.ml.route_table_write(0, bad)
+    lw.ml.route_table_write(0, table)
+    assert np.array_equal(lw.ml.route_table_read(0, w.n_requests).numpy().reshape(table.shape), table)
     lw.close()
 
 

@@ -336,6 +336,81 @@ def _tiny_stack(rng, d=8, d_ff=12, r=2, tenants=3):
     return ad
 
 
+def test_group_tokens_top_k_hand_example_and_library_sort():
+    """Eq. 3 with k > 1: a token sits in one bucket per selected module that has an adapter."""
+    # slot 0: tenant 1 selects modules (2, 0); slot 1: tenant 0 selects (2, 5) but has no adapter on 5;
+    # slot 2: closed; slot 3: tenant 2 selects (6, -1)
+    slot_tenant = [1, 0, -1, 2]
+    sel = np.array([[2, 0], [2, 5], [1, 3], [6, -1]])
+    token_slot = [0, 1, 2, 3, 0]
+    has = lambda tenant, module: not (tenant == 0 and module == 5)
+    g = O.group_tokens(token_slot, slot_tenant, sel, has, max_tenants=10)
+    # keys: slot0 -> 21 and 1; slot1 -> 20; slot3 -> 62
+    assert g["seg_key"].tolist() == [1, 20, 21, 62]
+    assert g["perm"].tolist() == [0, 4, 1, 0, 4, 3]
+    assert g["seg_offset"].tolist() == [0, 2, 3, 5, 6]
+    assert g["mod_offset"].tolist() == [0, 1, 1, 3, 3, 3, 3, 4]
+    assert g["n_excluded"] == 1
+    # a 2-D selection with one column is the top-1 case
+    col = np.array([2, 2, 1, 6])
+    g1 = O.group_tokens(token_slot, slot_tenant, col, has, 10)
+    g2 = O.group_tokens(token_slot, slot_tenant, col[:, None], has, 10)
+    for key in ("perm", "seg_key", "seg_offset", "mod_offset"):
+        assert np.array_equal(g1[key], g2[key])
+    # random case against a library sort of the explicit (key, token) pairs
+    rng = random.Random(31)
+    R, T, k, max_tenants = 9, 150, 3, 4
+    slot_tenant = [rng.choice([-1, 0, 1, 2, 3]) for _ in range(R)]
+    sel = np.array([rng.sample(range(7), k) for _ in range(R)])
+    sel[2, 1] = -1
+    token_slot = [rng.randrange(R) for _ in range(T)]
+    missing = {(1, 3), (2, 0), (3, 6)}
+    g = O.group_tokens(token_slot, slot_tenant, sel, lambda t, m: (t, m) not in missing, max_tenants)
+    keys, toks = [], []
+    for t in range(T):
+        s_ = token_slot[t]
+        for m in sel[s_]:
+            if slot_tenant[s_] >= 0 and m >= 0 and (slot_tenant[s_], int(m)) not in missing:
+                keys.append(int(m) * max_tenants + slot_tenant[s_]); toks.append(t)
+    keys, toks = np.array(keys), np.array(toks)
+    order = np.lexsort((toks, keys))
+    assert g["perm"].tolist() == toks[order].tolist()
+    assert g["n_excluded"] == T - len(set(toks.tolist()))
+    assert list(g["seg_key"]) == sorted(set(keys.tolist()))
+    counts = np.bincount(g["perm"], minlength=T)
+    assert counts.max() <= k
+
+
+def test_gate_weights_scale_the_lora_term():
+    """Weights of one reproduce hard selection; any weight scales that module's term linearly."""
+    rng = np.random.default_rng(33)
+    d, d_ff = 8, 12
+    ad = _tiny_stack(rng, d, d_ff, tenants=2)
+    slot_tenant = [0, 1]
+    sel = np.array([[4, 1], [1, 6]])
+    gate = np.array([[0.7, 0.2], [0.5, 0.25]])
+    token_slot = [0, 1, 1]
+    get = lambda t, mm: ad.get((t, mm))
+    for m in (1, 4, 6, 0):
+        d1, d2 = O.module_dims(d, d_ff, d, m)
+        x, yb = _rand(rng, 3, d1), _rand(rng, 3, d2)
+        hard = O.apply_module(yb, x, token_slot, slot_tenant, sel, m, get)
+        ones = O.apply_module(yb, x, token_slot, slot_tenant, sel, m, get, gate=np.ones((2, 2)))
+        assert np.array_equal(hard, ones)
+        soft = O.apply_module(yb, x, token_slot, slot_tenant, sel, m, get, gate=gate)
+        for t, slot in enumerate(token_slot):
+            if m in sel[slot]:
+                wgt = gate[slot][list(sel[slot]).index(m)]
+                A, B, s_ = ad[(slot_tenant[slot], m)]
+                np.testing.assert_allclose(soft[t], yb[t] + wgt * s_ * (x[t] @ A) @ B, rtol=1e-13)
+                np.testing.assert_allclose(soft[t] - yb[t], wgt * (hard[t] - yb[t]), rtol=1e-10, atol=1e-14)
+            else:
+                assert np.array_equal(soft[t], yb[t])
+        rows = [2, 0]
+        samp = O.apply_module_sampled(yb[rows], x[rows], rows, token_slot, slot_tenant, sel, m, get, gate=gate)
+        assert np.array_equal(samp, soft[rows])
+
+
 def test_apply_module_selection_invariants():
     rng = np.random.default_rng(21)
     d, d_ff = 8, 12
