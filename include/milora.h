@@ -241,6 +241,19 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
                                          const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                          void* stream);
 
+/* ---- fused projection (Eq. 1 in one pass) ---------------------------------------------------------
+ * Y_dev [T][d2] = X_dev [T][d1] . W_m + b_m for EVERY row of the step, plus s (x W^A) W^B on the rows of long
+ * sequences (the dense tiles of `groups`) whose request selects `module` at `layer`: the backbone's own
+ * projection and the LoRA term in one tensor-core kernel, so that Y is written once and never re-read.
+ * Wt_dev is W_m transposed, [d2][d1] row-major (the layout in which an nn.Linear keeps its weight);
+ * bias_dev is d2 values or NULL; all in bf16.  Rows of short sequences (the gathered list: decode tokens)
+ * receive only the base projection here; follow with milora_apply_decode for their LoRA term.
+ * Three launches (shrink, piece packing, persistent GEMM).  Returns MILORA_E_SHAPE unless the context is
+ * bf16, max_rank <= 32, d1 is a multiple of 64, d2 a multiple of 256 and T >= 128; such callers use their own
+ * GEMM followed by milora_apply_prefill.  Grows an internal scratch buffer like milora_route does. */
+milora_status milora_linear_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, const void* Wt_dev,
+                                    const void* bias_dev, void* Y_dev, const milora_groups* groups, void* stream);
+
 /* ---- one step from host buffers ------------------------------------------------------------------
  * The whole path for one layer with every input in HOST memory (pinned memory makes the copies
  * asynchronous): copy in, route the prompts (Eq. 2-3), group the step's sequences, apply Eq. 1 on

@@ -78,6 +78,7 @@ SIGNATURES = {
     "milora_apply_prefill": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_decode_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
     "milora_apply_prefill_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
+    "milora_linear_prefill": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_step_host_workspace": (_I, [_VP, C.POINTER(HostStep), C.POINTER(C.c_size_t)]),
     "milora_step_host": (_I, [_VP, C.POINTER(HostStep), _VP, C.c_size_t, _VP]),
     "milora_poll_error": (_I, [_VP, C.POINTER(_I), _VP]),
@@ -326,6 +327,17 @@ class Milora:
 
     def apply_prefill_multi(self, layer, modules, Xs, Ys, groups: Groups, stream=None):
         self._multi(self.lib.milora_apply_prefill_multi, "milora_apply_prefill_multi", layer, modules, Xs, Ys, groups, stream)
+
+    def linear_prefill(self, layer, module, X, Wt, Y, groups: Groups, bias=None, stream=None):
+        """milora_linear_prefill: Y = X W + b + LoRA term of the routed prompt rows; Wt is [d2, d1]."""
+        self._xy(module, X, Y, groups.T)
+        d1, d2 = self.module_dims(module)
+        self._tensor(Wt, self.torch_dtype, "Wt")
+        self._tensor(bias, self.torch_dtype, "bias")
+        if tuple(Wt.shape) != (d2, d1) or (bias is not None and bias.numel() != d2):
+            raise ValueError(f"linear_prefill: Wt must be [{d2}, {d1}] and bias [{d2}]")
+        self._check(self.lib.milora_linear_prefill(self.h, layer, module, _ptr(X), _ptr(Wt), _ptr(bias), _ptr(Y),
+                                                   C.byref(groups), _stream(stream)), "milora_linear_prefill")
 
     # -- one step from host buffers ------------------------------------------------------
     def make_host_step(self, layer, cu_prompts, prompt_slot, H, cu_seq, seq_slot, T, Xs, Ys) -> HostStep:

@@ -418,6 +418,284 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
 }
 
 // ------------------------------------------------------------------------------------------------------
+// fused projection: Y = X . W + b + s (X A) B on the routed rows   (Eq. 1 in one pass over Y)
+// ------------------------------------------------------------------------------------------------------
+// A persistent tensor-core GEMM over 128 x 256 output tiles (both operands K-major bf16, 64-element k steps
+// through a 4-stage TMA ring, two 256-column accumulators in tensor memory so that the epilogue of one tile
+// overlaps the main loop of the next).  The LoRA term rides on the same accumulator: after the k loop of a
+// tile, every dense LoRA tile that overlaps the tile's 128 rows contributes one more short MMA chain
+// V_piece (128 x rank, rows outside the overlap zero) . B (rank x 256).  V comes from the shrink kernel; a
+// small kernel packs it, per (LoRA tile, row block) piece, into the shared-memory operand image and lists the
+// pieces of every row block.  Y is written once and never read.
+constexpr int kLinBM = 128, kLinBN = 256, kLinBK = 64;
+constexpr int kLinStages = 4;
+constexpr int kLinAStage = kLinBM * kLinBK * 2;   // 16 KiB
+constexpr int kLinBStage = kLinBN * kLinBK * 2;   // 32 KiB
+constexpr int kLinThreads = 192;                  // warp 0 copies, warp 1 issues MMAs, warps 2..5 epilogue
+constexpr int kLinRPadMax = 32;
+constexpr int kMaxPieces = 12;                    // LoRA tile pieces that can overlap one block of 128 rows
+constexpr int kLinGroupM = 16;                    // row blocks per raster group (their X panels stay in L2)
+
+struct PackArgs {
+  int32_t* err;
+  const int32_t* ws;
+  milora_group_layout_t lay;
+  const float* vscratch;
+  unsigned char* vimg;       // [max_tiles][2][128 * rpad * 2 bytes]
+  int32_t* piece_cnt;        // [n_mblk], zero on entry
+  int32_t* piece_job;        // [n_mblk][kMaxPieces]: tile index * 2 + half
+  int module, T, rpad, n_mblk;
+};
+
+// One CTA per dense LoRA tile of the module: V = s * sum_k V_k rounded to bf16, written as the K-major operand
+// image (core matrix (row / 8, k / 8) at ((k / 8) * 16 + row / 8) * 128 bytes) of each of the (at most two)
+// 128-row blocks the tile overlaps, and the piece is appended to the block's list.
+__global__ void __launch_bounds__(kTileRows) linear_vpack_kernel(PackArgs a) {
+  const int tile_idx = blockIdx.x, m = threadIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int n_tiles = a.ws[a.lay.header + H_NTILES];
+  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
+  const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
+  if (job.module != a.module) return;
+  const int rp = job.rank_pad;
+  if (rp < 16 || rp > a.rpad || (rp & 15) || job.count < 1 || job.count > kTileRows || job.start < 0 ||
+      job.start + job.count > a.T) {
+    if (m == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  const size_t img_bytes = (size_t)kTileRows * a.rpad * 2;
+  unsigned char* img0 = a.vimg + (size_t)tile_idx * 2 * img_bytes;
+  for (int i = m; i < (int)(2 * img_bytes / 16); i += kTileRows) reinterpret_cast<uint4*>(img0)[i] = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  const int b0 = job.start / kTileRows;
+  if (m < job.count) {
+    const int row = job.start + m, h = row / kTileRows - b0, rb = row % kTileRows;
+    unsigned char* vrow = img0 + (size_t)h * img_bytes + (size_t)(rb >> 3) * 128 + (size_t)(rb & 7) * 16;
+    for (int c0 = 0; c0 < rp; c0 += 8) {
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll
+      for (int k = 0; k < kKSplit; ++k) {
+        const float4* src = reinterpret_cast<const float4*>(
+            a.vscratch + (((size_t)k * a.lay.max_tiles + tile_idx) * kTileRows + m) * a.rpad + c0);
+        const float4 u0 = __ldcg(src), u1 = __ldcg(src + 1);
+        acc[0] += u0.x; acc[1] += u0.y; acc[2] += u0.z; acc[3] += u0.w;
+        acc[4] += u1.x; acc[5] += u1.y; acc[6] += u1.z; acc[7] += u1.w;
+      }
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 hh = __floats2bfloat162_rn(acc[2 * i] * job.scale, acc[2 * i + 1] * job.scale);
+        w[i] = *reinterpret_cast<uint32_t*>(&hh);
+      }
+      *reinterpret_cast<uint4*>(vrow + (size_t)(c0 >> 3) * (kTileRows / 8) * 128) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+  if (m == 0) {
+    for (int h = 0; h < 2; ++h) {
+      const int b = b0 + h;
+      const int lo = max(job.start, b * kTileRows), hi = min(job.start + job.count, (b + 1) * kTileRows);
+      if (lo >= hi || b >= a.n_mblk) continue;
+      const int slot = atomicAdd(&a.piece_cnt[b], 1);
+      if (slot < kMaxPieces) a.piece_job[b * kMaxPieces + slot] = tile_idx * 2 + h;
+      else atomicOr(a.err, ERR_BAD_ITEM);
+    }
+  }
+}
+
+struct LinearArgs {
+  CUtensorMap xmap, wmap;
+  int32_t* err;
+  const int32_t* ws;
+  milora_group_layout_t lay;
+  const unsigned char* vimg;
+  const int32_t* piece_cnt;
+  const int32_t* piece_job;
+  const __nv_bfloat16* bias;   // d2 values or nullptr
+  __nv_bfloat16* Y;
+  int T, d1, d2, rpad, n_mblk, n_nblk;
+};
+
+__global__ void __launch_bounds__(kLinThreads, 1) linear_lora_kernel(const __grid_constant__ LinearArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t base = smem_u32(smem_raw);
+  const uint32_t as = base;
+  const uint32_t bs = as + kLinStages * kLinAStage;
+  const uint32_t vs = bs + kLinStages * kLinBStage;                 // V piece image, 128 x rpad bf16
+  const uint32_t lbs = vs + (uint32_t)kTileRows * a.rpad * 2u;      // B image, two 128-column chunks
+  const uint32_t bars = lbs + (uint32_t)a.rpad * 512u;
+  auto full = [&](int i) { return bars + 8u * i; };
+  auto empty = [&](int i) { return bars + 8u * (kLinStages + i); };
+  auto tfull = [&](int i) { return bars + 8u * (2 * kLinStages + i); };
+  auto tempty = [&](int i) { return bars + 8u * (2 * kLinStages + 2 + i); };
+  const uint32_t lfull = bars + 8u * (2 * kLinStages + 4), lempty = lfull + 8u;
+  const uint32_t slot = lempty + 8u;
+  volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  volatile int* abort_ptr = reinterpret_cast<volatile int*>(smem_raw + (slot + 4 - base));
+  constexpr uint32_t kCols = 2 * kLinBN;
+
+  pdl_launch_dependents();
+  if (tid == 0) {
+    *abort_ptr = 0;
+    for (int i = 0; i < kLinStages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
+    mbar_init(lfull, 1);
+    mbar_init(lempty, 1);
+    fence_barrier_init();
+    prefetch_tensormap(&a.xmap);
+    prefetch_tensormap(&a.wmap);
+  }
+  __syncthreads();
+  if (warp == 0) { tmem_alloc(slot, kCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *slot_ptr;
+  pdl_wait();
+
+  const int total = a.n_mblk * a.n_nblk, nk = a.d1 / kLinBK;
+  const int per_group = kLinGroupM * a.n_nblk;
+  auto tile_coords = [&](int t, int& mb, int& nb) {
+    const int g = t / per_group, r = t % per_group;
+    const int m0 = g * kLinGroupM;
+    const int gm = min(kLinGroupM, a.n_mblk - m0);
+    nb = r / gm;
+    mb = m0 + r % gm;
+  };
+  const TileJob* tiles = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles);
+  const bool bad = (base & 1023) != 0 || a.rpad > kLinRPadMax;
+  if (bad && tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+
+  if (!bad && warp == 0) {
+    if (lane == 0) {
+      // ---- copies: X and W tiles by TMA through the ring; V piece image and B image by bulk copies ----
+      int it = 0, lit = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        int mb, nb;
+        tile_coords(t, mb, nb);
+        for (int k = 0; k < nk && ok; ++k, ++it) {
+          const int s = it % kLinStages, ph = (it / kLinStages) & 1;
+          if (it >= kLinStages) ok = wait_bar(empty(s), ph ^ 1, abort_ptr, a.err);
+          if (!ok) break;
+          mbar_expect_tx(full(s), kLinAStage + kLinBStage);
+          tma_load_2d(as + s * kLinAStage, &a.xmap, k * kLinBK, mb * kLinBM, full(s));
+          tma_load_2d(bs + s * kLinBStage, &a.wmap, k * kLinBK, nb * kLinBN, full(s));
+        }
+        const int np = min(a.piece_cnt[mb], kMaxPieces);
+        for (int p = 0; p < np && ok; ++p, ++lit) {
+          if (lit >= 1) ok = wait_bar(lempty, (lit - 1) & 1, abort_ptr, a.err);
+          if (!ok) break;
+          const int pj = a.piece_job[mb * kMaxPieces + p];
+          const TileJob job = tiles[pj >> 1];
+          const uint32_t rp = (uint32_t)job.rank_pad;
+          mbar_expect_tx(lfull, rp * 256u + rp * 512u);
+          bulk_g2s(vs, a.vimg + (size_t)pj * ((size_t)kTileRows * a.rpad * 2), rp * 256u, lfull);
+          bulk_g2s(lbs, static_cast<const char*>(job.B_img) + (size_t)(2 * nb) * rp * 256u, rp * 512u, lfull);
+        }
+      }
+    }
+  } else if (!bad && warp == 1) {
+    if (lane == 0) {
+      // ---- MMAs ----
+      const uint32_t idesc = idesc_bf16_f32(kLinBM, kLinBN), idesc_l = idesc_bf16_f32(kLinBM, 128);
+      constexpr uint32_t kLbo = (kTileRows / 8) * 128u;
+      int it = 0, lit = 0, ti = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++ti) {
+        int mb, nb;
+        tile_coords(t, mb, nb);
+        const int b = ti & 1, bph = (ti >> 1) & 1;
+        if (ti >= 2) ok = wait_bar(tempty(b), bph ^ 1, abort_ptr, a.err);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t dcol = tmem_base + (uint32_t)b * kLinBN;
+        for (int k = 0; k < nk && ok; ++k, ++it) {
+          const int s = it % kLinStages, ph = (it / kLinStages) & 1;
+          ok = wait_bar(full(s), ph, abort_ptr, a.err);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kLinBK / 16; ++kk) {
+            const uint64_t da = smem_desc(as + s * kLinAStage + kk * 32, 16, 1024, 2);
+            const uint64_t db = smem_desc(bs + s * kLinBStage + kk * 32, 16, 1024, 2);
+            mma_bf16_ss(dcol, da, db, idesc, (k | kk) != 0);
+          }
+          mma_commit(empty(s));
+        }
+        if (!ok) break;
+        const int np = min(a.piece_cnt[mb], kMaxPieces);
+        for (int p = 0; p < np && ok; ++p, ++lit) {
+          const int pj = a.piece_job[mb * kMaxPieces + p];
+          const int rp = tiles[pj >> 1].rank_pad;
+          ok = wait_bar(lfull, lit & 1, abort_ptr, a.err);
+          if (!ok) break;
+          tc_fence_after();
+          for (int c = 0; c < 2; ++c) {
+            for (int kk = 0; kk < rp / 16; ++kk) {
+              const uint64_t da = smem_desc(vs + kk * 2 * kLbo, kLbo, 128, 0);
+              const uint64_t db = smem_desc(lbs + c * rp * 256 + kk * 2 * kLbo, kLbo, 128, 0);
+              mma_bf16_ss(dcol + c * 128, da, db, idesc_l, 1);
+            }
+          }
+          mma_commit(lempty);
+        }
+        if (!ok) break;
+        mma_commit(tfull(b));
+      }
+    }
+  } else if (!bad) {
+    // ---- epilogue: accumulator (+ bias) -> bf16 -> y, 64 bytes per thread and 32-column group ----
+    const int q = warp & 3;
+    const int rt = q * 32 + lane;
+    int ti = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++ti) {
+      int mb, nb;
+      tile_coords(t, mb, nb);
+      const int b = ti & 1, bph = (ti >> 1) & 1;
+      ok = wait_bar(tfull(b), bph, abort_ptr, a.err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = mb * kLinBM + rt;
+      __nv_bfloat16* yrow = a.Y + (size_t)row * a.d2 + (size_t)nb * kLinBN;
+      const uint32_t taddr = tmem_base + (uint32_t)b * kLinBN + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < kLinBN; c0 += 64) {
+        uint32_t d0[32], d1v[32];
+        tmem_ld32(taddr + c0, d0);
+        tmem_ld32(taddr + c0 + 32, d1v);
+        tmem_wait_ld();
+        if (a.bias) {
+          const __nv_bfloat16* bp = a.bias + (size_t)nb * kLinBN + c0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            d0[i] = __float_as_uint(__uint_as_float(d0[i]) + __bfloat162float(bp[i]));
+            d1v[i] = __float_as_uint(__uint_as_float(d1v[i]) + __bfloat162float(bp[32 + i]));
+          }
+        }
+        if (row < a.T) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(yrow + c0 + 8 * i) = pack8(d0 + 8 * i);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(yrow + c0 + 32 + 8 * i) = pack8(d1v + 8 * i);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty(b));
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, kCols);
+}
+
+// ------------------------------------------------------------------------------------------------------
 // registration-time operand images
 // ------------------------------------------------------------------------------------------------------
 // A image: for every 64-wide k chunk a block of rp x 64 bf16 as 8 x 16-byte core-matrix rows;
@@ -472,13 +750,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [rows][cols] bf16 row-major, tiles of 128 rows x 64 columns, 128-byte swizzle.
-bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols) {
+// [rows][cols] bf16 row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows = kTileRows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)kTileRows};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -506,9 +784,9 @@ milora_status launch_pack_images(milora_ctx* ctx, const void* At, const void* B,
   return MILORA_OK;
 }
 
-milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
-                                        cudaStream_t s) {
-  (void)layer;
+// shrink_only: stop after the shrink kernel (the fused projection consumes its partial products itself).
+static milora_status launch_prefill(milora_ctx* ctx, const ApplySites& sites, const milora_groups* g, bool shrink_only,
+                                    cudaStream_t s) {
   if (ctx->desc.dtype != MILORA_BF16) return MILORA_E_SHAPE;
   const int T = g->T;
   const int rpad = (ctx->desc.max_rank + 15) & ~15;
@@ -516,7 +794,8 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
   for (int i = 0; i < sites.n; ++i) {
     const ApplySite& st = sites.site[i];
     if (st.d1 % kBK || st.d2 % kBN) return MILORA_E_SHAPE;
-    if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (reinterpret_cast<uintptr_t>(st.Y) & 15)) return MILORA_E_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(st.X) & 15) || (!shrink_only && (reinterpret_cast<uintptr_t>(st.Y) & 15)))
+      return MILORA_E_SHAPE;
   }
   const size_t shrink_smem = (size_t)kShrinkStages * (kXStage + rpad * 128) + 128;
   const size_t expand_smem =
@@ -542,9 +821,10 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
   for (int i = 0; i < sites.n; ++i) {
     const ApplySite& st = sites.site[i];
     ps.module[i] = st.module; ps.d1[i] = st.d1; ps.d2[i] = st.d2; ps.Y[i] = st.Y;
-    if (!make_map(&sa.xmap[i], st.X, T, st.d1) || !make_map(&ea.ymap[i], st.Y, T, st.d2)) return MILORA_E_SHAPE;
+    if (!make_map(&sa.xmap[i], st.X, T, st.d1)) return MILORA_E_SHAPE;
+    if (!shrink_only && !make_map(&ea.ymap[i], st.Y, T, st.d2)) return MILORA_E_SHAPE;
   }
-  for (int i = sites.n; i < kMaxSites; ++i) { sa.xmap[i] = sa.xmap[0]; ea.ymap[i] = ea.ymap[0]; }
+  for (int i = sites.n; i < kMaxSites; ++i) { sa.xmap[i] = sa.xmap[0]; if (!shrink_only) ea.ymap[i] = ea.ymap[0]; }
   sa.sites = ps; sa.err = ctx->d_err; sa.ws = g->ws_dev; sa.lay = lay; sa.vscratch = ctx->d_vscratch; sa.T = T; sa.rpad = rpad;
   ea.sites = ps; ea.err = ctx->d_err; ea.ws = g->ws_dev; ea.lay = lay; ea.vscratch = ctx->d_vscratch; ea.T = T; ea.rpad = rpad;
 
@@ -553,7 +833,71 @@ milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplyS
   const size_t grid_s = (size_t)lay.max_tiles * kKSplit, grid_e = (size_t)lay.max_tiles * kNSplit;
   if (grid_s > 0x7fffffffull || grid_e > 0x7fffffffull) return MILORA_E_CAPACITY;
   MILORA_CUDA(ctx, launch_pdl(prefill_shrink_kernel, dim3((unsigned)grid_s), dim3(kShrinkThreads), shrink_smem, s, sa));
+  if (shrink_only) return MILORA_OK;
   MILORA_CUDA(ctx, launch_pdl(prefill_expand_kernel, dim3((unsigned)grid_e), dim3(kExpandThreads), expand_smem, s, ea));
+  return MILORA_OK;
+}
+
+milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                        cudaStream_t s) {
+  (void)layer;
+  return launch_prefill(ctx, sites, g, false, s);
+}
+
+// Y = X . W + b with the LoRA term of the routed dense tiles added in the same pass (Eq. 1):
+// shrink kernel (partial V) -> pack kernel (V pieces per row block) -> persistent GEMM.
+milora_status launch_linear_prefill_bf16(milora_ctx* ctx, int layer, int module, const void* X, const void* Wt,
+                                         const void* bias, void* Y, const milora_groups* g, cudaStream_t s) {
+  (void)layer;
+  if (ctx->desc.dtype != MILORA_BF16) return MILORA_E_SHAPE;
+  int d1, d2;
+  module_dims(ctx->desc, module, &d1, &d2);
+  const int T = g->T;
+  const int rpad = (ctx->desc.max_rank + 15) & ~15;
+  if (rpad > kLinRPadMax || T < kTileRows || d1 % kLinBK || d2 % kLinBN) return MILORA_E_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(X) & 15) || (reinterpret_cast<uintptr_t>(Y) & 15) ||
+      (reinterpret_cast<uintptr_t>(Wt) & 15) || (reinterpret_cast<uintptr_t>(bias) & 1))
+    return MILORA_E_SHAPE;
+  const milora_group_layout_t lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
+  const int n_mblk = (T + kLinBM - 1) / kLinBM, n_nblk = d2 / kLinBN;
+  const size_t img_bytes = (size_t)kTileRows * rpad * 2;
+  const size_t vimg_bytes = (size_t)lay.max_tiles * 2 * img_bytes;
+  const size_t cnt_off = (vimg_bytes + 255) & ~size_t(255);
+  const size_t job_off = cnt_off + (((size_t)n_mblk * 4 + 255) & ~size_t(255));
+  const size_t need = job_off + (size_t)n_mblk * kMaxPieces * 4;
+  if (need > ctx->lin_bytes) {
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+    if (ctx->d_lin) MILORA_CUDA(ctx, cudaFree(ctx->d_lin));
+    ctx->d_lin = nullptr;
+    ctx->lin_bytes = 0;
+    MILORA_CUDA(ctx, cudaMalloc(&ctx->d_lin, need));
+    ctx->lin_bytes = need;
+  }
+  unsigned char* lin = static_cast<unsigned char*>(ctx->d_lin);
+  MILORA_CUDA(ctx, cudaMemsetAsync(lin + cnt_off, 0, (size_t)n_mblk * 4, s));
+
+  ApplySites sites;
+  sites.n = 1;
+  sites.site[0].module = module; sites.site[0].X = X; sites.site[0].Y = nullptr; sites.site[0].d1 = d1; sites.site[0].d2 = d2;
+  milora_status st = launch_prefill(ctx, sites, g, true, s);
+  if (st != MILORA_OK) return st;
+
+  PackArgs pa;
+  pa.err = ctx->d_err; pa.ws = g->ws_dev; pa.lay = lay; pa.vscratch = ctx->d_vscratch; pa.vimg = lin;
+  pa.piece_cnt = reinterpret_cast<int32_t*>(lin + cnt_off); pa.piece_job = reinterpret_cast<int32_t*>(lin + job_off);
+  pa.module = module; pa.T = T; pa.rpad = rpad; pa.n_mblk = n_mblk;
+  if (lay.max_tiles > 0)
+    MILORA_CUDA(ctx, launch_pdl(linear_vpack_kernel, dim3((unsigned)lay.max_tiles), dim3(kTileRows), 0, s, pa));
+
+  LinearArgs la;
+  if (!make_map(&la.xmap, X, T, d1, kLinBM) || !make_map(&la.wmap, Wt, d2, d1, kLinBN)) return MILORA_E_SHAPE;
+  la.err = ctx->d_err; la.ws = g->ws_dev; la.lay = lay; la.vimg = lin; la.piece_cnt = pa.piece_cnt; la.piece_job = pa.piece_job;
+  la.bias = static_cast<const __nv_bfloat16*>(bias); la.Y = static_cast<__nv_bfloat16*>(Y);
+  la.T = T; la.d1 = d1; la.d2 = d2; la.rpad = rpad; la.n_mblk = n_mblk; la.n_nblk = n_nblk;
+  const size_t smem = (size_t)kLinStages * (kLinAStage + kLinBStage) + (size_t)kTileRows * rpad * 2 + (size_t)rpad * 512 + 256;
+  MILORA_CUDA(ctx, cudaFuncSetAttribute(linear_lora_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int grid = std::min(n_mblk * n_nblk, ctx->sm_count);
+  MILORA_CUDA(ctx, launch_pdl(linear_lora_kernel, dim3((unsigned)grid), dim3(kLinThreads), smem, s, la));
   return MILORA_OK;
 }
 

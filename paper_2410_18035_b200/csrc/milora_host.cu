@@ -167,6 +167,7 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->d_gate = nullptr;
   ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
   ctx->d_vscratch = nullptr; ctx->vscratch_floats = 0;
+  ctx->d_lin = nullptr; ctx->lin_bytes = 0;
   ctx->n_counters = 0;
   milora_status st = MILORA_OK;
   auto fail = [&](milora_status s) { milora_destroy(ctx); return s; };
@@ -226,6 +227,7 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_scratch);
   cudaFree(ctx->d_counters);
   cudaFree(ctx->d_vscratch);
+  cudaFree(ctx->d_lin);
   ctx->arena.release();
   delete ctx;
   return MILORA_OK;
@@ -548,6 +550,19 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
                                          const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                          void* stream) {
   return apply_common(ctx, layer, n_sites, modules, X_dev, Y_dev, groups, true, stream);
+}
+
+milora_status milora_linear_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, const void* Wt_dev,
+                                    const void* bias_dev, void* Y_dev, const milora_groups* groups, void* stream) {
+  if (!ctx || !groups || !X_dev || !Wt_dev || !Y_dev) return MILORA_E_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers || module < 0 || module >= MILORA_NMOD) return MILORA_E_ARG;
+  if (!groups->ws_dev || groups->n_seq < 0 || groups->T < 0 || (long long)groups->n_seq * top_k_of(ctx) > kMaxSeq)
+    return MILORA_E_ARG;
+  if (groups->T == 0) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);
+  if (st != MILORA_OK) return st;
+  return launch_linear_prefill_bf16(ctx, layer, module, X_dev, Wt_dev, bias_dev, Y_dev, groups, s);
 }
 
 // ---- one step from host buffers ---------------------------------------------------------------------

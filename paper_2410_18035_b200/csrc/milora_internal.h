@@ -121,6 +121,8 @@ struct milora_ctx {
   size_t n_counters;
   float* d_vscratch;                            // prefill: fp32 partial x.A products [k-split][T][rank_pad]
   size_t vscratch_floats;
+  void* d_lin;                                  // fused projection: V piece images and per-row-block piece lists
+  size_t lin_bytes;
   milora::Arena arena;
   std::string cuda_error;
 };
@@ -202,6 +204,9 @@ milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySi
 // and the registration-time packing of the operand images they read.
 milora_status launch_apply_prefill_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
                                         cudaStream_t s);
+// bf16 fused projection Y = X . W + b + LoRA term of the routed dense tiles (same MILORA_E_SHAPE convention).
+milora_status launch_linear_prefill_bf16(milora_ctx* ctx, int layer, int module, const void* X, const void* Wt,
+                                         const void* bias, void* Y, const milora_groups* g, cudaStream_t s);
 bool prefill_images_supported(const milora_ctx* ctx, int d1, int d2, int rank);
 size_t prefill_image_bytes(int d, int rank);
 milora_status launch_pack_images(milora_ctx* ctx, const void* At, const void* B, void* At_img, void* B_img, int d1, int d2,

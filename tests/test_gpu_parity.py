@@ -219,6 +219,58 @@ def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
     lw.close()
 
 
+def _assert_fused_close(Y, y_o, y_base_o, what):
+    """Fused projection against the oracle's x W + b + delta: full-output metric, and per element an error
+    budget of the delta tolerance plus the rounding of the stored bf16 output (two roundings on decode rows:
+    the projection is stored, then the gathered kernel adds the LoRA term) and of the fp32 accumulation."""
+    from parity_utils import TOL, half_ulp
+    yg, yr = R.to_f64(Y), np.asarray(y_o, dtype=np.float64)
+    assert O.max_rel_err(yg, yr) <= TOL["bf16"], what
+    delta = yr - y_base_o
+    rms = np.sqrt(np.mean(delta[np.any(delta != 0, axis=1)] ** 2)) if np.any(delta != 0) else 0.0
+    allowed = TOL["bf16"] * np.where(delta != 0, np.maximum(np.abs(delta), rms), 0.0) + 2.0 * half_ulp(yr, "bf16") + 2e-5
+    worst = float((np.abs(yg - yr) / allowed).max())
+    assert worst <= 1.0, f"{what}: error is {worst:.3f}x the allowed bound"
+
+
+@pytest.mark.parametrize("d,d_ff,d_kv,r,k", [(512, 1536, 256, 16, 1), (256, 768, 256, 32, 1), (512, 1536, 512, 8, 3)])
+def test_fused_projection_matches_oracle(d, d_ff, d_kv, r, k):
+    """milora_linear_prefill: y = x W + b + s (x A) B on the routed prompt rows in one kernel (Eq. 1), ragged
+    sequences that straddle the 128-row blocks of the GEMM, then the decode rows through milora_apply_decode."""
+    base = get_workload("c1")
+    n = len(RAGGED) + 6
+    lens = np.array(RAGGED + [1] * 6, dtype=np.int32)
+    tenants = np.array([0, 1, 2, 0, 1, 3, 2, 0, 0, 1, 1, 2, 3, 0], dtype=np.int32)
+    w = scaled_workload(base, name="fused", dtype="bf16", d_model=d, d_ff=d_ff, d_kv=d_kv, rank=r, n_tenants=5,
+                        request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(len(RAGGED)),
+                        decode_ids=np.arange(len(RAGGED), n), has_base_weights=False, n_layers=1)
+    lw = _loaded(w, tenants=[0, 1, 2, 3], top_k=k)
+    ml = lw.ml
+    ids = list(range(n))
+    lw.route(0, ids)
+    table = ml.route_table_read(0, w.n_requests).numpy().reshape(w.n_requests, 1, k)
+    prefill, decode = list(range(len(RAGGED)))[::-1], list(range(len(RAGGED), n))
+    cu, slots, T = lw.seq_arrays(prefill, decode)
+    n_seq = slots.numel()
+    ws = ml.alloc_group_ws(1, n_seq, T)
+    ml.group(0, 1, cu, slots, n_seq, T, ws)
+    groups = ml.groups(ws[0], n_seq, T)
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu.cpu().numpy()))
+    for m in range(7):
+        X = w.module_input(0, m, T, 21, "cuda")
+        W = w.base_weight(0, m, "cuda")
+        bias = (w.base_output(0, m, 1, 22, "cuda")[0] * 0.1).contiguous() if m % 2 else None
+        Y = torch.full((T, W.shape[1]), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ml.linear_prefill(0, m, X, W.t().contiguous(), Y, groups, bias=bias)
+        ml.apply_decode(0, m, X, Y, groups)
+        torch.cuda.synchronize()
+        yb = O.base_projection(R.to_f64(X), R.to_f64(W), None if bias is None else R.to_f64(bias))
+        y_o = R.apply_site(w, 0, m, X.cpu(), yb, token_slot, table[:, 0])
+        _assert_fused_close(Y, y_o, yb, f"fused projection module {m}")
+    assert ml.poll_error() == 0
+    lw.close()
+
+
 def test_tenant_without_adapter_is_excluded():
     base = get_workload("c1")
     w = scaled_workload(base, n_tenants=6)
