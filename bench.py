@@ -279,6 +279,9 @@ def run_ours(args, rank, world, device):
     ms_per_step = total_ms / args.steps
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
+    fused = None
+    if rank == 0 and not args.skip_fused and w.dtype == "bf16":
+        fused = run_fused_projection(step, routes, device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
 
@@ -321,6 +324,7 @@ def run_ours(args, rank, world, device):
             "router_gbs": rooflines["router"]["achieved"],
             "group_prefill_us": gp_ms * 1e3, "group_decode_us": gd_ms * 1e3,
             "ms_per_step_with_phase_events": float(phase_ms.sum()),
+            "fused_projection": fused,
         },
         "roofline": dict(rooflines[dom], kernel=dom),
         "rooflines": rooflines,
@@ -329,6 +333,45 @@ def run_ours(args, rank, world, device):
         "clocks": clocks,
     }
     out["cpu_baseline"] = None if args.skip_cpu else cpu_baseline(w, args)
+    return out
+
+
+def run_fused_projection(step, routes, device, peaks, iters=10):
+    """The fused projection y = x W + b + LoRA term (milora_linear_prefill) on the step's prompt rows, for the q and
+    down call sites: TFLOP/s of the whole call (shrink + piece packing + GEMM), with torch.matmul on the same
+    operands timed beside it.  Not part of the timed step; reported in `breakdown`."""
+    ml, w = step.lw.ml, step.w
+    out = {}
+    for name, m in (("q", 0), ("down", 6)):
+        d1, d2 = w.dims(m)
+        g = torch.Generator(device=device)
+        g.manual_seed(1234 + m)
+        Wt = (torch.randn((d2, d1), generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        X = step.Xp[m]
+        Y = torch.empty((step.T_p, d2), dtype=torch.bfloat16, device=device)
+        lora_flops = sum(2 * int(w.prompt_len[i]) * w.rank * (d1 + d2) for i in step.prefill_ids if int(routes[i]) == m)
+        flops = 2 * step.T_p * d1 * d2 + lora_flops
+
+        def timed(fn):
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize(device)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                fn()
+            e1.record()
+            torch.cuda.synchronize(device)
+            return e0.elapsed_time(e1) / iters
+
+        ms = timed(lambda: ml.linear_prefill(0, m, X, Wt, Y, step.g_p))
+        ms_lib = timed(lambda: torch.matmul(X, Wt.t(), out=Y))
+        out[name] = {"ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                     "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "library_matmul_ms_base_projection_only": ms_lib,
+                     "library_matmul_tflops": 2 * step.T_p * d1 * d2 / (ms_lib * 1e-3) / 1e12,
+                     "shape": [step.T_p, d1, d2], "launches": 3}
+        del Wt, Y
     return out
 
 
@@ -466,6 +509,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
+    ap.add_argument("--skip-fused", action="store_true", help="leave out the fused-projection timing")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle timing")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -172,3 +172,54 @@ def test_decode_batch_sweep_small_batches():
         table = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0].copy()
         _check_step(lw, 0, [], ids, table, tag=b, rng=rng)
         lw.close()
+
+
+def test_config2_fused_projection_full_size():
+    """milora_linear_prefill at the benchmark's size (32,768 prompt rows of the LLaMA-2-7B layer; q: 4096 -> 4096 and
+    down: 11008 -> 4096), weights drawn as bench.py draws them.  The oracle recomputes sampled rows one by one
+    (x W in fp64 plus the LoRA term); every row must differ from the plain projection exactly where its request
+    selects the module."""
+    from parity_utils import half_ulp
+    w = get_workload("c2")
+    w.gen_device = "cuda"
+    lw = _loaded(w, layers=[0])
+    ml = lw.ml
+    ids = list(range(64))
+    table, _ = _route_and_check(lw, 0, ids)
+    cu, slots, T = lw.seq_arrays(ids, [])
+    ws = ml.alloc_group_ws(1, 64, T)
+    ml.group(0, 1, cu, slots, 64, T, ws)
+    groups = ml.groups(ws[0], 64, T)
+    cu_h = cu.cpu().numpy()
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
+    rng = np.random.default_rng(5)
+    rows = _sample_rows(cu_h, rng, per_seq=2)
+    idx = torch.from_numpy(rows).cuda()
+    for m in (0, 6):
+        d1, d2 = w.dims(m)
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1234 + m)
+        Wt = (torch.randn((d2, d1), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        X = w.module_input(0, m, T, 0, "cuda")
+        Y = torch.full((T, d2), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ml.linear_prefill(0, m, X, Wt, Y, groups)
+        torch.cuda.synchronize()
+        assert ml.poll_error() == 0
+        assert not bool(torch.isnan(Y.float()).any()), "a tile of the output was not written"
+        yb = O.base_projection(R.to_f64(X[idx]), R.to_f64(Wt).T)
+        y_o = R.apply_site(w, 0, m, X[idx].cpu(), yb, token_slot, table, rows=rows)
+        yg = R.to_f64(Y[idx])
+        assert O.max_rel_err(yg, y_o) <= TOL["bf16"]
+        delta = y_o - yb
+        routed = table[token_slot[rows]] == m
+        assert np.array_equal(np.any(delta != 0, axis=1), routed)
+        rms = np.sqrt(np.mean(delta[routed] ** 2)) if routed.any() else 0.0
+        allowed = TOL["bf16"] * np.where(delta != 0, np.maximum(np.abs(delta), rms), 0.0) + 1.01 * half_ulp(y_o, "bf16") + 1e-4
+        worst = float((np.abs(yg - y_o) / allowed).max())
+        assert worst <= 1.0, f"fused projection module {m}: error is {worst:.3f}x the allowed bound"
+        # the LoRA term is really there: on routed rows the output differs from the plain projection
+        plain = (X[idx].float() @ Wt.float().t()).to(torch.bfloat16)
+        differs = (plain != Y[idx]).float().mean(dim=1).cpu().numpy()
+        assert (differs[routed] > 0.5).all() and (differs[~routed] < 0.02).all()
+        del Wt, X, Y
+    lw.close()
