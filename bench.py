@@ -279,9 +279,10 @@ def run_ours(args, rank, world, device):
     ms_per_step = total_ms / args.steps
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
-    fused = None
+    fused = stack = None
     if rank == 0 and not args.skip_fused and w.dtype == "bf16":
         fused = run_fused_projection(step, routes, device, load_peaks())
+        stack = run_decode_stack(step, device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
 
@@ -325,6 +326,7 @@ def run_ours(args, rank, world, device):
             "group_prefill_us": gp_ms * 1e3, "group_decode_us": gd_ms * 1e3,
             "ms_per_step_with_phase_events": float(phase_ms.sum()),
             "fused_projection": fused,
+            "decode_stack": stack,
         },
         "roofline": dict(rooflines[dom], kernel=dom),
         "rooflines": rooflines,
@@ -373,6 +375,56 @@ def run_fused_projection(step, routes, device, peaks, iters=10):
                      "shape": [step.T_p, d1, d2], "launches": 3}
         del Wt, Y
     return out
+
+
+def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
+    """The decode kernel in the setting it serves in: one launch per Transformer layer, back to back, each layer with
+    its own routes and adapters (here the first `n_layers` layers of a LLaMA-2-7B stack; 7 call sites per launch).
+    One round touches n_layers x ~27 MB of distinct adapters (more than L2), so every launch reads from HBM.
+    Reports the average launch duration inside the chain; not part of the timed step."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth.workloads import scaled_workload
+    w8 = scaled_workload(step.w, n_layers=n_layers)
+    w8.gen_device = str(device)
+    lw8 = LoadedWorkload(w8, device)
+    ml = lw8.ml
+    for li in range(n_layers):
+        ml.route(li, step.H, step.cu_p, step.slots_p)      # routers differ per layer, so the routes do too
+    n = len(step.decode_ids)
+    ws = ml.alloc_group_ws(n_layers, n, step.T_d)
+    ml.group(0, n_layers, step.cu_d, step.slots_d, n, step.T_d, ws)
+    groups = [ml.groups(ws[li], n, step.T_d) for li in range(n_layers)]
+    routes = ml.route_table_read(0, w8.n_requests).numpy()
+    nbytes = sum(algorithmic_work(w8, routes[:, li], [], step.decode_ids)["decode_bytes"] for li in range(n_layers))
+
+    def one_round():
+        for li in range(n_layers):
+            ml.apply_decode_multi(li, step.mods, step.Xd, step.Yd, groups[li])
+
+    for _ in range(3):
+        one_round()
+    torch.cuda.synchronize(device)
+    # the chain is replayed from a CUDA graph, as a serving engine replays its decode step: the Python binding
+    # needs longer per call than the kernel runs
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one_round()
+    graph.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(rounds):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    ms = e0.elapsed_time(e1) / (rounds * n_layers)
+    err = ml.poll_error()
+    del graph
+    lw8.close()
+    gbs = nbytes / n_layers / (ms * 1e-3) / 1e9
+    return {"layers": n_layers, "us_per_layer_launch": ms * 1e3, "algorithmic_bytes_per_layer": nbytes // n_layers,
+            "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
+            "decode_token_layers_per_s": n / (ms * 1e-3), "device_error_flag": err}
 
 
 def run_e2e(step, args, world, device, tokens_per_step):

@@ -5,14 +5,15 @@
 // design is about getting every byte requested at once:
 //   * one thread-block cluster of kC CTAs per job; CTA c owns a 1/kC slice of the d1 columns (shrink)
 //     and a 1/kC slice of the d2 columns (expand);
-//   * at start, one warp issues bulk copies (cp.async.bulk, completion on an mbarrier) for the CTA's
-//     slice of B, and every thread loads its 16-byte pieces of y into registers - neither depends on
-//     the shrink result, so they are in flight while x . A is being reduced;
-//   * the A^T slice is consumed straight from global memory with 128-bit loads, four per thread in
-//     flight (it is read once, so staging it in shared memory would only cost occupancy);
-//   * each CTA reduces its d1 slice to partial sums v_c[row][j]; the partials are exchanged through
-//     distributed shared memory and added in CTA order (deterministic), then each CTA finishes its
-//     d2 slice and writes y with 128-bit stores.
+//   * at start every thread asks for its lines of the A^T and x slices with L2 prefetches, one warp issues
+//     bulk copies (cp.async.bulk, completion on an mbarrier) for the CTA's slice of B, and every thread loads
+//     its 16-byte pieces of y into registers: the whole job is in flight before anything is consumed;
+//   * the A^T slice is then consumed from global memory with 128-bit loads, four per thread per batch
+//     (it is read once, so staging it in shared memory would only cost occupancy); later batches hit L2;
+//   * each CTA reduces its d1 slice to partial sums v_c[row][j]; the partials go to every CTA of the cluster
+//     through distributed shared memory with st.async, which counts their arrival on the receiver's
+//     mbarrier (no cluster-wide barrier), and are added in CTA order (deterministic); then each CTA
+//     finishes its d2 slice and writes y with 128-bit stores.
 // No scratch in global memory, no atomics.  Every wait is bounded; a timeout raises ERR_WAIT_TIMEOUT.
 #include "milora_internal.h"
 
@@ -63,20 +64,25 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
+// "This CTA is running and its barriers are initialised" (made visible by fence.mbarrier_init before it):
+// nothing else has to be released, so the arrive is relaxed.
 __device__ __forceinline__ void cluster_arrive() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void cluster_wait() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t peer, float v) {
-  uint32_t remote;
+// One fp32 value into the same shared-memory location of CTA `peer` of the cluster; its arrival is counted
+// (4 bytes) on that CTA's mbarrier, so the receiver needs no cluster-wide barrier to know the data is there.
+__device__ __forceinline__ void st_async_f32(uint32_t local_addr, uint32_t local_bar, uint32_t peer, float v) {
+  uint32_t remote, remote_bar;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote_bar) : "r"(local_bar), "r"(peer));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote),
+               "r"(__float_as_uint(v)), "r"(remote_bar)
+               : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   uint4 q;
@@ -167,17 +173,38 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   float* mine = part + kC * kR * a.rmax;                                    // [kR][rmax]
   float* v_sm = mine + kR * a.rmax;                                         // [kR][rmax]
   uint4* B_sm = reinterpret_cast<uint4*>(v_sm + kR * a.rmax);               // [rmax][per2max]
-  const uint32_t bar = smem_u32(&bars[0]);
+  const uint32_t bar = smem_u32(&bars[0]);        // completion of the B copies
+  const uint32_t xbar = smem_u32(&bars[1]);       // arrival of the partial sums of all CTAs of the cluster
 
+  // ---- everything the CTA will read is requested now: A^T and x into L2, B by bulk copies, y into registers ----
+  // (a thread's later 128-bit loads of A^T then find their lines in L2 or on the way, also when its slice
+  // needs several batches of loads)
+  {
+    const size_t slice_bytes = (size_t)cnt1 * 16;
+    const int n_lines = cnt1 > 0 ? (int)((slice_bytes + 127) / 128) + 1 : 0;
+    for (int j = tid / kSegs; j < r; j += kRowsPerPass) {
+      const char* p = reinterpret_cast<const char*>(At + (size_t)j * d1 + (size_t)lo1 * 8);
+      for (int l = tid % kSegs; l < n_lines; l += kSegs) prefetch_l2(p + min((size_t)l * 128, slice_bytes - 16));
+    }
+    if (tid / kSegs < n) {            // kRowsPerPass >= kR: one group of kSegs threads per row of the job
+      const int t = tid / kSegs;
+      int row = rows[0];
+#pragma unroll
+      for (int q = 1; q < kR; ++q) row = (t == q) ? rows[q] : row;
+      const char* p = reinterpret_cast<const char*>(X + (size_t)row * d1 + (size_t)lo1 * 8);
+      for (int l = tid % kSegs; l < n_lines; l += kSegs) prefetch_l2(p + min((size_t)l * 128, slice_bytes - 16));
+    }
+  }
   if (tid == 0) {
     mbar_init(bar, 1);
+    mbar_init(xbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  cluster_arrive();       // "this CTA is running"; waited for right before the first remote store
+  cluster_arrive();       // waited for right before the first remote store
+  if (tid == 0) mbar_expect_tx(xbar, (uint32_t)(kC * n * r) * 4u);
 
-  // ---- B slice by bulk copies, y pieces into registers: nothing here depends on the shrink ------
-  if (warp == 0) {
+  if (warp == kThreads / 32 - 1) {
     const char* Bm = static_cast<const char*>(job.B);
     if (lane == 0) mbar_expect_tx(bar, (uint32_t)r * cnt2 * 16u);
     __syncwarp();
@@ -249,13 +276,19 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
     }
   }
   __syncthreads();
-  cluster_wait();         // every CTA of the cluster has started, so its shared memory can be written
-  // hand this CTA's partial sums to every CTA of the cluster (slot `crank` of their `part`), one store per thread
+  cluster_wait();         // every CTA of the cluster has started and initialised its barriers
+  // hand this CTA's partial sums to every CTA of the cluster (slot `crank` of their `part`), one store per thread;
+  // each store is counted on the receiver's barrier
   for (int idx = tid; idx < n * r * kC; idx += kThreads) {
     const int peer = idx % kC, e = idx / kC, t = e / r, j = e % r;
-    st_cluster_f32(smem_u32(part + ((size_t)crank * kR + t) * a.rmax + j), (uint32_t)peer, mine[t * a.rmax + j]);
+    st_async_f32(smem_u32(part + ((size_t)crank * kR + t) * a.rmax + j), xbar, (uint32_t)peer, mine[t * a.rmax + j]);
   }
-  cluster_sync_all();     // all partial sums have landed everywhere; nobody writes remote memory after this
+  // all kC x n x r partial sums have landed here; the peers wait for theirs likewise, so nobody is written after it left
+  if (!mbar_wait(xbar, 0)) {
+    if (tid == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
+    mbar_wait(bar, 0);
+    return;
+  }
 
   for (int idx = tid; idx < n * r; idx += kThreads) {
     const int t = idx / r, j = idx % r;
