@@ -279,10 +279,11 @@ def run_ours(args, rank, world, device):
     ms_per_step = total_ms / args.steps
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
-    fused = stack = None
+    fused = stack = stack13 = None
     if rank == 0 and not args.skip_fused and w.dtype == "bf16":
         fused = run_fused_projection(step, routes, device, load_peaks())
         stack = run_decode_stack(step, device, load_peaks())
+        stack13 = run_decode_13b(device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
 
@@ -327,6 +328,7 @@ def run_ours(args, rank, world, device):
             "ms_per_step_with_phase_events": float(phase_ms.sum()),
             "fused_projection": fused,
             "decode_stack": stack,
+            "decode_stack_13b_zipf": stack13,
         },
         "roofline": dict(rooflines[dom], kernel=dom),
         "rooflines": rooflines,
@@ -377,35 +379,26 @@ def run_fused_projection(step, routes, device, peaks, iters=10):
     return out
 
 
-def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
-    """The decode kernel in the setting it serves in: one launch per Transformer layer, back to back, each layer with
-    its own routes and adapters (here the first `n_layers` layers of a LLaMA-2-7B stack; 7 call sites per launch).
-    One round touches n_layers x ~27 MB of distinct adapters (more than L2), so every launch reads from HBM.
-    Reports the average launch duration inside the chain; not part of the timed step."""
-    from paper_2410_18035_b200.workload_runner import LoadedWorkload
-    from synth.workloads import scaled_workload
-    w8 = scaled_workload(step.w, n_layers=n_layers)
-    w8.gen_device = str(device)
-    lw8 = LoadedWorkload(w8, device)
-    ml = lw8.ml
-    for li in range(n_layers):
-        ml.route(li, step.H, step.cu_p, step.slots_p)      # routers differ per layer, so the routes do too
-    n = len(step.decode_ids)
-    ws = ml.alloc_group_ws(n_layers, n, step.T_d)
-    ml.group(0, n_layers, step.cu_d, step.slots_d, n, step.T_d, ws)
-    groups = [ml.groups(ws[li], n, step.T_d) for li in range(n_layers)]
-    routes = ml.route_table_read(0, w8.n_requests).numpy()
-    nbytes = sum(algorithmic_work(w8, routes[:, li], [], step.decode_ids)["decode_bytes"] for li in range(n_layers))
+def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd, device, peaks, rounds):
+    """Groups the decode rows for n_layers layers, captures one decode launch per layer in a CUDA graph (a serving
+    engine replays its decode step the same way; the Python binding needs longer per call than the kernel runs)
+    and times `rounds` replays."""
+    n = len(decode_ids)
+    ws = ml.alloc_group_ws(n_layers, n, T_d)
+    ml.group(0, n_layers, cu_d, slots_d, n, T_d, ws)
+    groups = [ml.groups(ws[li], n, T_d) for li in range(n_layers)]
+    routes = ml.route_table_read(0, w.n_requests).numpy().reshape(w.n_requests, n_layers)
+    works = [algorithmic_work(w, routes[:, li], [], decode_ids) for li in range(n_layers)]
+    nbytes = sum(x["decode_bytes"] for x in works)
+    mods = list(range(7))
 
     def one_round():
         for li in range(n_layers):
-            ml.apply_decode_multi(li, step.mods, step.Xd, step.Yd, groups[li])
+            ml.apply_decode_multi(li, mods, Xd, Yd, groups[li])
 
     for _ in range(3):
         one_round()
     torch.cuda.synchronize(device)
-    # the chain is replayed from a CUDA graph, as a serving engine replays its decode step: the Python binding
-    # needs longer per call than the kernel runs
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         one_round()
@@ -420,11 +413,52 @@ def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
     ms = e0.elapsed_time(e1) / (rounds * n_layers)
     err = ml.poll_error()
     del graph
-    lw8.close()
     gbs = nbytes / n_layers / (ms * 1e-3) / 1e9
-    return {"layers": n_layers, "us_per_layer_launch": ms * 1e3, "algorithmic_bytes_per_layer": nbytes // n_layers,
+    return {"workload": w.name, "layers": n_layers, "decode_rows": n, "rank": w.rank,
+            "distinct_adapters_per_layer": float(np.mean([x["decode_distinct_adapters"] for x in works])),
+            "us_per_layer_launch": ms * 1e3, "algorithmic_bytes_per_layer": nbytes // n_layers,
             "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
             "decode_token_layers_per_s": n / (ms * 1e-3), "device_error_flag": err}
+
+
+def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
+    """The decode kernel in the setting it serves in: one launch per Transformer layer, back to back, each layer with
+    its own routes and adapters (here the first `n_layers` layers of a LLaMA-2-7B stack; 7 call sites per launch).
+    One round touches n_layers x ~27 MB of distinct adapters (more than L2), so every launch reads from HBM.
+    Reports the average launch duration inside the chain; not part of the timed step."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth.workloads import scaled_workload
+    w8 = scaled_workload(step.w, n_layers=n_layers)
+    w8.gen_device = str(device)
+    lw8 = LoadedWorkload(w8, device)
+    for li in range(n_layers):
+        lw8.ml.route(li, step.H, step.cu_p, step.slots_p)      # routers differ per layer, so the routes do too
+    out = _timed_decode_chain(lw8.ml, w8, n_layers, step.cu_d, step.slots_d, step.T_d, step.decode_ids, step.Xd, step.Yd,
+                              device, peaks, rounds)
+    lw8.close()
+    return out
+
+
+def run_decode_13b(device, peaks, n_layers=2, rounds=20):
+    """The same chain on the LLaMA-2-13B shapes of the skewed-reuse workload (rank 32, 256 decode requests whose
+    tenants follow Zipf(1.1) over 1000 ids, routes from 256-token prompts): ~100 MB of adapters per layer, two
+    layers alternating so that a launch never finds its adapters in L2."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth import get_workload
+    from synth.workloads import scaled_workload
+    w = scaled_workload(get_workload("c4"), n_layers=n_layers)
+    w.gen_device = str(device)
+    lw = LoadedWorkload(w, device)
+    ids = list(range(w.n_requests))
+    for li in range(n_layers):
+        for i0 in range(0, len(ids), 64):
+            lw.route(li, ids[i0:i0 + 64])
+    cu_d, slots_d, T_d = lw.seq_arrays([], ids)
+    Xd = [w.module_input(0, m, T_d, 1, device) for m in range(7)]
+    Yd = [w.base_output(0, m, T_d, 1, device) for m in range(7)]
+    out = _timed_decode_chain(lw.ml, w, n_layers, cu_d, slots_d, T_d, ids, Xd, Yd, device, peaks, rounds)
+    lw.close()
+    return out
 
 
 def run_e2e(step, args, world, device, tokens_per_step):

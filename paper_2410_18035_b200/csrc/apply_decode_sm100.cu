@@ -118,10 +118,24 @@ struct DecodeArgs {
   int T;
   int rmax;        // rank rows reserved in shared memory
   int per2max;     // 16-byte column groups reserved per row of the B staging
+  int resident;    // clusters the GPU holds at once: job i + resident is the one that follows job i on its SMs
 };
+
+// L2 prefetch of `nrows` row slices of `slice_bytes` bytes each (rows `pitch` bytes apart), spread over the CTA.
+__device__ __forceinline__ void prefetch_rows(const char* base, size_t pitch, int nrows, size_t slice_bytes, int tid) {
+  if (slice_bytes == 0) return;
+  const int n_lines = (int)((slice_bytes + 127) / 128) + 1;
+  for (int idx = tid; idx < nrows * n_lines; idx += kThreads) {
+    const int j = idx / n_lines, l = idx % n_lines;
+    prefetch_l2(base + (size_t)j * pitch + min((size_t)l * 128, slice_bytes - 16));
+  }
+}
 
 // Shared memory (dynamic): [0,16) mbarrier | part[kC][kR][rmax] f32 | mine[kR][rmax] f32 | v[kR][rmax] f32 |
 //                          B[rmax][per2max] uint4
+// STAGE_B: the CTA's B slice is staged in shared memory by bulk copies.  When rank x d2 is so large that this
+// would cost occupancy, it is prefetched into L2 and read from global memory instead (STAGE_B = false).
+template <bool STAGE_B>
 __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode_bf16_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -182,10 +196,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   {
     const size_t slice_bytes = (size_t)cnt1 * 16;
     const int n_lines = cnt1 > 0 ? (int)((slice_bytes + 127) / 128) + 1 : 0;
-    for (int j = tid / kSegs; j < r; j += kRowsPerPass) {
-      const char* p = reinterpret_cast<const char*>(At + (size_t)j * d1 + (size_t)lo1 * 8);
-      for (int l = tid % kSegs; l < n_lines; l += kSegs) prefetch_l2(p + min((size_t)l * 128, slice_bytes - 16));
-    }
+    prefetch_rows(reinterpret_cast<const char*>(At) + (size_t)lo1 * 16, (size_t)d1 * 2, r, slice_bytes, tid);
     if (tid / kSegs < n) {            // kRowsPerPass >= kR: one group of kSegs threads per row of the job
       const int t = tid / kSegs;
       int row = rows[0];
@@ -204,14 +215,18 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   cluster_arrive();       // waited for right before the first remote store
   if (tid == 0) mbar_expect_tx(xbar, (uint32_t)(kC * n * r) * 4u);
 
-  if (warp == kThreads / 32 - 1) {
-    const char* Bm = static_cast<const char*>(job.B);
-    if (lane == 0) mbar_expect_tx(bar, (uint32_t)r * cnt2 * 16u);
-    __syncwarp();
-    if (cnt2 > 0) {
-      for (int i = lane; i < r; i += 32)
-        bulk_g2s(smem_u32(B_sm + (size_t)i * a.per2max), Bm + ((size_t)i * d2 + lo2 * 8) * 2, cnt2 * 16, bar);
+  const char* Bslice = static_cast<const char*>(job.B) + (size_t)lo2 * 16;      // row j at + j * d2 * 2
+  if (STAGE_B) {
+    if (warp == kThreads / 32 - 1) {
+      if (lane == 0) mbar_expect_tx(bar, (uint32_t)r * cnt2 * 16u);
+      __syncwarp();
+      if (cnt2 > 0) {
+        for (int i = lane; i < r; i += 32)
+          bulk_g2s(smem_u32(B_sm + (size_t)i * a.per2max), Bslice + (size_t)i * d2 * 2, cnt2 * 16, bar);
+      }
     }
+  } else {
+    prefetch_rows(Bslice, (size_t)d2 * 2, r, (size_t)cnt2 * 16, tid);
   }
   uint4 ypre[kYIter];
 #pragma unroll
@@ -276,12 +291,40 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
     }
   }
   __syncthreads();
+  // The job that will run on these SMs next (`resident` clusters further down the list): its record is asked for
+  // now and its A^T and B slices are prefetched into L2 while this CTA waits for the partial sums, so that its
+  // loads find L2 warm and HBM stays busy between two generations of CTAs.
+  const int next_idx = job_idx + a.resident;
+  const bool has_next = a.resident > 0 && next_idx < n_jobs && next_idx < a.lay.max_gather;
+  uint4 nj0 = make_uint4(0, 0, 0, 0), nj1 = nj0;
+  if (has_next) {
+    const uint4* np = reinterpret_cast<const uint4*>(a.ws + a.lay.gather) + (size_t)next_idx * 4;
+    nj0 = np[0];
+    nj1 = np[1];
+  }
   cluster_wait();         // every CTA of the cluster has started and initialised its barriers
   // hand this CTA's partial sums to every CTA of the cluster (slot `crank` of their `part`), one store per thread;
   // each store is counted on the receiver's barrier
   for (int idx = tid; idx < n * r * kC; idx += kThreads) {
     const int peer = idx % kC, e = idx / kC, t = e / r, j = e % r;
     st_async_f32(smem_u32(part + ((size_t)crank * kR + t) * a.rmax + j), xbar, (uint32_t)peer, mine[t * a.rmax + j]);
+  }
+  if (has_next) {
+    const char* nAt = reinterpret_cast<const char*>(((uint64_t)nj0.y << 32) | nj0.x);
+    const char* nB = reinterpret_cast<const char*>(((uint64_t)nj0.w << 32) | nj0.z);
+    const int nr = (int)nj1.x, nmod = (int)nj1.z;
+    int nsi = -1;
+#pragma unroll
+    for (int i = 0; i < kMaxSites; ++i)
+      if (i < a.sites.n && a.sites.site[i].module == nmod) nsi = i;
+    if (nsi >= 0 && nAt && nB && nr > 0 && nr <= a.rmax) {
+      const int nd1 = a.sites.site[nsi].d1, nd2 = a.sites.site[nsi].d2;
+      const int p1 = ((nd1 >> 3) + kC - 1) / kC, p2 = ((nd2 >> 3) + kC - 1) / kC;
+      const int l1 = min((int)crank * p1, nd1 >> 3), c1 = min(p1, (nd1 >> 3) - l1);
+      const int l2 = min((int)crank * p2, nd2 >> 3), c2 = min(p2, (nd2 >> 3) - l2);
+      prefetch_rows(nAt + (size_t)l1 * 16, (size_t)nd1 * 2, nr, (size_t)c1 * 16, tid);
+      prefetch_rows(nB + (size_t)l2 * 16, (size_t)nd2 * 2, nr, (size_t)c2 * 16, tid);
+    }
   }
   // all kC x n x r partial sums have landed here; the peers wait for theirs likewise, so nobody is written after it left
   if (!mbar_wait(xbar, 0)) {
@@ -300,7 +343,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   __syncthreads();
 
   // ---- expand: this CTA's d2 slice ------------------------------------------------------------
-  if (!mbar_wait(bar, 0)) {
+  if (STAGE_B && !mbar_wait(bar, 0)) {
     if (tid == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
     mbar_wait(bar, 0);    // a second, equally bounded, chance for copies still in flight before leaving
     return;
@@ -313,12 +356,32 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
       float out[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) out[i] = 0.f;
-      for (int j = 0; j < r; ++j) {
-        float bv[8];
-        unpack8(B_sm[(size_t)j * a.per2max + g], bv);
-        const float vj = v_sm[t * a.rmax + j];
+      if (STAGE_B) {
+        for (int j = 0; j < r; ++j) {
+          float bv[8];
+          unpack8(B_sm[(size_t)j * a.per2max + g], bv);
+          const float vj = v_sm[t * a.rmax + j];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) out[i] = fmaf(vj, bv[i], out[i]);
+          for (int i = 0; i < 8; ++i) out[i] = fmaf(vj, bv[i], out[i]);
+        }
+      } else {
+        // rank rows in batches of eight: independent loads (L2 hits) first, then the multiply-adds in rank order
+        for (int j0 = 0; j0 < r; j0 += 8) {
+          uint4 bq[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            bq[u] = ldg_stream(Bslice + (size_t)min(j0 + u, r - 1) * d2 * 2 + (size_t)g * 16);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            if (j0 + u < r) {
+              float bv[8];
+              unpack8(bq[u], bv);
+              const float vj = v_sm[t * a.rmax + j0 + u];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) out[i] = fmaf(vj, bv[i], out[i]);
+            }
+          }
+        }
       }
       float yv[8];
       unpack8(ypre[it], yv);
@@ -353,14 +416,22 @@ milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySi
   }
   if (kR * per2 > kYIter * kThreads) return MILORA_E_SHAPE;
   a.per2max = per2;
-  size_t smem = 16 + (size_t)(kC + 2) * kR * a.rmax * sizeof(float) + (size_t)a.rmax * per2 * 16;
+  const size_t smem_base = 16 + (size_t)(kC + 2) * kR * a.rmax * sizeof(float);
+  size_t smem = smem_base + (size_t)a.rmax * per2 * 16;
+  // staging B pays only while four CTAs still fit on an SM (four is what the register budget allows)
+  const bool stage_b = (smem + 1024) * 4 <= 227 * 1024;
+  if (!stage_b) smem = smem_base;
   if (smem > 200 * 1024) return MILORA_E_SHAPE;
+  auto kernel = stage_b ? decode_bf16_kernel<true> : decode_bf16_kernel<false>;
   if (smem > 48 * 1024) {
-    MILORA_CUDA(ctx, cudaFuncSetAttribute(decode_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
+  int per_sm = 0;
+  MILORA_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem));
+  a.resident = ctx->sm_count * per_sm / kC;
   size_t grid = (size_t)a.lay.max_gather * kC;
   if (grid > 0x7fffffffull) return MILORA_E_CAPACITY;
-  MILORA_CUDA(ctx, launch_pdl(decode_bf16_kernel, dim3((unsigned)grid), dim3(kThreads), smem, s, a));
+  MILORA_CUDA(ctx, launch_pdl(kernel, dim3((unsigned)grid), dim3(kThreads), smem, s, a));
   return MILORA_OK;
 }
 
