@@ -26,7 +26,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kRows = 64;
+constexpr int kRowsMax = 128;   // rows of a chunk: 64 or 128, chosen per call so that one round of units fills the GPU
 
 template <typename T> struct VecOf;
 template <> struct VecOf<float> {
@@ -151,7 +151,7 @@ struct RouteArgs {
   float* partial;     // [total_chunks][d]
   float* stats;       // [total_chunks][2]  (self-attention pooler: chunk max, chunk sum of exp)
   int32_t* sched;     // next dynamic unit; zero on entry, put back to zero by pass 2
-  int layer, P, d, n_strips;
+  int layer, P, d, n_strips, rows;
 };
 
 // Router entry of prompt p, or nullptr when its slot is closed / its tenant has no router at this layer.
@@ -176,13 +176,16 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
   int32_t* pool_sm = sm_i + (a.P + 1);
   __shared__ int32_t carry;
   __shared__ int32_t wsum[kWarps];
-  __shared__ float u_all[kWarps][kRows];
+  __shared__ float u_all[kWarps][kRowsMax];
+  const int kRows = a.rows;
   constexpr int V = VecOf<T>::N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = a.d;
   const T* H = static_cast<const T*>(a.H);
-  pdl_launch_dependents();
+  // Pass 2 reads the prompt lengths, slots and router table before its own wait; it may do so only once
+  // everything ahead of this kernel has completed, so the trigger comes after the wait here.
   pdl_wait();
+  pdl_launch_dependents();
 
   // per-CTA prefix over prompts: chunks per prompt (from the lengths) and the pooler of each prompt
   if (tid == 0) carry = 0;
@@ -306,12 +309,14 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
 template <typename T>
 __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   constexpr int V = VecOf<T>::N;
+  const int kRows = a.rows;
   __shared__ float red[MILORA_NMOD * kWarps];
   __shared__ int32_t wsum[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int p = blockIdx.x, d = a.d;
+  // Launched behind pass 1, whose CTAs trigger only after their own wait: lengths, slots and tables are final
+  // when this CTA starts, so its look-ups overlap the tail of pass 1.  Only the partial sums need pdl_wait().
   pdl_launch_dependents();
-  pdl_wait();
   // first scratch row of this prompt = number of chunks of the prompts before it
   int mine = 0;
   for (int q = tid; q < p; q += kThreads) {
@@ -330,6 +335,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   const RouterEntry* rp = router_of(a, p, &slot);
   if (!rp || n_chunks == 0) {
     // closed slot, no router for this tenant at this layer, or an empty prompt: the request stays "not routed"
+    pdl_wait();
     if (tid == 0) {
       if (slot >= 0 && slot < a.tab.max_requests) {
         for (int j = 0; j < a.tab.top_k; ++j)
@@ -347,6 +353,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   if (pool == MILORA_POOL_LAST) { chunk0 += n_chunks - 1; n_chunks = 1; }   // only the chunk with the last row counts
   const float* part0 = a.partial + (size_t)chunk0 * d;
   const float* st0 = a.stats + 2 * (size_t)chunk0;
+  pdl_wait();                                   // the partial sums of pass 1
   float gmax = -FLT_MAX, denom = 1.f;
   if (sa) {
     for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, st0[2 * c]);
@@ -471,7 +478,7 @@ milora_status transpose(milora_ctx* ctx, const void* in, void* out, int rows, in
 }
 
 struct RoutePlan {
-  int n_strips;
+  int n_strips, rows;
   size_t max_chunks, scratch_floats, max_units;
 };
 
@@ -480,6 +487,12 @@ RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
   const int d = ctx->desc.d_model;
   const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
   pl.n_strips = (d + 32 * V - 1) / (32 * V);
+  // 128-row chunks when that still gives every resident warp about one unit (a warp then streams 64 KB without
+  // coming back to the queue); 64-row chunks for smaller batches, which need the parallelism
+  const size_t warp_slots = (size_t)ctx->sm_count * 5 * kWarps;
+  const size_t units128 = ((size_t)T_total / 128 + P) * pl.n_strips;
+  pl.rows = units128 * 10 >= warp_slots * 6 ? 128 : 64;
+  const int kRows = pl.rows;
   pl.max_chunks = (size_t)T_total / kRows + P;
   pl.scratch_floats = pl.max_chunks * d + 2 * pl.max_chunks;
   pl.max_units = pl.max_chunks * pl.n_strips;
@@ -497,7 +510,7 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   a.partial = scratch;
   a.stats = scratch + pl.max_chunks * ctx->desc.d_model;
   a.sched = sched;
-  a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_strips = pl.n_strips;
+  a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_strips = pl.n_strips; a.rows = pl.rows;
   const size_t smem = (size_t)(2 * P + 1) * sizeof(int32_t);
   const bool f32 = ctx->desc.dtype == MILORA_F32;
   // pass 1: one wave of resident CTAs (a warp's first unit is assigned by index, so every CTA must start at once)
@@ -563,8 +576,11 @@ milora_status launch_route_static(milora_ctx* ctx, int layer, const void* H, con
   constexpr int kMaxDevices = 64;
   static float* scratch_of_device[kMaxDevices] = {nullptr};
   const RoutePlan pl = plan_route(ctx, P, T_total);
-  // the scheduling word sits right behind the partial area
-  if (pl.scratch_floats > kStaticPartialFloats || (size_t)P > kStaticCounters) return MILORA_E_CAPACITY;
+  // the scheduling word sits right behind the partial area.  The documented limit is the need with 64-row
+  // chunks, whatever chunk size this call ends up using.
+  const size_t documented_need = ((size_t)T_total / 64 + P) * ((size_t)ctx->desc.d_model + 2);
+  if (documented_need > kStaticPartialFloats || pl.scratch_floats > kStaticPartialFloats || (size_t)P > kStaticCounters)
+    return MILORA_E_CAPACITY;
   int dev = -1;
   MILORA_CUDA(ctx, cudaGetDevice(&dev));
   if (dev != ctx->device) return MILORA_E_STATE;     // the context's device must be current
