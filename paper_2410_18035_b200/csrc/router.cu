@@ -114,7 +114,7 @@ __device__ __forceinline__ void unpack16(const uint4& q, float (&v)[8]) {
 // Column reduction over `nr` rows for the 16-byte column group at `col` (row stride d): sum, max, or sum
 // weighted by w[t].  Rows are fetched in batches of kDepth independent 128-bit loads and combined in order.
 enum { kRedSum = 0, kRedMax = 1, kRedWeighted = 2 };
-constexpr int kDepth = 8;
+constexpr int kDepth = 16;
 template <typename T, int MODE>
 __device__ __forceinline__ void reduce_rows(const T* col, int d, int nr, const float* w, float (&acc)[VecOf<T>::N]) {
   constexpr int V = VecOf<T>::N;
