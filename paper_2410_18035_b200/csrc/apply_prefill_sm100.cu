@@ -27,7 +27,7 @@ namespace {
 using namespace ptx;
 
 constexpr int kKSplit = 4;            // k-slices of the shrink
-constexpr int kNSplit = 4;            // n-slices of the expand
+constexpr int kNSplit = 8;            // n-slices of the expand
 constexpr int kBK = 64;               // k elements per shrink stage (128 bytes: one swizzle row)
 constexpr int kBN = 128;              // y columns per expand chunk
 constexpr int kRPadMax = 64;          // largest padded rank this path takes
