@@ -140,15 +140,16 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t crank = cluster_ctarank();
-  const int job_idx = blockIdx.x / kC;
   pdl_launch_dependents();
   pdl_wait();
-  if (job_idx >= a.lay.max_gather) return;                              // same decision in the whole cluster
-  // the job record is fetched together with the job count (the list has max_gather slots, so the read is in bounds)
+  if ((int)(blockIdx.x / kC) >= a.lay.max_gather) return;               // same decision in the whole cluster
+  // The list is ordered by module, and the modules with the most bytes (gate, up, down) come last: clusters take
+  // the jobs from the end of the list, so that the longest jobs start first and the short ones fill the tail.
+  const int n_jobs = a.ws[a.lay.header + H_NGATHER];
+  const int job_idx = n_jobs - 1 - (int)(blockIdx.x / kC);
+  if (job_idx < 0) return;
   const uint4* jp = reinterpret_cast<const uint4*>(a.ws + a.lay.gather) + (size_t)job_idx * 4;
   const uint4 j0 = jp[0], j1 = jp[1], j2 = jp[2], j3 = jp[3];
-  const int n_jobs = a.ws[a.lay.header + H_NGATHER];
-  if (job_idx >= n_jobs) return;
   GatherJob job;
   {
     uint4* dst = reinterpret_cast<uint4*>(&job);
@@ -294,8 +295,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
   // The job that will run on these SMs next (`resident` clusters further down the list): its record is asked for
   // now and its A^T and B slices are prefetched into L2 while this CTA waits for the partial sums, so that its
   // loads find L2 warm and HBM stays busy between two generations of CTAs.
-  const int next_idx = job_idx + a.resident;
-  const bool has_next = a.resident > 0 && next_idx < n_jobs && next_idx < a.lay.max_gather;
+  const int next_idx = job_idx - a.resident;
+  const bool has_next = a.resident > 0 && next_idx >= 0;
   uint4 nj0 = make_uint4(0, 0, 0, 0), nj1 = nj0;
   if (has_next) {
     const uint4* np = reinterpret_cast<const uint4*>(a.ws + a.lay.gather) + (size_t)next_idx * 4;
