@@ -271,6 +271,48 @@ def test_fused_projection_matches_oracle(d, d_ff, d_kv, r, k):
     lw.close()
 
 
+def test_fused_projection_refuses_what_it_cannot_run():
+    """Shapes and dtypes outside the tensor-core kernel's limits are refused before anything is launched."""
+    from paper_2410_18035_b200 import Milora, MiloraError
+    def call(ml, module, T, dtype):
+        d1, d2 = ml.module_dims(module)
+        X = torch.zeros((T, d1), dtype=dtype, device="cuda")
+        Wt = torch.zeros((d2, d1), dtype=dtype, device="cuda")
+        Y = torch.full((T, d2), 7.0, dtype=dtype, device="cuda")
+        slots = torch.zeros(1, dtype=torch.int32, device="cuda")
+        cu = torch.tensor([0, T], dtype=torch.int32, device="cuda")
+        ws = ml.alloc_group_ws(1, 1, T)
+        ml.request_open(0, 0) if not getattr(ml, "_opened", False) else None
+        ml._opened = True
+        ml.group(0, 1, cu, slots, 1, T, ws)
+        ml.linear_prefill(0, module, X, Wt, Y, ml.groups(ws[0], 1, T))
+        torch.cuda.synchronize()
+        return Y
+    ml = Milora(1, 256, 768, 256, "f32", 8, 2, 2)                 # fp32 context
+    with pytest.raises(MiloraError) as e:
+        call(ml, 0, 256, torch.float32)
+    assert e.value.status == 2
+    ml.close()
+    ml = Milora(1, 512, 1408, 128, "bf16", 16, 2, 2)              # d_ff and d_kv are not multiples of 256
+    for module in (1, 4):
+        with pytest.raises(MiloraError) as e:
+            call(ml, module, 256, torch.bfloat16)
+        assert e.value.status == 2
+    with pytest.raises(MiloraError) as e:                         # fewer rows than one tile
+        call(ml, 0, 64, torch.bfloat16)
+    assert e.value.status == 2
+    # a step without any routed adapter is a plain projection: x = 0 gives y = 0 on every row
+    Y = call(ml, 0, 300, torch.bfloat16)
+    assert float(Y.float().abs().max()) == 0.0
+    assert ml.poll_error() == 0
+    ml.close()
+    ml = Milora(1, 512, 1536, 256, "bf16", 64, 2, 2)              # rank limit of the fused kernel
+    with pytest.raises(MiloraError) as e:
+        call(ml, 0, 256, torch.bfloat16)
+    assert e.value.status == 2
+    ml.close()
+
+
 def test_tenant_without_adapter_is_excluded():
     base = get_workload("c1")
     w = scaled_workload(base, n_tenants=6)
