@@ -68,7 +68,8 @@ milora_group_layout_t group_layout(int n_seq, int T, int top_k) {
   L.max_tiles = (int)(TT / kTileRows + n_ent);
   L.tiles = o; o += (size_t)L.max_tiles * kJobInts;
   L.gather_rows = o; o += round4(2 * TT);      // row and sequence of every gathered (token, module) pair
-  L.max_gather = (int)(TT / kGatherRows + n_ent + 1);
+  // gathered rows belong to sequences shorter than kLongSeq, so there are at most (kLongSeq - 1) per entry
+  L.max_gather = (int)(std::min(TT, (size_t)(kLongSeq - 1) * n_ent) / kGatherRows + n_ent + 1);
   L.gather = o; o += (size_t)L.max_gather * kJobInts;
   L.total = round4(o);
   return L;
