@@ -313,6 +313,63 @@ def test_fused_projection_refuses_what_it_cannot_run():
     ml.close()
 
 
+def test_back_to_back_launches_equal_serialised_ones_bit_for_bit():
+    """Every kernel may start while the one before it is still draining (programmatic dependent launch) and takes
+    its work from device-side lists.  The results must not depend on that: the whole step enqueued back to back,
+    twice, and once with a device synchronisation after every call give bit-identical routes, logits and outputs."""
+    base = get_workload("c1")
+    lens = np.array([700, 130, 257, 64, 33, 512, 31, 7] + [1] * 24, dtype=np.int32)
+    n = len(lens)
+    tenants = (np.arange(n) % 5).astype(np.int32)
+    w = scaled_workload(base, name="pdl", dtype="bf16", d_model=1024, d_ff=2816, d_kv=256, rank=16, n_tenants=5,
+                        request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(8), decode_ids=np.arange(8, n),
+                        has_base_weights=False, n_layers=1)
+    w.gen_device = "cuda"
+    lw = _loaded(w)
+    ml = lw.ml
+    prefill, decode = list(range(8)), list(range(8, n))
+    lw.route(0, decode)                                   # the running requests were routed earlier
+    H = w.hidden_batch(0, prefill, "cuda")
+    cu_p = torch.from_numpy(w.cu_seqlens(prefill)).cuda()
+    slots_p = torch.tensor(prefill, dtype=torch.int32, device="cuda")
+    cu, slots, T = lw.seq_arrays(prefill, decode)
+    n_seq = slots.numel()
+    Xs = [w.module_input(0, m, T, 1, "cuda") for m in range(7)]
+    Ybs = [w.base_output(0, m, T, 1, "cuda") for m in range(7)]
+    mods = list(range(7))
+
+    def step(sync):
+        wait = torch.cuda.synchronize if sync else (lambda: None)
+        logits = torch.zeros((len(prefill), 7), dtype=torch.float32, device="cuda")
+        ws = ml.alloc_group_ws(1, n_seq, T)
+        Ys = [y.clone() for y in Ybs]
+        torch.cuda.synchronize()
+        ml.route(0, H, cu_p, slots_p, logits); wait()
+        ml.group(0, 1, cu, slots, n_seq, T, ws); wait()
+        g = ml.groups(ws[0], n_seq, T)
+        ml.apply_prefill_multi(0, mods, Xs, Ys, g); wait()
+        ml.apply_decode_multi(0, mods, Xs, Ys, g); wait()
+        torch.cuda.synchronize()
+        return ml.route_table_read(0, n).numpy().copy(), logits.cpu(), ws.cpu(), [y.cpu() for y in Ys]
+
+    ref = step(sync=True)
+    for _ in range(2):
+        got = step(sync=False)
+        assert np.array_equal(got[0], ref[0])
+        assert torch.equal(got[1], ref[1])
+        lay = ml.group_layout(n_seq, T)
+        hdr = ref[2][0, lay.header:lay.header + 5].tolist()
+        used = [(lay.header, 16), (lay.seg_key, hdr[0]), (lay.seg_offset, hdr[0] + 1), (lay.perm, hdr[2]),
+                (lay.tiles, 16 * hdr[3]), (lay.gather, 16 * hdr[4])]
+        for off, cnt in used:
+            assert torch.equal(got[2][0, off:off + cnt], ref[2][0, off:off + cnt])
+        for m in range(7):
+            assert torch.equal(got[3][m], ref[3][m]), f"module {m}: output depends on launch overlap"
+    assert (ref[3][0] != Ybs[0].cpu()).any()
+    assert ml.poll_error() == 0
+    lw.close()
+
+
 def test_tenant_without_adapter_is_excluded():
     base = get_workload("c1")
     w = scaled_workload(base, n_tenants=6)
