@@ -92,13 +92,16 @@ __device__ __forceinline__ uint32_t tmem_cols_for(int rp) { return rp <= 32 ? 32
 __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __grid_constant__ ShrinkArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tile_idx = blockIdx.x / kKSplit, ks = blockIdx.x % kKSplit;
+  const int ks = blockIdx.x % kKSplit;
   // The expand kernel starts its copies of y and B before its own wait; it may do so only once
   // everything ahead of this kernel has completed, so the trigger comes after the wait here.
   pdl_wait();
   pdl_launch_dependents();
-  const int n_tiles = a.ws[a.lay.header + H_NTILES];
-  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) return;
+  // The tile list is ordered by module and the modules with the longest rows (gate, up, down) come last: CTAs
+  // take the list from its end, so that the long tiles start first and the short ones fill the tail.
+  const int n_tiles = min(a.ws[a.lay.header + H_NTILES], a.lay.max_tiles);
+  const int tile_idx = n_tiles - 1 - (int)(blockIdx.x / kKSplit);
+  if (tile_idx < 0) return;
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
   const int si = find_site(a.sites, job.module);
   if (si < 0) return;
@@ -217,12 +220,13 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* d) {
 __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __grid_constant__ ExpandArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tile_idx = blockIdx.x / kNSplit, ns = blockIdx.x % kNSplit;
+  const int ns = blockIdx.x % kNSplit;
   // Launched behind the shrink kernel, whose CTAs trigger only after their own wait: the job list, y and
   // the B images are final when this CTA starts.  Only the partial products of the shrink need pdl_wait().
   pdl_launch_dependents();
-  const int n_tiles = a.ws[a.lay.header + H_NTILES];
-  if (tile_idx >= n_tiles || tile_idx >= a.lay.max_tiles) { pdl_wait(); return; }
+  const int n_tiles = min(a.ws[a.lay.header + H_NTILES], a.lay.max_tiles);
+  const int tile_idx = n_tiles - 1 - (int)(blockIdx.x / kNSplit);       // longest tiles first, as in the shrink kernel
+  if (tile_idx < 0) { pdl_wait(); return; }
   const TileJob job = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles)[tile_idx];
   const int si = find_site(a.sites, job.module);
   if (si < 0) { pdl_wait(); return; }
