@@ -105,6 +105,7 @@ def test_config2_full_size_bench_configuration():
     _check_step(lw, 0, ids, [], table, tag=0, rng=rng)          # prefill rows (dense tiles)
     _check_step(lw, 0, [], ids, table, tag=1, rng=rng)          # decode rows (gathered)
     _check_step(lw, 0, ids[:8], ids[8:], table, tag=2, rng=rng, multi=False)   # mixed, per-site calls
+    _check_step(lw, 0, ids, ids, table, tag=3, rng=rng)         # all prompts and all decode rows as one batch
     lw.close()
 
 
