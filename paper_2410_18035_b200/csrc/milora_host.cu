@@ -169,6 +169,8 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
   ctx->d_vscratch = nullptr; ctx->vscratch_floats = 0;
   ctx->d_lin = nullptr; ctx->lin_bytes = 0;
+  ctx->copy_stream = nullptr; ctx->ev_done = nullptr; ctx->copy_ready = false;
+  for (int m = 0; m < MILORA_NMOD; ++m) ctx->ev_site[m] = nullptr;
   ctx->n_counters = 0;
   milora_status st = MILORA_OK;
   auto fail = [&](milora_status s) { milora_destroy(ctx); return s; };
@@ -229,6 +231,10 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_counters);
   cudaFree(ctx->d_vscratch);
   cudaFree(ctx->d_lin);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
+  for (int m = 0; m < MILORA_NMOD; ++m)
+    if (ctx->ev_site[m]) cudaEventDestroy(ctx->ev_site[m]);
   ctx->arena.release();
   delete ctx;
   return MILORA_OK;
@@ -639,42 +645,48 @@ milora_status milora_step_host(milora_ctx* ctx, const milora_host_step* step, vo
     MILORA_CUDA(ctx, h2d(pl.cu_s, step->cu_seq_host, (size_t)(step->n_seq + 1) * 4));
     MILORA_CUDA(ctx, h2d(pl.slot_s, step->seq_slot_host, (size_t)step->n_seq * 4));
   }
-  int modules[MILORA_NMOD], n_sites = 0;
-  const void* X[MILORA_NMOD];
-  void* Y[MILORA_NMOD];
-  for (int m = 0; m < MILORA_NMOD; ++m) {
-    if (!step->X_host[m]) continue;
-    int d1, d2;
-    module_dims(ctx->desc, m, &d1, &d2);
-    MILORA_CUDA(ctx, h2d(pl.X[m], step->X_host[m], (size_t)step->T * d1 * e));
-    MILORA_CUDA(ctx, h2d(pl.Y[m], step->Y_host[m], (size_t)step->T * d2 * e));
-    modules[n_sites] = m;
-    X[n_sites] = w + pl.X[m];
-    Y[n_sites] = w + pl.Y[m];
-    ++n_sites;
-  }
   // the path
   if (step->n_prompts > 0 && pl.T_p > 0) {
     st = milora_route(ctx, step->layer, w + pl.H, reinterpret_cast<const int32_t*>(w + pl.cu_p),
                       reinterpret_cast<const int32_t*>(w + pl.slot_p), step->n_prompts, pl.T_p, nullptr, nullptr, stream);
     if (st != MILORA_OK) return st;
   }
-  if (step->n_seq > 0 && step->T > 0 && n_sites > 0) {
+  bool any_site = false;
+  for (int m = 0; m < MILORA_NMOD; ++m) any_site = any_site || step->X_host[m];
+  if (step->n_seq > 0 && step->T > 0 && any_site) {
+    // The transfers dominate a step from host memory, and the link carries both directions at once: the modules
+    // are processed one after the other, and the copy of module m's output back to the host runs on a second
+    // stream while module m + 1 is being uploaded.
+    if (!ctx->copy_ready) {
+      MILORA_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+      MILORA_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming));
+      for (int m = 0; m < MILORA_NMOD; ++m)
+        MILORA_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_site[m], cudaEventDisableTiming));
+      ctx->copy_ready = true;
+    }
     int32_t* ws = reinterpret_cast<int32_t*>(w + pl.ws);
     st = milora_group(ctx, step->layer, 1, reinterpret_cast<const int32_t*>(w + pl.cu_s),
                       reinterpret_cast<const int32_t*>(w + pl.slot_s), step->n_seq, step->T, ws, pl.ws_stride, stream);
     if (st != MILORA_OK) return st;
     milora_groups g{ws, step->n_seq, step->T};
-    st = milora_apply_prefill_multi(ctx, step->layer, n_sites, modules, X, Y, &g, stream);
-    if (st != MILORA_OK) return st;
-    st = milora_apply_decode_multi(ctx, step->layer, n_sites, modules, X, Y, &g, stream);
-    if (st != MILORA_OK) return st;
-    // outputs
-    for (int i = 0; i < n_sites; ++i) {
+    for (int m = 0; m < MILORA_NMOD; ++m) {
+      if (!step->X_host[m]) continue;
       int d1, d2;
-      module_dims(ctx->desc, modules[i], &d1, &d2);
-      MILORA_CUDA(ctx, cudaMemcpyAsync(step->Y_host[modules[i]], Y[i], (size_t)step->T * d2 * e, cudaMemcpyDeviceToHost, s));
+      module_dims(ctx->desc, m, &d1, &d2);
+      const size_t y_bytes = (size_t)step->T * d2 * e;
+      MILORA_CUDA(ctx, h2d(pl.X[m], step->X_host[m], (size_t)step->T * d1 * e));
+      MILORA_CUDA(ctx, h2d(pl.Y[m], step->Y_host[m], y_bytes));
+      st = milora_apply_prefill(ctx, step->layer, m, w + pl.X[m], w + pl.Y[m], &g, stream);
+      if (st != MILORA_OK) return st;
+      st = milora_apply_decode(ctx, step->layer, m, w + pl.X[m], w + pl.Y[m], &g, stream);
+      if (st != MILORA_OK) return st;
+      MILORA_CUDA(ctx, cudaEventRecord(ctx->ev_site[m], s));
+      MILORA_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_site[m], 0));
+      MILORA_CUDA(ctx, cudaMemcpyAsync(step->Y_host[m], w + pl.Y[m], y_bytes, cudaMemcpyDeviceToHost, ctx->copy_stream));
     }
+    // the caller's stream is done only when every output has arrived (and the workspace may be reused)
+    MILORA_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->copy_stream));
+    MILORA_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_done, 0));
   }
   return MILORA_OK;
 }

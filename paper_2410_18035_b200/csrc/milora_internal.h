@@ -123,6 +123,10 @@ struct milora_ctx {
   size_t vscratch_floats;
   void* d_lin;                                  // fused projection: V piece images and per-row-block piece lists
   size_t lin_bytes;
+  cudaStream_t copy_stream;                     // milora_step_host: device-to-host copies run beside the uploads
+  cudaEvent_t ev_site[MILORA_NMOD];             // "module m is done" / "all copies back are done"
+  cudaEvent_t ev_done;
+  bool copy_ready;
   milora::Arena arena;
   std::string cuda_error;
 };
