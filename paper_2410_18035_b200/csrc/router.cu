@@ -68,8 +68,8 @@ __device__ inline float activate(float h, const RouterEntry& r) {
 }
 
 // Sum over the block in a fixed order: lanes by xor-shuffle, then every thread adds the warp totals in order.
-template <int NV>
-__device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][kWarps] */) {
+template <int NV, int NW>
+__device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][NW] */) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
@@ -79,14 +79,14 @@ __device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][kWarps] */)
   __syncthreads();
   if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) smem[i * kWarps + warp] = v[i];
+    for (int i = 0; i < NV; ++i) smem[i * NW + warp] = v[i];
   }
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) s += smem[i * kWarps + w];
+    for (int w = 0; w < NW; ++w) s += smem[i * NW + w];
     v[i] = s;
   }
 }
@@ -306,12 +306,16 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
 }
 
 // ---- pass 2: one CTA per prompt combines the partials in chunk order and routes -----------------------
+// 512 threads: at d = 4096 (bf16) every thread owns one 16-byte column group, so the chain a warp has to run
+// after pass 1 has finished (fetch the partial sums, eight accurate tanh, 56 multiply-adds) is gone through once.
+constexpr int kFinThreads = 512;
+constexpr int kFinWarps = kFinThreads / 32;
 template <typename T>
-__global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
+__global__ void __launch_bounds__(kFinThreads) route_finalize_kernel(RouteArgs a) {
   constexpr int V = VecOf<T>::N;
   const int kRows = a.rows;
-  __shared__ float red[MILORA_NMOD * kWarps];
-  __shared__ int32_t wsum[kWarps];
+  __shared__ float red[MILORA_NMOD * kFinWarps];
+  __shared__ int32_t wsum[kFinWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int p = blockIdx.x, d = a.d;
   // Launched behind pass 1, whose CTAs trigger only after their own wait: lengths, slots and tables are final
@@ -319,7 +323,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   pdl_launch_dependents();
   // first scratch row of this prompt = number of chunks of the prompts before it
   int mine = 0;
-  for (int q = tid; q < p; q += kThreads) {
+  for (int q = tid; q < p; q += kFinThreads) {
     const int n_q = a.cu[q + 1] - a.cu[q];
     if (n_q > 0) mine += (n_q + kRows - 1) / kRows;
   }
@@ -328,7 +332,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   if (lane == 0) wsum[warp] = mine;
   __syncthreads();
   int chunk0 = 0;
-  for (int w = 0; w < kWarps; ++w) chunk0 += wsum[w];
+  for (int w = 0; w < kFinWarps; ++w) chunk0 += wsum[w];
   const int n_p = a.cu[p + 1] - a.cu[p];
   int n_chunks = n_p > 0 ? (n_p + kRows - 1) / kRows : 0;
   int slot;
@@ -364,7 +368,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
   float z[MILORA_NMOD];
 #pragma unroll
   for (int j = 0; j < MILORA_NMOD; ++j) z[j] = 0.f;
-  for (int c0 = tid * V; c0 < d; c0 += kThreads * V) {
+  for (int c0 = tid * V; c0 < d; c0 += kFinThreads * V) {
     float h[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) h[i] = pool == MILORA_POOL_MAX ? -FLT_MAX : 0.f;
@@ -414,7 +418,7 @@ __global__ void __launch_bounds__(kThreads) route_finalize_kernel(RouteArgs a) {
       for (int i = 0; i < V; ++i) z[j] = fmaf(h[i], wv[i], z[j]);
     }
   }
-  block_sum<MILORA_NMOD>(z, red);
+  block_sum<MILORA_NMOD, kFinWarps>(z, red);
   if (tid == 0) {
     float zmax = -FLT_MAX;
 #pragma unroll
@@ -523,8 +527,8 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   if (f32) MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<float>, dim3(grid), dim3(kThreads), smem, s, a));
   else MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), smem, s, a));
   // pass 2: one CTA per prompt
-  if (f32) MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<float>, dim3(P), dim3(kThreads), 0, s, a));
-  else MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<__nv_bfloat16>, dim3(P), dim3(kThreads), 0, s, a));
+  if (f32) MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<float>, dim3(P), dim3(kFinThreads), 0, s, a));
+  else MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<__nv_bfloat16>, dim3(P), dim3(kFinThreads), 0, s, a));
   return MILORA_OK;
 }
 
