@@ -473,6 +473,22 @@ def test_host_validation_reports_errors_before_launch():
     ml.route_table_write(2, [[3, -1]])
     assert ml.route_table_read(2, 1).tolist() == [[3, -1]]
     ml.close()
+    # invalid k or weighting mode; with k selected modules per sequence a grouping call takes 4096 / k sequences
+    for kw in ({"top_k": 8}, {"top_k": -1}, {"gate": 5}):
+        with pytest.raises(MiloraError) as e:
+            Milora(1, 256, 688, 256, "f32", 8, 4, 4, **kw)
+        assert e.value.status == 1
+    ml = Milora(1, 256, 688, 256, "f32", 8, 4, 4, top_k=3)
+    with pytest.raises(MiloraError) as e:
+        ml.group_layout(2000, 2000)
+    assert e.value.status == 5
+    assert ml.group_layout(1365, 1365).total > 0
+    slots = torch.zeros(2000, dtype=torch.int32, device="cuda")
+    ws = torch.zeros((1, 1 << 20), dtype=torch.int32, device="cuda")
+    with pytest.raises(MiloraError) as e:
+        ml.group(0, 1, None, slots, 2000, 2000, ws)
+    assert e.value.status == 5
+    ml.close()
 
 
 def test_step_from_host_buffers_matches_oracle():
