@@ -215,9 +215,10 @@ class Step:
         rec(3)
         ml.group(0, 1, self.cu_d, self.slots_d, len(self.decode_ids), self.T_d, self.ws_d)
         rec(4)
-        ml.apply_decode_multi(0, self.mods, self.Xd, self.Yd, self.g_d)      # all 7 call sites, one launch
+        ml.apply_decode_multi(0, self.mods, self.Xd, self.Yd, self.g_d)      # all 7 call sites, one call
         rec(5)
-        self.n_launches = 2 + 1 + 2 + 1 + 1
+        self.decode_launches = 2 if ml.decode_path_for(len(self.decode_ids), self.T_d) == 2 else 1
+        self.n_launches = 2 + 1 + 2 + 1 + self.decode_launches
         return self.n_launches
 
 
@@ -246,6 +247,12 @@ def run_ours(args, rank, world, device):
     for _ in range(max(args.warmup, 3)):
         step.run()
     barrier()
+    if args.only_chains:
+        if rank == 0:
+            sampler.stop()
+            print(json.dumps({"decode_stack": run_decode_stack(step, device, load_peaks()),
+                              "decode_stack_13b_zipf": run_decode_13b(device, load_peaks())}))
+        return None
     routes = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0]
     work = algorithmic_work(w, routes, step.prefill_ids, step.decode_ids)
     barrier()
@@ -398,29 +405,45 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
         for li in range(n_layers):
             ml.apply_decode_multi(li, mods, Xd, Yd, groups[li])
 
-    for _ in range(3):
-        one_round()
-    torch.cuda.synchronize(device)
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        one_round()
-    graph.replay()
-    torch.cuda.synchronize(device)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(rounds):
+    def timed():
+        for _ in range(3):
+            one_round()
+        torch.cuda.synchronize(device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_round()
         graph.replay()
-    e1.record()
-    torch.cuda.synchronize(device)
-    ms = e0.elapsed_time(e1) / (rounds * n_layers)
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(rounds):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize(device)
+        del graph
+        return e0.elapsed_time(e1) / (rounds * n_layers)
+
+    def figures(ms):
+        gbs = nbytes / n_layers / (ms * 1e-3) / 1e9
+        return {"us_per_layer": ms * 1e3, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "decode_token_layers_per_s": n / (ms * 1e-3)}
+
+    # both kernel sets on the same chain, then the library's own choice (the figures reported at the top level)
+    by_path = {}
+    for path in ("cluster", "split"):
+        ml.set_decode_path(path)
+        by_path[path] = figures(timed())
+    ml.set_decode_path("auto")
+    ms = timed()
     err = ml.poll_error()
-    del graph
-    gbs = nbytes / n_layers / (ms * 1e-3) / 1e9
+    top = figures(ms)
     return {"workload": w.name, "layers": n_layers, "decode_rows": n, "rank": w.rank,
             "distinct_adapters_per_layer": float(np.mean([x["decode_distinct_adapters"] for x in works])),
-            "us_per_layer_launch": ms * 1e3, "algorithmic_bytes_per_layer": nbytes // n_layers,
-            "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
-            "decode_token_layers_per_s": n / (ms * 1e-3), "device_error_flag": err}
+            "us_per_layer_launch": top["us_per_layer"], "algorithmic_bytes_per_layer": nbytes // n_layers,
+            "gbs": top["gbs"], "frac_of_measured_hbm": top["frac_of_measured_hbm"],
+            "frac_of_8TBs_nominal": top["frac_of_8TBs_nominal"],
+            "decode_token_layers_per_s": top["decode_token_layers_per_s"], "device_error_flag": err,
+            "by_decode_path": by_path}
 
 
 def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
@@ -636,6 +659,8 @@ def main():
     ap.add_argument("--config", default="c2")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-fused", action="store_true", help="leave out the fused-projection timing")
+    ap.add_argument("--only-chains", action="store_true",
+                    help="print only the decode-chain figures (both decode kernel sets) and exit; not a bench line")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle timing")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -232,6 +232,26 @@ milora_status milora_apply_decode(milora_ctx* ctx, int layer, int module, const 
 milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
                                    const milora_groups* groups, void* stream);
 
+/* Which kernels milora_apply_decode uses in a bf16 context (both compute the same Eq. 1; results agree to
+ * rounding of the fp32 sums, and each is deterministic from call to call):
+ *   MILORA_DECODE_CLUSTER  one launch; a cluster of eight CTAs per job exchanges partial sums of x W^A through
+ *                          distributed shared memory.  Shortest latency when the step has few jobs.
+ *   MILORA_DECODE_SPLIT    two launches (x W^A, then the product with W^B added into y), both plain streams over
+ *                          equally sized units handed out by a counter, with the contractions on mma.sync tiles;
+ *                          the r values per row in between go through a scratch buffer of the context (the
+ *                          second launch takes them as bf16 value + bf16 remainder, i.e. to 2^-17), which the first call (and any call with a larger
+ *                          batch than every earlier one) grows with cudaMalloc after a stream sync.  Highest
+ *                          bandwidth when the step's adapters exceed what one wave of clusters covers.
+ *   MILORA_DECODE_AUTO     (default) SPLIT when the work list has room for more jobs than two waves of clusters
+ *                          cover (more than one job slot per SM), else CLUSTER.
+ * Calls of one context that use SPLIT must be ordered on one stream (they share the scratch buffer).
+ * Returns MILORA_E_ARG for another value.  fp32 contexts always use the generic kernel. */
+typedef enum { MILORA_DECODE_AUTO = 0, MILORA_DECODE_CLUSTER = 1, MILORA_DECODE_SPLIT = 2 } milora_decode_path;
+milora_status milora_set_decode_path(milora_ctx* ctx, milora_decode_path path);
+/* The kernel set (CLUSTER or SPLIT) that milora_apply_decode would use, with the current setting, for a bf16
+ * batch of n_seq sequences and T rows whose shapes fit both; host arithmetic only. */
+milora_status milora_decode_path_for(const milora_ctx* ctx, int n_seq, int T, milora_decode_path* out);
+
 /* Several module call sites of one layer in a single launch (for example q,k,v share an input,
  * gate,up share an input).  modules[i], X_dev[i], Y_dev[i] describe site i; a module may appear once. */
 milora_status milora_apply_decode_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,

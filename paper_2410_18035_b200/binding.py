@@ -74,6 +74,8 @@ SIGNATURES = {
     "milora_gate_table_write": (_I, [_VP, _I, _I, _VP, _VP]),
     "milora_group_layout": (_I, [_VP, _I, _I, C.POINTER(GroupLayout)]),
     "milora_group": (_I, [_VP, _I, _I, _VP, _VP, _I, _I, _VP, C.c_size_t, _VP]),
+    "milora_set_decode_path": (_I, [_VP, _I]),
+    "milora_decode_path_for": (_I, [_VP, _I, _I, C.POINTER(_I)]),
     "milora_apply_decode": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_prefill": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_decode_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
@@ -302,6 +304,17 @@ class Milora:
         self._tensor(Y, self.torch_dtype, "Y")
         if X.shape[0] < T or Y.shape[0] < T or X.shape[1] != d1 or Y.shape[1] != d2:
             raise ValueError(f"apply: X/Y shapes {tuple(X.shape)}/{tuple(Y.shape)} do not fit module {module} with T={T}")
+
+    def set_decode_path(self, path):
+        """milora_set_decode_path: 0 / "auto", 1 / "cluster" (one launch), 2 / "split" (two streaming launches)."""
+        code = {"auto": 0, "cluster": 1, "split": 2}.get(path, path)
+        self._check(self.lib.milora_set_decode_path(self.h, int(code)), "milora_set_decode_path")
+
+    def decode_path_for(self, n_seq, T):
+        """milora_decode_path_for: 1 (cluster, one launch) or 2 (split, two launches) for such a batch."""
+        out = C.c_int(0)
+        self._check(self.lib.milora_decode_path_for(self.h, n_seq, T, C.byref(out)), "milora_decode_path_for")
+        return out.value
 
     def apply_decode(self, layer, module, X, Y, groups: Groups, stream=None):
         self._xy(module, X, Y, groups.T)

@@ -169,6 +169,8 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->d_err = nullptr; ctx->d_scratch = nullptr; ctx->scratch_floats = 0; ctx->d_counters = nullptr;
   ctx->d_vscratch = nullptr; ctx->vscratch_floats = 0;
   ctx->d_lin = nullptr; ctx->lin_bytes = 0;
+  ctx->d_dsplit = nullptr; ctx->dsplit_floats = 0; ctx->dsplit_dirty = true;
+  ctx->dsplit_occ_s = 0; ctx->dsplit_occ_e = 0; ctx->decode_path = MILORA_DECODE_AUTO;
   ctx->copy_stream = nullptr; ctx->ev_done = nullptr; ctx->copy_ready = false;
   for (int m = 0; m < MILORA_NMOD; ++m) ctx->ev_site[m] = nullptr;
   ctx->n_counters = 0;
@@ -231,6 +233,7 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_counters);
   cudaFree(ctx->d_vscratch);
   cudaFree(ctx->d_lin);
+  cudaFree(ctx->d_dsplit);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
   for (int m = 0; m < MILORA_NMOD; ++m)
@@ -504,6 +507,20 @@ milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   return launch_group(ctx, layer_begin, n_layers, cu_seqlens_dev, seq_slot_dev, n_seq, T, ws_dev, ws_stride, s);
 }
 
+// AUTO: the two-kernel path once the work list has room for more jobs than two waves of clusters cover
+// (four CTAs per SM, eight per cluster: half the SM count per wave).  Below that the single launch wins on latency.
+static milora_decode_path pick_decode_path(const milora_ctx* ctx, int n_seq, int T) {
+  if (ctx->decode_path != MILORA_DECODE_AUTO) return (milora_decode_path)ctx->decode_path;
+  const milora_group_layout_t lay = group_layout(n_seq, T, top_k_of(ctx));
+  return lay.max_gather > ctx->sm_count ? MILORA_DECODE_SPLIT : MILORA_DECODE_CLUSTER;
+}
+
+milora_status milora_decode_path_for(const milora_ctx* ctx, int n_seq, int T, milora_decode_path* out) {
+  if (!ctx || !out || n_seq < 0 || T < 0) return MILORA_E_ARG;
+  *out = pick_decode_path(ctx, n_seq, T);
+  return MILORA_OK;
+}
+
 static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const int* modules,
                                   const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                   bool dense, void* stream) {
@@ -530,11 +547,26 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
   milora_status st = sync_tables(ctx, s);
   if (st != MILORA_OK) return st;
   if (ctx->desc.dtype == MILORA_BF16) {
-    st = dense ? launch_apply_prefill_bf16(ctx, layer, sites, groups, s)
-               : launch_apply_decode_bf16(ctx, layer, sites, groups, s);
+    if (dense) {
+      st = launch_apply_prefill_bf16(ctx, layer, sites, groups, s);
+    } else {
+      st = MILORA_E_SHAPE;
+      if (ctx->decode_path != MILORA_DECODE_CLUSTER) {
+        if (pick_decode_path(ctx, groups->n_seq, groups->T) == MILORA_DECODE_SPLIT)
+          st = launch_apply_decode_split(ctx, layer, sites, groups, s);
+      }
+      if (st == MILORA_E_SHAPE) st = launch_apply_decode_bf16(ctx, layer, sites, groups, s);
+    }
     if (st != MILORA_E_SHAPE) return st;     // MILORA_E_SHAPE: this batch does not fit the specialised kernel
   }
   return launch_apply_generic(ctx, layer, sites, groups, dense, s);
+}
+
+milora_status milora_set_decode_path(milora_ctx* ctx, milora_decode_path path) {
+  if (!ctx) return MILORA_E_ARG;
+  if (path != MILORA_DECODE_AUTO && path != MILORA_DECODE_CLUSTER && path != MILORA_DECODE_SPLIT) return MILORA_E_ARG;
+  ctx->decode_path = (int)path;
+  return MILORA_OK;
 }
 
 milora_status milora_apply_decode(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,

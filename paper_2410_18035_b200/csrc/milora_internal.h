@@ -121,6 +121,11 @@ struct milora_ctx {
   size_t n_counters;
   float* d_vscratch;                            // prefill: fp32 partial x.A products [k-split][T][rank_pad]
   size_t vscratch_floats;
+  float* d_dsplit;                              // two-kernel decode path: unit counters (64 words), then v [jobs][rows][rank]
+  size_t dsplit_floats;
+  bool dsplit_dirty;                            // counters must be cleared before the next launch pair
+  int dsplit_occ_s, dsplit_occ_e;               // resident CTAs per SM of its two kernels (0 = not asked yet)
+  int decode_path;                              // milora_decode_path
   void* d_lin;                                  // fused projection: V piece images and per-row-block piece lists
   size_t lin_bytes;
   cudaStream_t copy_stream;                     // milora_step_host: device-to-host copies run beside the uploads
@@ -203,6 +208,11 @@ milora_status launch_apply_generic(milora_ctx* ctx, int layer, const ApplySites&
 // Returns MILORA_E_SHAPE when shapes or alignment do not fit it (the caller then uses the generic path).
 milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
                                        cudaStream_t s);
+
+// bf16 decode path as two streaming kernels (shrink over whole rows of A^T, expand over column slices of B) that
+// take equally sized units from a counter; v goes through a scratch buffer of the context.  Same convention.
+milora_status launch_apply_decode_split(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
+                                        cudaStream_t s);
 
 // bf16 prefill path: tcgen05 shrink and expand kernels over the dense tiles (same MILORA_E_SHAPE convention),
 // and the registration-time packing of the operand images they read.

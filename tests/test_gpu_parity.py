@@ -42,10 +42,12 @@ def _route_all_layers(lw, ids, **okw):
     return table_g, table_o, excused
 
 
-def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, gate=None):
+def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, gate=None, decode_path="auto"):
     """group + apply (prefill and decode lists) on one step; compares grouping and all 7 module outputs.
-    table is [R, L] (top-1) or [R, L, k]; gate, when given, holds the [R, L, k] weights of the selected modules."""
+    table is [R, L] (top-1) or [R, L, k]; gate, when given, holds the [R, L, k] weights of the selected modules.
+    decode_path picks the kernel set of milora_apply_decode (bf16 contexts)."""
     w, ml = lw.w, lw.ml
+    ml.set_decode_path(decode_path)
     layer = lw.layers[li]
     cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
     n_seq = slots.numel()
@@ -136,7 +138,8 @@ RAGGED = [1, 33, 130, 257, 31, 32, 7, 129]
 @pytest.mark.parametrize("dtype,d,d_ff,d_kv,r", [("f32", 256, 688, 256, 8), ("bf16", 512, 1376, 128, 16),
                                                  ("bf16", 256, 688, 256, 40), ("bf16", 1024, 2816, 256, 16),
                                                  ("bf16", 512, 1408, 512, 32), ("bf16", 512, 1408, 128, 64)])
-def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r):
+@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r, decode_path):
     """Sequences of 1..257 rows (both work lists, ragged tile tails) mixed with decode rows; tenants repeat so
     that several sequences share a bucket; one slot is closed and one tenant has no adapters."""
     base = get_workload("c1")
@@ -153,13 +156,13 @@ def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r):
     table = table_g.copy()        # use the GPU's decisions downstream so that an excused near tie cannot cascade
     prefill, decode = list(range(len(RAGGED))), list(range(len(RAGGED), n))
     for li in range(2):
-        _step_parity(lw, li, prefill, decode, table, tag=7)
-        _step_parity(lw, li, prefill[::-1], decode, table, tag=8, use_multi=True)
+        _step_parity(lw, li, prefill, decode, table, tag=7, decode_path=decode_path)
+        _step_parity(lw, li, prefill[::-1], decode, table, tag=8, use_multi=True, decode_path=decode_path)
     # close a slot: its rows become excluded and stay bit-identical
     lw.ml.request_close(3)
     w.request_tenant = w.request_tenant.copy()
     w.request_tenant[3] = -1
-    _step_parity(lw, 0, prefill, decode, table, tag=9)
+    _step_parity(lw, 0, prefill, decode, table, tag=9, decode_path=decode_path)
     lw.close()
 
 
@@ -205,8 +208,8 @@ def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
     gate_arg = gates_o if gate else None
     prefill, decode = list(range(len(RAGGED))), list(range(len(RAGGED), n))
     for li in range(2):
-        _step_parity(lw, li, prefill, decode, table, tag=11, gate=gate_arg)
-        _step_parity(lw, li, prefill[::-1], decode, table, tag=12, use_multi=True, gate=gate_arg)
+        _step_parity(lw, li, prefill, decode, table, tag=11, gate=gate_arg, decode_path="cluster")
+        _step_parity(lw, li, prefill[::-1], decode, table, tag=12, use_multi=True, gate=gate_arg, decode_path="split")
     # restoring a table by hand: duplicates inside a cell are refused
     from paper_2410_18035_b200 import MiloraError
     if k >= 2:
