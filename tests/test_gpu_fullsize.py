@@ -38,9 +38,11 @@ def _sample_rows(cu, rng, per_seq=6):
     return np.array(sorted(set(rows)), dtype=np.int64)
 
 
-def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True):
-    """One step in the bench's configuration: group, multi-site prefill apply, multi-site decode apply."""
+def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True, decode_path="auto"):
+    """One step in the bench's configuration: group, multi-site prefill apply, multi-site decode apply
+    (decode_path: which kernel set milora_apply_decode uses)."""
     w, ml = lw.w, lw.ml
+    ml.set_decode_path(decode_path)
     layer = lw.layers[li]
     cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
     n_seq = slots.numel()
@@ -104,6 +106,7 @@ def test_config2_full_size_bench_configuration():
     rng = np.random.default_rng(0)
     _check_step(lw, 0, ids, [], table, tag=0, rng=rng)          # prefill rows (dense tiles)
     _check_step(lw, 0, [], ids, table, tag=1, rng=rng)          # decode rows (gathered)
+    _check_step(lw, 0, [], ids, table, tag=4, rng=rng, decode_path="split")
     _check_step(lw, 0, ids[:8], ids[8:], table, tag=2, rng=rng, multi=False)   # mixed, per-site calls
     _check_step(lw, 0, ids, ids, table, tag=3, rng=rng)         # all prompts and all decode rows as one batch
     lw.close()
@@ -135,8 +138,9 @@ def test_config4_shape_zipf_decode_one_layer():
     table, excused = _route_and_check(lw, 0, ids)
     assert excused <= 8
     rng = np.random.default_rng(2)
-    _check_step(lw, 0, [], ids, table, tag=0, rng=rng)
-    # the same requests as three-row sequences (beams share slot, tenant and route)
+    assert lw.ml.decode_path_for(len(ids), len(ids)) == 2       # a batch of this size takes the two-launch kernels
+    _check_step(lw, 0, [], ids, table, tag=0, rng=rng, decode_path="split")
+    _check_step(lw, 0, [], ids, table, tag=1, rng=rng, decode_path="cluster")
     lw.close()
 
 

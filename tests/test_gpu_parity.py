@@ -316,7 +316,8 @@ def test_fused_projection_refuses_what_it_cannot_run():
     ml.close()
 
 
-def test_back_to_back_launches_equal_serialised_ones_bit_for_bit():
+@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+def test_back_to_back_launches_equal_serialised_ones_bit_for_bit(decode_path):
     """Every kernel may start while the one before it is still draining (programmatic dependent launch) and takes
     its work from device-side lists.  The results must not depend on that: the whole step enqueued back to back,
     twice, and once with a device synchronisation after every call give bit-identical routes, logits and outputs."""
@@ -330,6 +331,7 @@ def test_back_to_back_launches_equal_serialised_ones_bit_for_bit():
     w.gen_device = "cuda"
     lw = _loaded(w)
     ml = lw.ml
+    ml.set_decode_path(decode_path)     # the two-launch set hands its units out through a counter: same requirement
     prefill, decode = list(range(8)), list(range(8, n))
     lw.route(0, decode)                                   # the running requests were routed earlier
     H = w.hidden_batch(0, prefill, "cuda")
