@@ -466,8 +466,8 @@ def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
 
 def run_mixed_step(step, device, iters=50):
     """The same rows as one continuous batch: the 64 prompts and the 64 decode rows in ONE grouping call, then the
-    dense-tile kernels and the gathered kernel on the same group block (6 launches).  The job list of such a batch
-    is sized for the worst case, so the decode kernel runs in its looped form.  Reported beside the step."""
+    dense-tile kernels and the gathered kernels on the same group block.  The job list of such a batch is sized
+    for the worst case (every row short).  Reported beside the step."""
     lw, ml, w = step.lw, step.lw.ml, step.w
     cu, slots, T = lw.seq_arrays(step.prefill_ids, step.decode_ids)
     n_seq = len(step.prefill_ids) + len(step.decode_ids)
@@ -493,7 +493,8 @@ def run_mixed_step(step, device, iters=50):
     torch.cuda.synchronize(device)
     ms = e0.elapsed_time(e1) / iters
     err = ml.poll_error()
-    return {"ms_per_step": ms, "token_layers_per_s": T / (ms * 1e-3), "launches": 6, "rows": T, "sequences": n_seq,
+    launches = 2 + 1 + 2 + (2 if ml.decode_path_for(n_seq, T) == 2 else 1)
+    return {"ms_per_step": ms, "token_layers_per_s": T / (ms * 1e-3), "launches": launches, "rows": T, "sequences": n_seq,
             "device_error_flag": err}
 
 
