@@ -33,7 +33,9 @@ constexpr int kSRows = 16;         // rank rows per shrink unit: the M of one mm
 constexpr int kSCols = 1024;       // columns of A^T per shrink unit
 constexpr int kSGroups = kSCols / 32 / kSWarps;   // 32-column groups a warp owns in a unit
 constexpr int kSBatch = 4;         // groups whose loads a warp issues before it consumes them
-constexpr int kEThreads = 128;     // 1024 columns of B per expand unit: four warps, four 64-column spans each
+constexpr int kEThreads = 128;
+constexpr int kECols = 1024;       // columns of B per expand unit: four warps, four 64-column spans each
+                                   // (512-column units: 52.1 us per layer on the 13B chain against 48.7)
 constexpr int kMaxRankSplit = 256;
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
@@ -95,7 +97,7 @@ __device__ __forceinline__ void build_map(const SplitArgs& a, UnitMap* m, int ti
       int upj = 0;
       if (si >= 0) {
         if (EXPAND) {
-          upj = ((a.sites.site[si].d2 >> 3) + kEThreads - 1) / kEThreads;
+          upj = (a.sites.site[si].d2 + kECols - 1) / kECols;
         } else {
           upj = shrink_units(a.sites.site[si].d1, a.rmax);
         }
@@ -266,7 +268,7 @@ __global__ void __launch_bounds__(kSThreads, 6) decode_shrink_kernel(SplitArgs a
 // (g, q) are 16 consecutive columns of row g of y.  v enters as bf16 twice, as its rounded value and as the
 // rounding remainder, which keeps the fp32 value of v to 2^-17.
 constexpr int kESpan = 64;                                   // columns per group of eight MMAs
-constexpr int kESpans = kEThreads * 8 / kESpan / (kEThreads / 32);   // spans a warp owns in a unit (4)
+constexpr int kESpans = kECols / kESpan / (kEThreads / 32);          // spans a warp owns in a unit
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -316,8 +318,17 @@ __device__ __forceinline__ void expand_unit(const SplitArgs& a, const GatherJob&
     const int chunks = shrink_chunks(site.d1);
     for (int idx = tid; idx < n * r; idx += kEThreads) {
       const int t = idx / r, j = idx % r;
+      // the loads of sixteen chunks go out together; the additions keep the chunk order
+      const float* vp = a.v + (((size_t)job_idx * a.kcmax) * kR + t) * a.rmax + j;
+      const size_t cstride = (size_t)kR * a.rmax;
       float sum = 0.f;
-      for (int c = 0; c < chunks; ++c) sum += a.v[(((size_t)job_idx * a.kcmax + c) * kR + t) * a.rmax + j];
+      for (int c0 = 0; c0 < chunks; c0 += 16) {
+        float part[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) part[i] = (c0 + i < chunks) ? vp[(size_t)(c0 + i) * cstride] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum += part[i];
+      }
       vs[t][j] = sum;
     }
   }
@@ -345,49 +356,62 @@ __device__ __forceinline__ void expand_unit(const SplitArgs& a, const GatherJob&
   for (int t = 1; t < kR; ++t) yr = (g == t) ? job.rows[t] : yr;
   const bool y_row_ok = g < n;
   uint4* Yrow = static_cast<uint4*>(site.Y) + (size_t)(y_row_ok ? yr : 0) * nv2;
+  // The warp's spans and their rank blocks form one sequence of steps; the piece of step s + 1 is loaded before the
+  // MMAs of step s, across span boundaries too, and the y pieces of the next span at the start of the current one,
+  // so that the warp always has loads in flight.
+  const int col8_0 = (sub * kECols + warp * kESpans * kESpan) >> 3;     // first span's start, in 8-column pieces
+  const int nspans = min(kESpans, (nv2 - col8_0 + 7) >> 3);                      // spans that start inside the matrix
+  if (nspans > 0) {
+    // this thread loads pieces col8 + g of a span and owns the results of its pieces col8 + 2q, col8 + 2q + 1
+    auto piece_of = [&](int sp, int kb) {
+      return load_piece(static_cast<const char*>(job.B) + (size_t)min(col8_0 + sp * 8 + g, nv2 - 1) * 16, kb, q, r, pitch);
+    };
+    auto y_of = [&](int sp, int which) {
+      const int c = col8_0 + sp * 8 + 2 * q + which;
+      return (y_row_ok && sp < nspans && c < nv2) ? Yrow[c] : make_uint4(0, 0, 0, 0);
+    };
+    BPiece cur = piece_of(0, 0);
+    uint4 y0 = y_of(0, 0), y1 = y_of(0, 1);
 #pragma unroll 1
-  for (int sp = 0; sp < kESpans; ++sp) {
-    const int col8 = (sub * (kEThreads * 8) + (warp * kESpans + sp) * kESpan) >> 3;    // span start, in 8-column pieces
-    if (col8 >= nv2) break;
-    // this thread loads pieces col8 + g and owns the results of pieces col8 + 2q, col8 + 2q + 1
-    const char* bcol = static_cast<const char*>(job.B) + (size_t)min(col8 + g, nv2 - 1) * 16;
-    const bool y_ok0 = y_row_ok && col8 + 2 * q < nv2, y_ok1 = y_row_ok && col8 + 2 * q + 1 < nv2;
-    uint4 y0 = make_uint4(0, 0, 0, 0), y1 = y0;
-    if (y_ok0) y0 = Yrow[col8 + 2 * q];
-    if (y_ok1) y1 = Yrow[col8 + 2 * q + 1];
-    float acc[8][4];
+    for (int sp = 0; sp < nspans; ++sp) {
+      const int col8 = col8_0 + sp * 8;
+      const uint4 yn0 = y_of(sp + 1, 0), yn1 = y_of(sp + 1, 1);
+      float acc[8][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
-    BPiece cur = load_piece(bcol, 0, q, r, pitch);
+        for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
 #pragma unroll 1
-    for (int kb = 0; kb < kblocks; ++kb) {
-      BPiece nxt = cur;
-      if (kb + 1 < kblocks) nxt = load_piece(bcol, kb + 1, q, r, pitch);
-      mma_piece(acc, cur, va_sm[kb][lane]);
-      cur = nxt;
-    }
-    // acc[i][0] is column 16q + i of the span, acc[i][1] column 16q + 8 + i, both of row g
-    if (y_ok0) {
-      const uint32_t w[4] = {y0.x, y0.y, y0.z, y0.w};
-      float o[8];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        o[2 * i] = bf16_lo(w[i]) + acc[2 * i][0];
-        o[2 * i + 1] = bf16_hi(w[i]) + acc[2 * i + 1][0];
+      for (int kb = 0; kb < kblocks; ++kb) {
+        BPiece nxt = cur;
+        if (kb + 1 < kblocks) nxt = piece_of(sp, kb + 1);
+        else if (sp + 1 < nspans) nxt = piece_of(sp + 1, 0);
+        mma_piece(acc, cur, va_sm[kb][lane]);
+        cur = nxt;
       }
-      Yrow[col8 + 2 * q] = pack8(o);
-    }
-    if (y_ok1) {
-      const uint32_t w[4] = {y1.x, y1.y, y1.z, y1.w};
-      float o[8];
+      // acc[i][0] is column 16q + i of the span, acc[i][1] column 16q + 8 + i, both of row g
+      if (y_row_ok && col8 + 2 * q < nv2) {
+        const uint32_t w[4] = {y0.x, y0.y, y0.z, y0.w};
+        float o[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        o[2 * i] = bf16_lo(w[i]) + acc[2 * i][1];
-        o[2 * i + 1] = bf16_hi(w[i]) + acc[2 * i + 1][1];
+        for (int i = 0; i < 4; ++i) {
+          o[2 * i] = bf16_lo(w[i]) + acc[2 * i][0];
+          o[2 * i + 1] = bf16_hi(w[i]) + acc[2 * i + 1][0];
+        }
+        Yrow[col8 + 2 * q] = pack8(o);
       }
-      Yrow[col8 + 2 * q + 1] = pack8(o);
+      if (y_row_ok && col8 + 2 * q + 1 < nv2) {
+        const uint32_t w[4] = {y1.x, y1.y, y1.z, y1.w};
+        float o[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          o[2 * i] = bf16_lo(w[i]) + acc[2 * i][1];
+          o[2 * i + 1] = bf16_hi(w[i]) + acc[2 * i + 1][1];
+        }
+        Yrow[col8 + 2 * q + 1] = pack8(o);
+      }
+      y0 = yn0;
+      y1 = yn1;
     }
   }
   __syncthreads();    // vs and va_sm are rewritten by the next unit
@@ -411,9 +435,9 @@ __global__ void __launch_bounds__(kEThreads, 4) decode_expand_kernel(SplitArgs a
     const GatherJob job = load_job(a, un.job_idx);
     if (job_ok(a, job, un.site)) {
       const ApplySite& st = a.sites.site[un.site];
-      const int c0 = un.sub * kEThreads * 8;
+      const int c0 = un.sub * kECols;
       prefetch_rows(static_cast<const char*>(job.B) + (size_t)c0 * 2, (size_t)st.d2 * 2, job.rank,
-                    min(kEThreads * 16, (st.d2 - c0) * 2), tid, kEThreads);
+                    min(kECols * 2, (st.d2 - c0) * 2), tid, kEThreads);
     }
   }
   pdl_wait();
@@ -449,7 +473,7 @@ milora_status launch_apply_decode_split(milora_ctx* ctx, int layer, const ApplyS
     if ((st.d1 & 7) || (st.d2 & 7)) return MILORA_E_SHAPE;
     upj_s = std::max(upj_s, shrink_units(st.d1, a.rmax));
     kcmax = std::max(kcmax, shrink_chunks(st.d1));
-    upj_e = std::max(upj_e, ((st.d2 >> 3) + kEThreads - 1) / kEThreads);
+    upj_e = std::max(upj_e, (st.d2 + kECols - 1) / kECols);
   }
   if (a.lay.max_gather < 1) return MILORA_OK;
   // scratch: 64 floats of counters, then v
