@@ -430,6 +430,66 @@ def test_group_edge_cases_and_device_flags():
     lw.close()
 
 
+@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+def test_decode_kernel_sets_edge_cases(decode_path):
+    """Both decode kernel sets: a batch without any short sequence (empty gathered list) leaves every row
+    bit-identical; the same decode batch applied five times in a row (the two-launch set hands its unit counters
+    from one call to the next) gives bit-identical results each time, equal to the oracle's; a set other than
+    the three named ones is refused."""
+    from paper_2410_18035_b200 import MiloraError
+    base = get_workload("c1")
+    lens = np.array([40, 64] + [1] * 9, dtype=np.int32)
+    n = len(lens)
+    tenants = (np.arange(n) % 3).astype(np.int32)
+    w = scaled_workload(base, name="decode_edges", dtype="bf16", d_model=512, d_ff=1376, d_kv=128, rank=24, n_tenants=3,
+                        request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(2), decode_ids=np.arange(2, n),
+                        has_base_weights=False, n_layers=1)
+    lw = _loaded(w)
+    ml = lw.ml
+    with pytest.raises(MiloraError):
+        ml.set_decode_path(3)
+    ml.set_decode_path(decode_path)
+    ids = list(range(n))
+    lw.route(0, ids)
+    table = ml.route_table_read(0, n).numpy()[:, 0].copy()
+    # 1. prompts only: nothing for the decode kernels to do
+    cu, slots, T = lw.seq_arrays([0, 1], [])
+    ws = ml.alloc_group_ws(1, 2, T)
+    ml.group(0, 1, cu, slots, 2, T, ws)
+    groups = ml.groups(ws[0], 2, T)
+    for m in range(7):
+        X = w.module_input(0, m, T, 3, "cuda")
+        Yb = w.base_output(0, m, T, 3, "cuda")
+        Y = Yb.clone()
+        ml.apply_decode(0, m, X, Y, groups)
+        torch.cuda.synchronize()
+        assert torch.equal(Y, Yb)
+    # 2. the decode rows, five calls in a row on fresh copies of y
+    dec = list(range(2, n))
+    cu, slots, T = lw.seq_arrays([], dec)
+    ws = ml.alloc_group_ws(1, len(dec), T)
+    ml.group(0, 1, cu, slots, len(dec), T, ws)
+    groups = ml.groups(ws[0], len(dec), T)
+    token_slot = slots.cpu().numpy()
+    Xs = [w.module_input(0, m, T, 4, "cuda") for m in range(7)]
+    Ybs = [w.base_output(0, m, T, 4, "cuda") for m in range(7)]
+    first = None
+    for rep in range(5):
+        Ys = [y.clone() for y in Ybs]
+        ml.apply_decode_multi(0, list(range(7)), Xs, Ys, groups)
+        torch.cuda.synchronize()
+        if first is None:
+            first = Ys
+            for m in range(7):
+                y_o = R.apply_site(w, 0, m, Xs[m].cpu(), Ybs[m].cpu(), token_slot, table)
+                assert_apply_close(Ys[m], y_o, Ybs[m], "bf16", what=f"decode edges module {m}")
+        else:
+            for m in range(7):
+                assert torch.equal(Ys[m], first[m]), f"call {rep}, module {m}: result changed between calls"
+    assert ml.poll_error() == 0
+    lw.close()
+
+
 @pytest.mark.parametrize("pool,act,bias", [(O.POOL_MAX, O.ACT_RELU, False), (O.POOL_LAST, O.ACT_GELU, True),
                                             (O.POOL_SELFATTN, O.ACT_RATIONAL, False),
                                             (O.POOL_MEAN, O.ACT_IDENTITY, True), (O.POOL_SELFATTN, O.ACT_TANH, True)])
