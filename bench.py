@@ -251,7 +251,8 @@ def run_ours(args, rank, world, device):
         if rank == 0:
             sampler.stop()
             print(json.dumps({"decode_stack": run_decode_stack(step, device, load_peaks()),
-                              "decode_stack_13b_zipf": run_decode_13b(device, load_peaks())}))
+                              "decode_stack_13b_zipf": run_decode_13b(device, load_peaks()),
+                              "decode_batch_sweep": run_decode_sweep(device, load_peaks())}))
         return None
     routes = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0]
     work = algorithmic_work(w, routes, step.prefill_ids, step.decode_ids)
@@ -286,12 +287,13 @@ def run_ours(args, rank, world, device):
     ms_per_step = total_ms / args.steps
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
-    fused = stack = stack13 = mixed = None
+    fused = stack = stack13 = mixed = sweep = None
     if rank == 0 and not args.skip_fused and w.dtype == "bf16":
         mixed = run_mixed_step(step, device)
         fused = run_fused_projection(step, routes, device, load_peaks())
         stack = run_decode_stack(step, device, load_peaks())
         stack13 = run_decode_13b(device, load_peaks())
+        sweep = run_decode_sweep(device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
 
@@ -337,6 +339,7 @@ def run_ours(args, rank, world, device):
             "fused_projection": fused,
             "decode_stack": stack,
             "decode_stack_13b_zipf": stack13,
+            "decode_batch_sweep": sweep,
             "mixed_batch_step": mixed,
         },
         "roofline": dict(rooflines[dom], kernel=dom),
@@ -518,6 +521,36 @@ def run_decode_13b(device, peaks, n_layers=2, rounds=20):
     out = _timed_decode_chain(lw.ml, w, n_layers, cu_d, slots_d, T_d, ids, Xd, Yd, device, peaks, rounds)
     lw.close()
     return out
+
+
+def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=2, rounds=20):
+    """Decode-only batch sweep on the LLaMA-3-8B shapes (GQA k/v, rank 16, tenants = batch size): the same replayed
+    chain as above for each batch size, two layers alternating, with either decode kernel set and with the
+    library's own choice.  Small batches are bound by the launch, large ones by the adapter stream."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth.workloads import decode_sweep_workload, scaled_workload
+    out = []
+    for b in batches:
+        w = scaled_workload(decode_sweep_workload(b), n_layers=n_layers, prompt_len=np.full(b, 64, dtype=np.int32))
+        w.gen_device = str(device)
+        lw = LoadedWorkload(w, device)
+        ids = list(range(b))
+        for li in range(n_layers):
+            for i0 in range(0, b, 64):
+                lw.route(li, ids[i0:i0 + 64])
+        cu_d, slots_d, T_d = lw.seq_arrays([], ids)
+        Xd = [w.module_input(0, m, T_d, 1, device) for m in range(7)]
+        Yd = [w.base_output(0, m, T_d, 1, device) for m in range(7)]
+        r = _timed_decode_chain(lw.ml, w, n_layers, cu_d, slots_d, T_d, ids, Xd, Yd, device, peaks, rounds)
+        out.append({"batch": b, "us_per_layer": r["us_per_layer_launch"], "gbs": r["gbs"],
+                    "frac_of_measured_hbm": r["frac_of_measured_hbm"],
+                    "algorithmic_bytes_per_layer": r["algorithmic_bytes_per_layer"],
+                    "chosen": "split" if lw.ml.decode_path_for(b, b) == 2 else "cluster",
+                    "us_per_layer_by_path": {k: v["us_per_layer"] for k, v in r["by_decode_path"].items()},
+                    "device_error_flag": r["device_error_flag"]})
+        lw.close()
+        del Xd, Yd
+    return {"workload": "c5_llama3_8b_decode_sweep_bf16", "layers": n_layers, "rank": 16, "sweep": out}
 
 
 def run_e2e(step, args, world, device, tokens_per_step):

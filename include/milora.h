@@ -242,8 +242,9 @@ milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const
  *                          second launch takes them as bf16 value + bf16 remainder, i.e. to 2^-17), which the first call (and any call with a larger
  *                          batch than every earlier one) grows with cudaMalloc after a stream sync.  Highest
  *                          bandwidth when the step's adapters exceed what one wave of clusters covers.
- *   MILORA_DECODE_AUTO     (default) SPLIT when the work list has room for more jobs than two waves of clusters
- *                          cover (more than one job slot per SM), else CLUSTER.
+ *   MILORA_DECODE_AUTO     (default) SPLIT when the work list has room for more than two jobs per SM (on a B200:
+ *                          decode batches from about 240 requests, and every batch that mixes prompts with
+ *                          decode rows), else CLUSTER.
  * Calls of one context that use SPLIT must be ordered on one stream (they share the scratch buffer).
  * Returns MILORA_E_ARG for another value.  fp32 contexts always use the generic kernel. */
 typedef enum { MILORA_DECODE_AUTO = 0, MILORA_DECODE_CLUSTER = 1, MILORA_DECODE_SPLIT = 2 } milora_decode_path;
