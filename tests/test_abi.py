@@ -45,6 +45,10 @@ def test_status_strings(lib):
     # host-side argument validation needs no device
     assert lib.milora_create(None, None) == 1
     assert lib.milora_destroy(None) == 0
+    lib.milora_set_decode_path.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.milora_decode_path_for.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+    assert lib.milora_set_decode_path(None, 2) == 1
+    assert lib.milora_decode_path_for(None, 1, 1, None) == 1
 
 
 def test_product_path_does_not_touch_the_oracle():
