@@ -313,6 +313,29 @@ __device__ __forceinline__ void expand_unit(const SplitArgs& a, const GatherJob&
   const int d2 = site.d2, nv2 = d2 >> 3, r = job.rank, n = min(job.count, kR);
   const int kblocks = (r + 15) >> 4;
   const size_t pitch = (size_t)d2 * 2;
+  int yr = job.rows[0];
+#pragma unroll
+  for (int t = 1; t < kR; ++t) yr = (g == t) ? job.rows[t] : yr;
+  const bool y_row_ok = g < n;
+  uint4* Yrow = static_cast<uint4*>(site.Y) + (size_t)(y_row_ok ? yr : 0) * nv2;
+  // The warp's spans and their rank blocks form one sequence of steps; the piece of step s + 1 is loaded before the
+  // MMAs of step s, across span boundaries too, and the y pieces of the next span at the start of the current one,
+  // so that the warp always has loads in flight.  The first piece and the first span's y go out before v is put
+  // together, so that their latency and that of the chunk sums overlap.
+  const int col8_0 = (sub * kECols + warp * kESpans * kESpan) >> 3;     // first span's start, in 8-column pieces
+  const int nspans = max(0, min(kESpans, (nv2 - col8_0 + 7) >> 3));              // spans that start inside the matrix
+  // this thread loads pieces col8 + g of a span and owns the results of its pieces col8 + 2q, col8 + 2q + 1
+  auto piece_of = [&](int sp, int kb) {
+    return load_piece(static_cast<const char*>(job.B) + (size_t)min(col8_0 + sp * 8 + g, nv2 - 1) * 16, kb, q, r, pitch);
+  };
+  auto y_of = [&](int sp, int which) {
+    const int c = col8_0 + sp * 8 + 2 * q + which;
+    return (y_row_ok && sp < nspans && c < nv2) ? Yrow[c] : make_uint4(0, 0, 0, 0);
+  };
+  BPiece cur;
+  cur.r0 = cur.r1 = cur.r8 = cur.r9 = make_uint4(0, 0, 0, 0);
+  if (nspans > 0) cur = piece_of(0, 0);
+  uint4 y0 = y_of(0, 0), y1 = y_of(0, 1);
   // v = sum of the shrink kernel's partial products over the column chunks of d1, in chunk order
   {
     const int chunks = shrink_chunks(site.d1);
@@ -351,27 +374,7 @@ __device__ __forceinline__ void expand_unit(const SplitArgs& a, const GatherJob&
     va_sm[kb][l] = f;
   }
   __syncthreads();
-  int yr = job.rows[0];
-#pragma unroll
-  for (int t = 1; t < kR; ++t) yr = (g == t) ? job.rows[t] : yr;
-  const bool y_row_ok = g < n;
-  uint4* Yrow = static_cast<uint4*>(site.Y) + (size_t)(y_row_ok ? yr : 0) * nv2;
-  // The warp's spans and their rank blocks form one sequence of steps; the piece of step s + 1 is loaded before the
-  // MMAs of step s, across span boundaries too, and the y pieces of the next span at the start of the current one,
-  // so that the warp always has loads in flight.
-  const int col8_0 = (sub * kECols + warp * kESpans * kESpan) >> 3;     // first span's start, in 8-column pieces
-  const int nspans = min(kESpans, (nv2 - col8_0 + 7) >> 3);                      // spans that start inside the matrix
   if (nspans > 0) {
-    // this thread loads pieces col8 + g of a span and owns the results of its pieces col8 + 2q, col8 + 2q + 1
-    auto piece_of = [&](int sp, int kb) {
-      return load_piece(static_cast<const char*>(job.B) + (size_t)min(col8_0 + sp * 8 + g, nv2 - 1) * 16, kb, q, r, pitch);
-    };
-    auto y_of = [&](int sp, int which) {
-      const int c = col8_0 + sp * 8 + 2 * q + which;
-      return (y_row_ok && sp < nspans && c < nv2) ? Yrow[c] : make_uint4(0, 0, 0, 0);
-    };
-    BPiece cur = piece_of(0, 0);
-    uint4 y0 = y_of(0, 0), y1 = y_of(0, 1);
 #pragma unroll 1
     for (int sp = 0; sp < nspans; ++sp) {
       const int col8 = col8_0 + sp * 8;
