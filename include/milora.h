@@ -232,7 +232,7 @@ milora_status milora_apply_decode(milora_ctx* ctx, int layer, int module, const 
 milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, void* Y_dev,
                                    const milora_groups* groups, void* stream);
 
-/* Which kernels milora_apply_decode uses in a bf16 context (both compute the same Eq. 1; results agree to
+/* Which kernels milora_apply_decode uses in a bf16 context (all compute the same Eq. 1; results agree to
  * rounding of the fp32 sums, and each is deterministic from call to call):
  *   MILORA_DECODE_CLUSTER  one launch; a cluster of eight CTAs per job exchanges partial sums of x W^A through
  *                          distributed shared memory.  Shortest latency when the step has few jobs.
@@ -245,13 +245,47 @@ milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const
  *   MILORA_DECODE_AUTO     (default) SPLIT when the work list has room for more than two jobs per SM (on a B200:
  *                          decode batches from about 240 requests, and every batch that mixes prompts with
  *                          decode rows), else CLUSTER.
- * Calls of one context that use SPLIT must be ordered on one stream (they share the scratch buffer).
- * Returns MILORA_E_ARG for another value.  fp32 contexts always use the generic kernel. */
-typedef enum { MILORA_DECODE_AUTO = 0, MILORA_DECODE_CLUSTER = 1, MILORA_DECODE_SPLIT = 2 } milora_decode_path;
+ *   MILORA_DECODE_STREAM   one persistent launch (one CTA per SM) whose warps each stream pieces of the adapters'
+ *                          operand images through their own ring of shared-memory buffers (cp.async.bulk) and
+ *                          contract them on mma.sync tiles; x W^A goes from its producers to the consumers of W^B
+ *                          inside the launch (scratch buffer of the context, grown like SPLIT's).  It is the kernel
+ *                          behind milora_apply_decode_layers.  Needs a bf16 context with d_model, d_ff and d_kv
+ *                          multiples of 128 and max_rank <= 64; other contexts fall back to CLUSTER.
+ * Calls of one context that use SPLIT or STREAM must be ordered on one stream (they share a scratch buffer).
+ * Returns MILORA_E_ARG for another value.  fp32 contexts always use the generic kernel.
+ */
+typedef enum { MILORA_DECODE_AUTO = 0, MILORA_DECODE_CLUSTER = 1, MILORA_DECODE_SPLIT = 2, MILORA_DECODE_STREAM = 3 }
+    milora_decode_path;
 milora_status milora_set_decode_path(milora_ctx* ctx, milora_decode_path path);
-/* The kernel set (CLUSTER or SPLIT) that milora_apply_decode would use, with the current setting, for a bf16
+/* The kernel set (CLUSTER, SPLIT or STREAM) that milora_apply_decode would use, with the current setting, for a bf16
  * batch of n_seq sequences and T rows whose shapes fit both; host arithmetic only. */
 milora_status milora_decode_path_for(const milora_ctx* ctx, int n_seq, int T, milora_decode_path* out);
+
+/* ---- a whole decode step in one launch (Eq. 1 on every layer; Section 3.3: routes are reused) --------
+ * Applies Eq. 1 to the short sequences (decode rows) of n_layers layers with ONE persistent kernel launch.
+ * Entry i describes one layer: its group block (written by milora_group for that layer) and, per module m,
+ * the inputs X_dev[m] [T][d1(m)] and the outputs Y_dev[m] [T][d2(m)], updated in place on the rows whose request
+ * selects m at that layer; a NULL pair skips the module.  The layers are processed concurrently, so no buffer
+ * that one entry writes may be read or written by another entry (every layer its own Y; X may be shared).
+ * This is the call for an engine that has the inputs of several layers at hand (LoRA terms applied after the
+ * backbone's projections were computed, speculative or pipelined layers, benchmark chains); a layer-by-layer
+ * engine passes one entry per call.  `layers` is host memory and is read before the call returns.
+ * Uses the MILORA_DECODE_STREAM kernel when the context allows it (see milora_set_decode_path), otherwise, or when
+ * the CLUSTER or SPLIT set is forced, one milora_apply_decode_multi per layer.  More than 40 layers, or more
+ * scratch than 512 MB, are split into several launches.  The first call, and calls with larger batches, allocate
+ * (scratch, a pinned staging buffer for the layer records); the records are re-sent to the device only when they
+ * differ from the previous call's, so a decode loop over fixed buffers uploads nothing.  Every wait inside the
+ * kernel is bounded; a wait that runs out raises the device error flag (milora_poll_error). */
+typedef struct {
+  int layer;
+  milora_groups groups;
+  const void* X_dev[MILORA_NMOD];
+  void* Y_dev[MILORA_NMOD];
+} milora_decode_layer;
+milora_status milora_apply_decode_layers(milora_ctx* ctx, const milora_decode_layer* layers, int n_layers, void* stream);
+/* Stages (16 KB pieces of an operand image) per work unit of the STREAM kernel: 1..64, or 0 (default) to let the
+ * library choose from the batch size (long units for large batches, single stages for small ones). */
+milora_status milora_set_decode_unit_stages(milora_ctx* ctx, int unit_stages);
 
 /* Several module call sites of one layer in a single launch (for example q,k,v share an input,
  * gate,up share an input).  modules[i], X_dev[i], Y_dev[i] describe site i; a module may appear once. */

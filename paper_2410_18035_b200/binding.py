@@ -45,6 +45,10 @@ class Groups(C.Structure):
     _fields_ = [("ws_dev", C.c_void_p), ("n_seq", C.c_int), ("T", C.c_int)]
 
 
+class DecodeLayer(C.Structure):
+    _fields_ = [("layer", C.c_int), ("groups", Groups), ("X_dev", C.c_void_p * 7), ("Y_dev", C.c_void_p * 7)]
+
+
 class HostStep(C.Structure):
     _fields_ = [("layer", C.c_int), ("n_prompts", C.c_int), ("cu_prompts_host", C.c_void_p),
                 ("prompt_slot_host", C.c_void_p), ("H_host", C.c_void_p), ("n_seq", C.c_int), ("T", C.c_int),
@@ -76,6 +80,8 @@ SIGNATURES = {
     "milora_group": (_I, [_VP, _I, _I, _VP, _VP, _I, _I, _VP, C.c_size_t, _VP]),
     "milora_set_decode_path": (_I, [_VP, _I]),
     "milora_decode_path_for": (_I, [_VP, _I, _I, C.POINTER(_I)]),
+    "milora_apply_decode_layers": (_I, [_VP, C.POINTER(DecodeLayer), _I, _VP]),
+    "milora_set_decode_unit_stages": (_I, [_VP, _I]),
     "milora_apply_decode": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_prefill": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_decode_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
@@ -306,8 +312,9 @@ class Milora:
             raise ValueError(f"apply: X/Y shapes {tuple(X.shape)}/{tuple(Y.shape)} do not fit module {module} with T={T}")
 
     def set_decode_path(self, path):
-        """milora_set_decode_path: 0 / "auto", 1 / "cluster" (one launch), 2 / "split" (two streaming launches)."""
-        code = {"auto": 0, "cluster": 1, "split": 2}.get(path, path)
+        """milora_set_decode_path: 0 / "auto", 1 / "cluster" (one launch), 2 / "split" (two streaming launches),
+        3 / "stream" (the persistent kernel of apply_decode_layers)."""
+        code = {"auto": 0, "cluster": 1, "split": 2, "stream": 3}.get(path, path)
         self._check(self.lib.milora_set_decode_path(self.h, int(code)), "milora_set_decode_path")
 
     def decode_path_for(self, n_seq, T):
@@ -315,6 +322,27 @@ class Milora:
         out = C.c_int(0)
         self._check(self.lib.milora_decode_path_for(self.h, n_seq, T, C.byref(out)), "milora_decode_path_for")
         return out.value
+
+    def set_decode_unit_stages(self, unit_stages):
+        self._check(self.lib.milora_set_decode_unit_stages(self.h, int(unit_stages)), "milora_set_decode_unit_stages")
+
+    def decode_layers(self, entries) -> "C.Array":
+        """Marshals [(layer, groups, {module: (X, Y)}), ...] into the milora_decode_layer array that
+        apply_decode_layers takes (build it once for a decode loop over fixed buffers)."""
+        arr = (DecodeLayer * len(entries))()
+        for i, (layer, groups, sites) in enumerate(entries):
+            arr[i].layer = layer
+            arr[i].groups = groups
+            for m, (X, Y) in sites.items():
+                self._xy(m, X, Y, groups.T)
+                arr[i].X_dev[m] = X.data_ptr()
+                arr[i].Y_dev[m] = Y.data_ptr()
+        return arr
+
+    def apply_decode_layers(self, layers, stream=None):
+        """milora_apply_decode_layers on an array made by decode_layers()."""
+        self._check(self.lib.milora_apply_decode_layers(self.h, layers, len(layers), _stream(stream)),
+                    "milora_apply_decode_layers")
 
     def apply_decode(self, layer, module, X, Y, groups: Groups, stream=None):
         self._xy(module, X, Y, groups.T)

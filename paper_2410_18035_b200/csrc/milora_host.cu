@@ -172,6 +172,10 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->d_dsplit = nullptr; ctx->dsplit_floats = 0; ctx->dsplit_dirty = true;
   ctx->dsplit_occ_s = 0; ctx->dsplit_occ_e = 0; ctx->decode_path = MILORA_DECODE_AUTO;
   ctx->copy_stream = nullptr; ctx->ev_done = nullptr; ctx->copy_ready = false;
+  ctx->d_stream = nullptr; ctx->stream_jobs_cap = 0; ctx->stream_frag_bytes = 0; ctx->stream_part_bytes = 0;
+  ctx->stream_dirty = true; ctx->stream_attr_set = false; ctx->stream_unit_stages = 0;
+  ctx->d_stream_layers = nullptr; ctx->h_stream_stage = nullptr; ctx->stream_stage_next = 0; ctx->stream_layers_cached = 0;
+  for (int i = 0; i < 4; ++i) ctx->stream_stage_ev[i] = nullptr;
   for (int m = 0; m < MILORA_NMOD; ++m) ctx->ev_site[m] = nullptr;
   ctx->n_counters = 0;
   milora_status st = MILORA_OK;
@@ -234,6 +238,11 @@ milora_status milora_destroy(milora_ctx* ctx) {
   cudaFree(ctx->d_vscratch);
   cudaFree(ctx->d_lin);
   cudaFree(ctx->d_dsplit);
+  cudaFree(ctx->d_stream);
+  cudaFree(ctx->d_stream_layers);
+  if (ctx->h_stream_stage) cudaFreeHost(ctx->h_stream_stage);
+  for (int i = 0; i < 4; ++i)
+    if (ctx->stream_stage_ev[i]) cudaEventDestroy(ctx->stream_stage_ev[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
   for (int m = 0; m < MILORA_NMOD; ++m)
@@ -260,13 +269,12 @@ milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, in
   int d1, d2;
   module_dims(ctx->desc, module, &d1, &d2);
   size_t idx = adapter_index(tenant, layer, module, ctx->desc.n_layers);
-  size_t bytes_a = ((size_t)rank * d1 * ctx->elem + 255) & ~size_t(255);
-  size_t bytes_b = ((size_t)rank * d2 * ctx->elem + 255) & ~size_t(255);
-  // tensor-core operand images (bf16 contexts, dimensions that fit the tiled kernels)
+  // tensor-core operand images (bf16 contexts, dimensions that fit the tiled kernels) follow A^T and B in the
+  // same allocation; adapter_layout is also what the kernels use to find them from a job record
   const bool images = prefill_images_supported(ctx, d1, d2, rank);
-  size_t bytes_ai = images ? (prefill_image_bytes(d1, rank) + 255) & ~size_t(255) : 0;
-  size_t bytes_bi = images ? (prefill_image_bytes(d2, rank) + 255) & ~size_t(255) : 0;
-  const size_t total = bytes_a + bytes_b + bytes_ai + bytes_bi;
+  const AdapterLayout lay = adapter_layout(d1, d2, rank, ctx->elem);
+  if (images != images_fit(d1, d2, rank, ctx->elem)) return MILORA_E_STATE;
+  const size_t total = lay.total;
   AdapterEntry& ent = ctx->h_adapters[idx];
   void* store = const_cast<void*>(ent.At);
   if (!store || ctx->adapter_bytes[idx] != total) {
@@ -276,9 +284,9 @@ milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, in
     ctx->adapter_bytes[idx] = total;
   }
   void* At = store;
-  void* Bs = static_cast<char*>(store) + bytes_a;
-  void* Ai = images ? static_cast<char*>(store) + bytes_a + bytes_b : nullptr;
-  void* Bi = images ? static_cast<char*>(store) + bytes_a + bytes_b + bytes_ai : nullptr;
+  void* Bs = static_cast<char*>(store) + lay.off_b;
+  void* Ai = images ? static_cast<char*>(store) + lay.off_a_img : nullptr;
+  void* Bi = images ? static_cast<char*>(store) + lay.off_b_img : nullptr;
   milora_status st = launch_repack_adapter(ctx, A_dev, B_dev, At, Bs, d1, d2, rank, as_stream(stream));
   if (st != MILORA_OK) return st;
   if (images) {
@@ -511,6 +519,7 @@ milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const
 // batch sweep: at 128 requests on 128 tenants the single launch is still 10 % faster, at 256 the pair is 12 %
 // faster; 13B shapes at 256 requests: 29 %).
 static milora_decode_path pick_decode_path(const milora_ctx* ctx, int n_seq, int T) {
+  if (ctx->decode_path == MILORA_DECODE_STREAM && !decode_stream_supported(ctx)) return MILORA_DECODE_CLUSTER;
   if (ctx->decode_path != MILORA_DECODE_AUTO) return (milora_decode_path)ctx->decode_path;
   const milora_group_layout_t lay = group_layout(n_seq, T, top_k_of(ctx));
   return lay.max_gather > 2 * ctx->sm_count ? MILORA_DECODE_SPLIT : MILORA_DECODE_CLUSTER;
@@ -520,6 +529,20 @@ milora_status milora_decode_path_for(const milora_ctx* ctx, int n_seq, int T, mi
   if (!ctx || !out || n_seq < 0 || T < 0) return MILORA_E_ARG;
   *out = pick_decode_path(ctx, n_seq, T);
   return MILORA_OK;
+}
+
+// The part of a layer record that follows from the group block alone.
+static StreamLayer stream_layer_of(const milora_ctx* ctx, const milora_groups* g) {
+  StreamLayer L;
+  std::memset(&L, 0, sizeof(L));
+  const milora_group_layout_t lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
+  L.ws = g->ws_dev;
+  L.off_header = (int32_t)lay.header;
+  L.off_mod_gather = (int32_t)lay.mod_gather_offset;
+  L.off_gather = (int32_t)lay.gather;
+  L.max_gather = lay.max_gather;
+  L.T = g->T;
+  return L;
 }
 
 static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const int* modules,
@@ -552,9 +575,18 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
       st = launch_apply_prefill_bf16(ctx, layer, sites, groups, s);
     } else {
       st = MILORA_E_SHAPE;
-      if (ctx->decode_path != MILORA_DECODE_CLUSTER) {
-        if (pick_decode_path(ctx, groups->n_seq, groups->T) == MILORA_DECODE_SPLIT)
-          st = launch_apply_decode_split(ctx, layer, sites, groups, s);
+      const milora_decode_path path = pick_decode_path(ctx, groups->n_seq, groups->T);
+      if (path == MILORA_DECODE_STREAM) {
+        StreamLayer one = stream_layer_of(ctx, groups);
+        bool aligned = true;
+        for (int i = 0; i < sites.n; ++i) {
+          one.X[sites.site[i].module] = sites.site[i].X;
+          one.Y[sites.site[i].module] = sites.site[i].Y;
+          aligned = aligned && !((reinterpret_cast<uintptr_t>(sites.site[i].X) | reinterpret_cast<uintptr_t>(sites.site[i].Y)) & 15);
+        }
+        if (aligned) st = launch_apply_decode_stream(ctx, &one, 1, groups->n_seq, s);
+      } else if (path == MILORA_DECODE_SPLIT) {
+        st = launch_apply_decode_split(ctx, layer, sites, groups, s);
       }
       if (st == MILORA_E_SHAPE) st = launch_apply_decode_bf16(ctx, layer, sites, groups, s);
     }
@@ -565,8 +597,75 @@ static milora_status apply_common(milora_ctx* ctx, int layer, int n_sites, const
 
 milora_status milora_set_decode_path(milora_ctx* ctx, milora_decode_path path) {
   if (!ctx) return MILORA_E_ARG;
-  if (path != MILORA_DECODE_AUTO && path != MILORA_DECODE_CLUSTER && path != MILORA_DECODE_SPLIT) return MILORA_E_ARG;
+  if (path != MILORA_DECODE_AUTO && path != MILORA_DECODE_CLUSTER && path != MILORA_DECODE_SPLIT &&
+      path != MILORA_DECODE_STREAM)
+    return MILORA_E_ARG;
   ctx->decode_path = (int)path;
+  return MILORA_OK;
+}
+
+milora_status milora_set_decode_unit_stages(milora_ctx* ctx, int unit_stages) {
+  if (!ctx || unit_stages < 0 || unit_stages > 64) return MILORA_E_ARG;
+  ctx->stream_unit_stages = unit_stages;
+  return MILORA_OK;
+}
+
+milora_status milora_apply_decode_layers(milora_ctx* ctx, const milora_decode_layer* layers, int n_layers, void* stream) {
+  if (!ctx || n_layers < 0 || (n_layers > 0 && !layers)) return MILORA_E_ARG;
+  if (n_layers == 0) return MILORA_OK;
+  std::vector<StreamLayer> recs;
+  std::vector<int> keep;
+  try {
+    recs.reserve(n_layers);
+    keep.reserve(n_layers);
+  } catch (...) {
+    return MILORA_E_CAPACITY;
+  }
+  int n_seq_hint = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    const milora_decode_layer& d = layers[i];
+    if (d.layer < 0 || d.layer >= ctx->desc.n_layers) return MILORA_E_ARG;
+    const milora_groups& g = d.groups;
+    if (!g.ws_dev || g.n_seq < 0 || g.T < 0 || (long long)g.n_seq * top_k_of(ctx) > kMaxSeq) return MILORA_E_ARG;
+    bool any = false;
+    for (int m = 0; m < MILORA_NMOD; ++m) {
+      if ((d.X_dev[m] == nullptr) != (d.Y_dev[m] == nullptr)) return MILORA_E_ARG;
+      any = any || d.X_dev[m];
+    }
+    if (!any || g.T == 0 || g.n_seq == 0) continue;
+    StreamLayer L = stream_layer_of(ctx, &g);
+    for (int m = 0; m < MILORA_NMOD; ++m) {
+      L.X[m] = d.X_dev[m];
+      L.Y[m] = d.Y_dev[m];
+    }
+    recs.push_back(L);
+    keep.push_back(i);
+    n_seq_hint = std::max(n_seq_hint, g.n_seq);
+  }
+  if (recs.empty()) return MILORA_OK;
+  cudaStream_t s = as_stream(stream);
+  milora_status st = sync_tables(ctx, s);
+  if (st != MILORA_OK) return st;
+  bool aligned = true;
+  for (const StreamLayer& L : recs)
+    for (int m = 0; m < MILORA_NMOD; ++m)
+      aligned = aligned && !((reinterpret_cast<uintptr_t>(L.X[m]) | reinterpret_cast<uintptr_t>(L.Y[m])) & 15);
+  if (decode_stream_supported(ctx) && aligned && ctx->decode_path != MILORA_DECODE_CLUSTER &&
+      ctx->decode_path != MILORA_DECODE_SPLIT) {
+    st = launch_apply_decode_stream(ctx, recs.data(), (int)recs.size(), n_seq_hint, s);
+    if (st != MILORA_E_SHAPE) return st;
+  }
+  // shapes, dtype or a forced kernel set that the persistent kernel does not cover: one call per layer
+  for (int i : keep) {
+    const milora_decode_layer& d = layers[i];
+    int mods[MILORA_NMOD], n = 0;
+    const void* X[MILORA_NMOD];
+    void* Y[MILORA_NMOD];
+    for (int m = 0; m < MILORA_NMOD; ++m)
+      if (d.X_dev[m]) { mods[n] = m; X[n] = d.X_dev[m]; Y[n] = d.Y_dev[m]; ++n; }
+    st = apply_common(ctx, d.layer, n, mods, X, Y, &d.groups, false, stream);
+    if (st != MILORA_OK) return st;
+  }
   return MILORA_OK;
 }
 
@@ -730,6 +829,11 @@ milora_status milora_poll_error(milora_ctx* ctx, int* device_flag_out, void* str
   int32_t flag = 0;
   MILORA_CUDA(ctx, cudaMemcpyAsync(&flag, ctx->d_err, sizeof(flag), cudaMemcpyDeviceToHost, s));
   MILORA_CUDA(ctx, cudaStreamSynchronize(s));
+  if (flag & ERR_WAIT_TIMEOUT) {
+    // a kernel gave up on a wait: its self-cleaning counters may not be back at zero
+    ctx->stream_dirty = true;
+    ctx->dsplit_dirty = true;
+  }
   if (flag) {
     MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_err, 0, sizeof(int32_t), s));
     MILORA_CUDA(ctx, cudaStreamSynchronize(s));

@@ -87,6 +87,39 @@ __host__ __device__ inline size_t adapter_index(int tenant, int layer, int modul
   return ((size_t)tenant * n_layers + layer) * MILORA_NMOD + module;
 }
 
+// Where the four parts of one registered adapter sit inside its single pool allocation: A^T (rank x d1), B
+// (rank x d2), then, when the operand images exist, the A image and the B image; every part starts on a 256-byte
+// boundary.  Registration and the kernels that find the images from a job record's `At` use this one function.
+constexpr int kImagePadMax = 64;   // largest padded rank that gets operand images
+struct AdapterLayout {
+  size_t off_b, off_a_img, off_b_img, total;
+};
+__host__ __device__ inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+__host__ __device__ inline bool images_fit(int d1, int d2, int rank, size_t elem) {
+  return elem == 2 && d1 % 64 == 0 && d2 % 128 == 0 && rank >= 1 && rank <= kImagePadMax;
+}
+__host__ __device__ inline AdapterLayout adapter_layout(int d1, int d2, int rank, size_t elem) {
+  AdapterLayout L;
+  const size_t rp = (size_t)((rank + 15) & ~15);
+  const bool img = images_fit(d1, d2, rank, elem);
+  L.off_b = align256((size_t)rank * d1 * elem);
+  L.off_a_img = L.off_b + align256((size_t)rank * d2 * elem);
+  L.off_b_img = L.off_a_img + (img ? align256((size_t)d1 * rp * 2) : 0);
+  L.total = L.off_b_img + (img ? align256((size_t)d2 * rp * 2) : 0);
+  return L;
+}
+
+// One layer of a multi-layer decode launch (apply_decode_stream.cu), as the kernel reads it.
+constexpr int kMaxStreamLayers = 40;
+struct StreamLayer {
+  const int32_t* ws;                 // the layer's group block
+  const void* X[MILORA_NMOD];        // nullptr: the module is skipped
+  void* Y[MILORA_NMOD];
+  int32_t off_header, off_mod_gather, off_gather, max_gather;   // int32 offsets into ws, capacity of the gather list
+  int32_t T, job_base;               // rows of X / Y; first job slot of the layer in the launch's scratch arrays
+};
+static_assert(sizeof(StreamLayer) == 144, "StreamLayer is copied as 9 x 16 bytes");
+
 struct Arena {
   struct Chunk { char* base; size_t size, used; };
   std::vector<Chunk> chunks;
@@ -126,6 +159,16 @@ struct milora_ctx {
   bool dsplit_dirty;                            // counters must be cleared before the next launch pair
   int dsplit_occ_s, dsplit_occ_e;               // resident CTAs per SM of its two kernels (0 = not asked yet)
   int decode_path;                              // milora_decode_path
+  // persistent multi-layer decode kernel (apply_decode_stream.cu)
+  void* d_stream;                               // control words, job states, v fragments, partial sums
+  size_t stream_jobs_cap, stream_frag_bytes, stream_part_bytes;   // what d_stream is laid out for
+  bool stream_dirty;                            // job states must be cleared before the next launch
+  bool stream_attr_set;
+  int stream_unit_stages;                       // stages per unit; 0 = chosen from the batch size
+  void* d_stream_layers;                        // layer records of a multi-layer launch
+  void* h_stream_stage;                         // pinned: four staging copies of those records
+  cudaEvent_t stream_stage_ev[4];
+  int stream_stage_next, stream_layers_cached;
   void* d_lin;                                  // fused projection: V piece images and per-row-block piece lists
   size_t lin_bytes;
   cudaStream_t copy_stream;                     // milora_step_host: device-to-host copies run beside the uploads
@@ -213,6 +256,12 @@ milora_status launch_apply_decode_bf16(milora_ctx* ctx, int layer, const ApplySi
 // take equally sized units from a counter; v goes through a scratch buffer of the context.  Same convention.
 milora_status launch_apply_decode_split(milora_ctx* ctx, int layer, const ApplySites& sites, const milora_groups* g,
                                         cudaStream_t s);
+
+// bf16 decode path as one persistent launch over any number of layers (operand images, bulk-copy rings).
+// `layers` is a host array whose job_base fields the call fills in.  Same MILORA_E_SHAPE convention.
+bool decode_stream_supported(const milora_ctx* ctx);
+milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, int n_layers, int n_seq_hint,
+                                         cudaStream_t s);
 
 // bf16 prefill path: tcgen05 shrink and expand kernels over the dense tiles (same MILORA_E_SHAPE convention),
 // and the registration-time packing of the operand images they read.

@@ -137,8 +137,9 @@ RAGGED = [1, 33, 130, 257, 31, 32, 7, 129]
 
 @pytest.mark.parametrize("dtype,d,d_ff,d_kv,r", [("f32", 256, 688, 256, 8), ("bf16", 512, 1376, 128, 16),
                                                  ("bf16", 256, 688, 256, 40), ("bf16", 1024, 2816, 256, 16),
-                                                 ("bf16", 512, 1408, 512, 32), ("bf16", 512, 1408, 128, 64)])
-@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+                                                 ("bf16", 512, 1408, 512, 32), ("bf16", 512, 1408, 128, 64),
+                                                 ("bf16", 256, 768, 256, 40)])
+@pytest.mark.parametrize("decode_path", ["cluster", "split", "stream"])
 def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r, decode_path):
     """Sequences of 1..257 rows (both work lists, ragged tile tails) mixed with decode rows; tenants repeat so
     that several sequences share a bucket; one slot is closed and one tenant has no adapters."""
@@ -316,7 +317,7 @@ def test_fused_projection_refuses_what_it_cannot_run():
     ml.close()
 
 
-@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+@pytest.mark.parametrize("decode_path", ["cluster", "split", "stream"])
 def test_back_to_back_launches_equal_serialised_ones_bit_for_bit(decode_path):
     """Every kernel may start while the one before it is still draining (programmatic dependent launch) and takes
     its work from device-side lists.  The results must not depend on that: the whole step enqueued back to back,
@@ -430,24 +431,25 @@ def test_group_edge_cases_and_device_flags():
     lw.close()
 
 
-@pytest.mark.parametrize("decode_path", ["cluster", "split"])
+@pytest.mark.parametrize("decode_path", ["cluster", "split", "stream"])
 def test_decode_kernel_sets_edge_cases(decode_path):
-    """Both decode kernel sets: a batch without any short sequence (empty gathered list) leaves every row
+    """Every decode kernel set: a batch without any short sequence (empty gathered list) leaves every row
     bit-identical; the same decode batch applied five times in a row (the two-launch set hands its unit counters
     from one call to the next) gives bit-identical results each time, equal to the oracle's; a set other than
-    the three named ones is refused."""
+    the named ones is refused."""
     from paper_2410_18035_b200 import MiloraError
     base = get_workload("c1")
     lens = np.array([40, 64] + [1] * 9, dtype=np.int32)
     n = len(lens)
     tenants = (np.arange(n) % 3).astype(np.int32)
-    w = scaled_workload(base, name="decode_edges", dtype="bf16", d_model=512, d_ff=1376, d_kv=128, rank=24, n_tenants=3,
+    d_ff = 1408 if decode_path == "stream" else 1376      # the persistent kernel wants multiples of 128
+    w = scaled_workload(base, name="decode_edges", dtype="bf16", d_model=512, d_ff=d_ff, d_kv=128, rank=24, n_tenants=3,
                         request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(2), decode_ids=np.arange(2, n),
                         has_base_weights=False, n_layers=1)
     lw = _loaded(w)
     ml = lw.ml
     with pytest.raises(MiloraError):
-        ml.set_decode_path(3)
+        ml.set_decode_path(4)
     ml.set_decode_path(decode_path)
     ids = list(range(n))
     lw.route(0, ids)
@@ -486,6 +488,63 @@ def test_decode_kernel_sets_edge_cases(decode_path):
         else:
             for m in range(7):
                 assert torch.equal(Ys[m], first[m]), f"call {rep}, module {m}: result changed between calls"
+    assert ml.poll_error() == 0
+    lw.close()
+
+
+@pytest.mark.parametrize("d,d_ff,d_kv,r,n_dec,unit_stages", [(512, 1408, 128, 16, 37, 0), (1024, 2816, 256, 32, 70, 1),
+                                                             (512, 1536, 512, 48, 9, 3), (256, 688, 256, 8, 12, 0)])
+def test_decode_layers_one_launch(d, d_ff, d_kv, r, n_dec, unit_stages):
+    """milora_apply_decode_layers: three layers with their own routes, adapters and outputs in ONE call, against
+    the oracle layer by layer; tenants repeat (jobs of up to four rows, several jobs per adapter), one layer skips
+    two modules (NULL pair: those outputs stay bit-identical), and repeated calls give bit-identical results (the
+    kernel's job states and unit counter clean themselves up).  The last shape does not fit the persistent kernel
+    and takes the per-layer calls behind the same entry point."""
+    base = get_workload("c1")
+    L = 3
+    lens = np.full(n_dec, 8, dtype=np.int32)
+    tenants = (np.arange(n_dec) * 7 % 5).astype(np.int32)
+    w = scaled_workload(base, name="decode_layers", dtype="bf16", d_model=d, d_ff=d_ff, d_kv=d_kv, rank=r, n_tenants=5,
+                        request_tenant=tenants, prompt_len=lens, prefill_ids=np.arange(0), decode_ids=np.arange(n_dec),
+                        has_base_weights=False, n_layers=L)
+    lw = _loaded(w)
+    ml = lw.ml
+    ml.set_decode_unit_stages(unit_stages)
+    ids = list(range(n_dec))
+    for li in range(L):
+        for i0 in range(0, n_dec, 32):
+            lw.route(li, ids[i0:i0 + 32])
+    table = ml.route_table_read(0, n_dec).numpy().copy()
+    cu, slots, T = lw.seq_arrays([], ids)
+    ws = ml.alloc_group_ws(L, n_dec, T)
+    ml.group(0, L, cu, slots, n_dec, T, ws)
+    token_slot = slots.cpu().numpy()
+    Xs = [[w.module_input(li, m, T, 20 + li, "cuda") for m in range(7)] for li in range(L)]
+    Ybs = [[w.base_output(li, m, T, 20 + li, "cuda") for m in range(7)] for li in range(L)]
+    skipped = {1: (2, 5)}
+    first = None
+    for rep in range(3):
+        Ys = [[y.clone() for y in row] for row in Ybs]
+        entries = []
+        for li in range(L):
+            sites = {m: (Xs[li][m], Ys[li][m]) for m in range(7) if m not in skipped.get(li, ())}
+            entries.append((li, ml.groups(ws[li], n_dec, T), sites))
+        ml.apply_decode_layers(ml.decode_layers(entries))
+        torch.cuda.synchronize()
+        if first is None:
+            first = Ys
+            for li in range(L):
+                for m in range(7):
+                    if m in skipped.get(li, ()):
+                        assert torch.equal(Ys[li][m], Ybs[li][m])
+                        continue
+                    y_o = R.apply_site(w, li, m, Xs[li][m].cpu(), Ybs[li][m].cpu(), token_slot, table[:, li])
+                    assert_apply_close(Ys[li][m], y_o, Ybs[li][m], "bf16", what=f"decode layers: layer {li} module {m}")
+        else:
+            for li in range(L):
+                for m in range(7):
+                    assert torch.equal(Ys[li][m], first[li][m]), f"call {rep}, layer {li}, module {m}"
+    assert any((first[li][m] != Ybs[li][m]).any() for li in range(L) for m in range(7))
     assert ml.poll_error() == 0
     lw.close()
 
