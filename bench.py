@@ -408,13 +408,14 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
         for li in range(n_layers):
             ml.apply_decode_multi(li, mods, Xd, Yd, groups[li])
 
-    def timed():
+    def timed(fn=None):
+        fn = fn or one_round
         for _ in range(3):
-            one_round()
+            fn()
         torch.cuda.synchronize(device)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            one_round()
+            fn()
         graph.replay()
         torch.cuda.synchronize(device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -431,12 +432,18 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
         return {"us_per_layer": ms * 1e3, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
                 "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "decode_token_layers_per_s": n / (ms * 1e-3)}
 
-    # both kernel sets on the same chain, then the library's own choice (the figures reported at the top level)
+    # the kernel sets on the same chain (one call per layer), the whole chain as ONE call of
+    # milora_apply_decode_layers (every layer its own outputs: the layers of one call run concurrently), then the
+    # library's own choice for per-layer calls (the figures reported at the top level)
     by_path = {}
-    for path in ("cluster", "split"):
+    for path in ("cluster", "split", "stream"):
         ml.set_decode_path(path)
         by_path[path] = figures(timed())
     ml.set_decode_path("auto")
+    Yl = [[y.clone() for y in Yd] for _ in range(n_layers)]
+    entries = [(li, groups[li], {m: (Xd[m], Yl[li][m]) for m in mods}) for li in range(n_layers)]
+    layers_arr = ml.decode_layers(entries)
+    one_call = figures(timed(lambda: ml.apply_decode_layers(layers_arr)))
     ms = timed()
     err = ml.poll_error()
     top = figures(ms)
@@ -446,7 +453,7 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
             "gbs": top["gbs"], "frac_of_measured_hbm": top["frac_of_measured_hbm"],
             "frac_of_8TBs_nominal": top["frac_of_8TBs_nominal"],
             "decode_token_layers_per_s": top["decode_token_layers_per_s"], "device_error_flag": err,
-            "by_decode_path": by_path}
+            "by_decode_path": by_path, "one_call_all_layers": one_call}
 
 
 def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):

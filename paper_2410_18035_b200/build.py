@@ -65,7 +65,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
             rebuilt = True
-    if rebuilt or force or not os.path.exists(LIB):
+    if rebuilt or force or not os.path.exists(LIB) or os.path.getmtime(LIB) < _newest(objs):
         cmd = [nvcc, "-shared", "-o", LIB, *objs, "-lcuda"]
         if verbose:
             print(" ".join(cmd), flush=True)

@@ -23,8 +23,9 @@
 //     8 x 16-byte core matrices, exactly what ldmatrix reads without bank conflicts).  The path is bound by the
 //     adapter stream; the tensor cores are used for the instruction count.
 //     shrink: M = rank rows, N = rows of x, K = columns of d1.
-//     expand: M = columns of d2, N = (row t, value | remainder), K = rank rows; y is updated in shared memory and
-//     written back with one bulk store per row.
+//     expand: M = columns of d2, N = (row t, value | remainder), K = rank rows; the products are added to y with
+//     red.global.add.noftz.bf16: y never travels to the SM, every element of y receives exactly one addition
+//     (deterministic), and its error is half an ulp of y plus the bf16 rounding of the term (2^-9 of it).
 //   * The job states and the unit counter clean themselves up (last expand unit of a job, last worker of the grid),
 //     so a launch leaves the scratch ready for the next one.
 #include <algorithm>
@@ -39,19 +40,25 @@ namespace {
 using namespace ptx;
 
 constexpr int kR = kGatherRows;
-constexpr int kWarps = 5;                        // worker warps per CTA
 constexpr int kBufs = 2;                         // buffers (stages in flight) per worker
-constexpr int kThreads = kWarps * 32;
-constexpr int kStageBytes = 16384;               // adapter bytes per stage
-constexpr int kRowBytesMax = kStageBytes / 16;   // a row of x / y per stage: cols * 2 bytes, cols <= kStageBytes / 32
 constexpr int kRowPad = 16;                      // keeps the rows of one stage on different banks
-constexpr int kBufBytes = kStageBytes + kR * (kRowBytesMax + kRowPad);
-constexpr int kBufStride = (kBufBytes + 127) & ~127;
 constexpr int kStaticRounds = 2;                 // units per worker assigned by index before the counter is used
 constexpr int kUnitRing = 4;                     // unit records a worker keeps (issue runs ahead of compute)
 constexpr int kMaxSeg = 2 * kMaxStreamLayers * MILORA_NMOD;
-constexpr uint32_t kReady = 0x80000000u;
 constexpr uint32_t kDepSpin = 1u << 22;          // polls of a job's ready flag before an expand unit gives up
+constexpr int kMaxWarps = 10;
+
+// Two shapes of the kernel: many warps on small stages for the usual ranks (the warps hide each other's
+// latencies; 20 stages of 8 KB in flight per SM), fewer warps on 16 KB stages for padded ranks of 48 and 64,
+// whose smallest stage (one 128-column block of B) no longer fits 8 KB.
+template <int WARPS, int STAGE>
+struct Shape {
+  static constexpr int kWarps = WARPS;
+  static constexpr int kStageBytes = STAGE;
+  static constexpr int kThreads = WARPS * 32;
+};
+using ShapeSmall = Shape<10, 8192>;
+using ShapeLarge = Shape<6, 16384>;
 
 struct StreamArgs {
   int32_t* err;
@@ -61,12 +68,15 @@ struct StreamArgs {
   int d1[MILORA_NMOD], d2[MILORA_NMOD];
   int rp;                      // rank pad of the context: fixes the columns per stage
   int cols;                    // columns of d1 / d2 per stage
+  int stage_bytes;             // adapter bytes per stage (the rows of x follow them in a buffer)
+  int buf_stride;              // bytes from one buffer to the next: stage + kR rows of x, rounded up
   int unit_stages;             // stages per unit
   int kcmax;                   // most shrink units per job over the modules
   uint32_t* ctrl;              // [0] units handed out beyond the static rounds, [1] workers that have finished
-  uint32_t* job_state;         // [jobs][2]: shrink units arrived | kReady, expand units done
+  uint32_t* job_state;         // [jobs]: shrink units of the job that have delivered their partial sums
+  uint32_t epoch;              // tag of this launch (never 0): marks the fragments written by it
   float* partial;              // [jobs][kcmax][kR][rp]
-  uint2* vfrag;                // [jobs][rp / 16][32]
+  uint4* vfrag;                // [jobs][rp / 16][32] of {word 0, epoch, word 1, epoch}
 };
 
 struct UnitRec {               // what a worker needs to know about a unit, in shared memory
@@ -87,10 +97,9 @@ struct Smem {
   int32_t seg_base[kMaxSeg + 1];
   int32_t first[kMaxStreamLayers][MILORA_NMOD + 1];
   int32_t upj[2][MILORA_NMOD];
-  UnitRec unit[kWarps][kUnitRing];
-  float vsum[kWarps][kR][kImagePadMax];
-  uint64_t full[kWarps][kBufs];
-  int32_t buf_unit[kWarps][kBufs], buf_stage[kWarps][kBufs];
+  UnitRec unit[kMaxWarps][kUnitRing];
+  uint64_t full[kMaxWarps][kBufs];
+  int32_t buf_unit[kMaxWarps][kBufs], buf_stage[kMaxWarps][kBufs];
 };
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -109,28 +118,33 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
-  uint16_t v;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ void sts16(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
-}
-__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
+}
+// Two neighbouring elements of y += (v0, v1) in bf16, performed by the L2 (one rounding of each sum).  The packed
+// form is a native operation; the scalar bf16 form is not (measured: 40 us for one row of 4096 columns).
+__device__ __forceinline__ void red_add_bf16x2(void* addr, float v0, float v1) {
+  const uint32_t h = pack_bf16(v0, v1);
+  asm volatile("red.global.add.noftz.bf16x2 [%0], %1;" ::"l"(addr), "r"(h) : "memory");
+}
+// counts on a job; release for this warp's earlier writes, acquire for the other units' partial sums
+__device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+// A fragment word travels together with the tag of the launch that wrote it, as one 8-byte access (8-byte
+// accesses are single-copy atomic): whoever reads the right tag has the right word, without a flag or a fence.
+__device__ __forceinline__ void st_tagged(uint4* p, uint32_t w0, uint32_t w1, uint32_t tag) {
+  asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(w0), "r"(tag) : "memory");
+  asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(reinterpret_cast<char*>(p) + 8), "r"(w1), "r"(tag) : "memory");
+}
+__device__ __forceinline__ uint4 ld_tagged(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.z), "=r"(v.w) : "l"(reinterpret_cast<const char*>(p) + 8) : "memory");
+  return v;
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
@@ -144,34 +158,46 @@ __device__ __forceinline__ void pos_to_layer(int p, int L, int* li, int* phase) 
 }
 
 // ---- unit look-up ------------------------------------------------------------------------------------
-// Fills `r` for unit u (all lanes compute the same values; lanes 0..3 fetch the 64-byte job record).
-__device__ __forceinline__ void decode_unit(const StreamArgs& a, const Smem& sm, int n_seg, int u, UnitRec* r, int lane) {
+// In two halves, so that the 64-byte job record travels while the worker does something else: locate_unit finds
+// the unit's place in the work lists and asks for the record (lanes 0..3, 16 bytes each); fill_unit, called when the
+// worker needs the unit, hands the pieces around the warp, checks the record and writes the unit record.
+struct UnitLoc {
+  int li, phase, m, job_local, sub;
+  uint4 piece;
+};
+__device__ __forceinline__ UnitLoc locate_unit(const StreamArgs& a, const Smem& sm, int n_seg, int u, int lane) {
   // segment = (queue position, module): binary search over the prefix table
   int lo = 0, hi = n_seg;
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (sm.seg_base[mid] <= u) lo = mid; else hi = mid;
   }
-  const int p = lo / MILORA_NMOD, m = lo % MILORA_NMOD;
-  int li, phase;
-  pos_to_layer(p, a.n_layers, &li, &phase);
+  UnitLoc x;
+  const int p = lo / MILORA_NMOD;
+  x.m = lo % MILORA_NMOD;
+  pos_to_layer(p, a.n_layers, &x.li, &x.phase);
   const int local = u - sm.seg_base[lo];
-  const int upj = sm.upj[phase][m];
-  const int job_local = sm.first[li][m] + local / upj, sub = local % upj;
-  const StreamLayer& L = sm.layers[li];
-  // the job record: four 16-byte pieces, one per lane, then handed around the warp
-  const uint4* jp = reinterpret_cast<const uint4*>(L.ws + L.off_gather) + (size_t)job_local * (kJobInts / 4);
-  uint4 piece = make_uint4(0, 0, 0, 0);
-  if (lane < 4) piece = jp[lane];
+  const int upj = sm.upj[x.phase][x.m];
+  x.job_local = sm.first[x.li][x.m] + local / upj;
+  x.sub = local % upj;
+  const StreamLayer& L = sm.layers[x.li];
+  const uint4* jp = reinterpret_cast<const uint4*>(L.ws + L.off_gather) + (size_t)x.job_local * (kJobInts / 4);
+  x.piece = make_uint4(0, 0, 0, 0);
+  if (lane < 4) x.piece = jp[lane];
+  return x;
+}
+__device__ __forceinline__ void fill_unit(const StreamArgs& a, const Smem& sm, const UnitLoc& x, UnitRec* r, int lane) {
   GatherJob job;
   uint32_t* jw = reinterpret_cast<uint32_t*>(&job);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    jw[4 * i + 0] = __shfl_sync(0xffffffffu, piece.x, i);
-    jw[4 * i + 1] = __shfl_sync(0xffffffffu, piece.y, i);
-    jw[4 * i + 2] = __shfl_sync(0xffffffffu, piece.z, i);
-    jw[4 * i + 3] = __shfl_sync(0xffffffffu, piece.w, i);
+    jw[4 * i + 0] = __shfl_sync(0xffffffffu, x.piece.x, i);
+    jw[4 * i + 1] = __shfl_sync(0xffffffffu, x.piece.y, i);
+    jw[4 * i + 2] = __shfl_sync(0xffffffffu, x.piece.z, i);
+    jw[4 * i + 3] = __shfl_sync(0xffffffffu, x.piece.w, i);
   }
+  const StreamLayer& L = sm.layers[x.li];
+  const int m = x.m, phase = x.phase;
   const int d1 = a.d1[m], d2 = a.d2[m];
   const int rpj = (job.rank + 15) & ~15;
   bool ok = job.rank > 0 && rpj <= a.rp && job.count > 0 && job.count <= kR && job.At != nullptr && job.module == m &&
@@ -190,189 +216,222 @@ __device__ __forceinline__ void decode_unit(const StreamArgs& a, const Smem& sm,
     r->scale = job.scale;
     r->n = job.count; r->rp = rpj; r->rank = job.rank;
     r->d = d; r->phase = phase; r->module = m;
-    r->stage0 = sub * a.unit_stages;
-    r->n_stages = min(a.unit_stages, stages - sub * a.unit_stages);
-    r->job = L.job_base + job_local; r->sub = sub;
+    r->stage0 = x.sub * a.unit_stages;
+    r->n_stages = min(a.unit_stages, stages - x.sub * a.unit_stages);
+    r->job = L.job_base + x.job_local; r->sub = x.sub;
     r->upj_s = sm.upj[0][m]; r->upj_e = sm.upj[1][m];
     r->ok = ok ? 1 : 0;
   }
 }
 
 // ---- issue: the copies of one stage -------------------------------------------------------------------
-// Lane 0 only.  buf: shared address of the buffer; bar: its mbarrier.
-__device__ __forceinline__ void issue_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf, uint32_t bar,
-                                            bool rows_too) {
+// Lane 0 only.  buf: shared address of the buffer; bar: its mbarrier.  A shrink stage also brings the job's rows
+// of x; an expand stage needs nothing but its piece of the B image (y is updated in place in global memory).
+__device__ __forceinline__ void issue_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf, uint32_t bar) {
   const int c0 = (r.stage0 + stage_in_unit) * a.cols;
   const int ncols = min(a.cols, r.d - c0);
   // both images are contiguous in column order: rp * 2 bytes per column
   const uint32_t bytes_img = (uint32_t)ncols * r.rp * 2;
   const uint32_t bytes_row = (uint32_t)ncols * 2;
-  if (!rows_too) {
-    mbar_expect_tx(bar, bytes_img + (uint32_t)r.n * bytes_row);
-    bulk_g2s(buf, r.img + (size_t)c0 * r.rp * 2, bytes_img, bar);
-  } else {
-    const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
-    for (int t = 0; t < r.n; ++t)
-      bulk_g2s(buf + kStageBytes + t * rstride, r.rows_base + ((size_t)r.rows[t] * r.d + c0) * 2, bytes_row, bar);
-  }
+  const int n_rows = r.phase == 0 ? r.n : 0;
+  mbar_expect_tx(bar, bytes_img + (uint32_t)n_rows * bytes_row);
+  bulk_g2s(buf, r.img + (size_t)c0 * r.rp * 2, bytes_img, bar);
+  const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
+  for (int t = 0; t < n_rows; ++t)
+    bulk_g2s(buf + a.stage_bytes + t * rstride, r.rows_base + ((size_t)r.rows[t] * r.d + c0) * 2, bytes_row, bar);
 }
 
 // ---- shrink: one stage into the unit's accumulators ---------------------------------------------------------
-// acc[jb] is the 16 x 8 tile (rank rows jb*16.., rows of x) of this lane: c0, c1 = (rank row g, x rows 2q, 2q+1),
+// JB = rank blocks of 16.  The instructions of one 64-column chunk are grouped by kind (x fragments, ldmatrix, MMA)
+// so that independent ones follow each other: the asm statements keep their order, and a chain
+// ldmatrix -> mma -> next ldmatrix would run at one latency per step.  Consecutive k steps go to kAcc independent
+// accumulator sets, which are added when the unit ends.
+// acc[s * JB + jb] is a 16 x 8 tile (rank rows jb*16.., rows of x): c0, c1 = (rank row g, x rows 2q, 2q+1),
 // c2, c3 = (rank row g + 8, same x rows).
+constexpr int kAccSets = 8;     // accumulator tiles a worker holds: steps-per-batch x JB
+template <int JB>
 __device__ __forceinline__ void shrink_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf,
-                                             float (&acc)[kImagePadMax / 16][4], int lane) {
+                                             float (&acc)[kAccSets][4], int lane) {
+  constexpr int SB = JB <= 2 ? 4 : 2;          // k steps whose loads are issued together
   const int g = lane >> 2, q = lane & 3, mi = lane >> 3;
   const int c0 = (r.stage0 + stage_in_unit) * a.cols;
   const int ncols = min(a.cols, r.d - c0);
-  const int rp = r.rp, jblocks = rp >> 4;
+  constexpr int rp = JB * 16;
   const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
   const bool x_ok = g < r.n;
-  const uint32_t xrow = buf + kStageBytes + (x_ok ? g : 0) * rstride + 4 * q;
+  const uint32_t xrow = buf + a.stage_bytes + (x_ok ? g : 0) * rstride + 4 * q;
   // ldmatrix row address of this lane inside a 64-column chunk, for k step 0 and rank block 0
   const uint32_t lane_off = (uint32_t)(((mi >> 1) * (rp >> 3) + (mi & 1)) * 128 + (lane & 7) * 16);
   for (int kc = 0; kc < (ncols >> 6); ++kc) {
     const uint32_t chunk = buf + (uint32_t)kc * rp * 128 + lane_off;
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      uint32_t b0 = 0, b1 = 0;
-      if (x_ok) {
-        b0 = lds32(xrow + (kc * 64 + s * 16) * 2);
-        b1 = lds32(xrow + (kc * 64 + s * 16 + 8) * 2);
-      }
+    for (int s0 = 0; s0 < 4; s0 += SB) {
+      uint32_t b0[SB], b1[SB], am[SB][JB][4];
 #pragma unroll
-      for (int jb = 0; jb < kImagePadMax / 16; ++jb) {
-        if (jb < jblocks) {
-          uint32_t a0, a1, a2, a3;
-          ldmatrix_x4(chunk + (uint32_t)((2 * s) * (rp >> 3) + 2 * jb) * 128, a0, a1, a2, a3);
-          mma_16816(acc[jb], a0, a1, a2, a3, b0, b1);
+      for (int s = 0; s < SB; ++s) {
+        b0[s] = b1[s] = 0;
+        if (x_ok) {
+          b0[s] = lds32(xrow + (kc * 64 + (s0 + s) * 16) * 2);
+          b1[s] = lds32(xrow + (kc * 64 + (s0 + s) * 16 + 8) * 2);
         }
       }
+#pragma unroll
+      for (int s = 0; s < SB; ++s)
+#pragma unroll
+        for (int jb = 0; jb < JB; ++jb)
+          ldmatrix_x4(chunk + (uint32_t)((2 * (s0 + s)) * (rp >> 3) + 2 * jb) * 128, am[s][jb][0], am[s][jb][1], am[s][jb][2],
+                      am[s][jb][3]);
+#pragma unroll
+      for (int s = 0; s < SB; ++s)
+#pragma unroll
+        for (int jb = 0; jb < JB; ++jb)
+          mma_16816(acc[s * JB + jb], am[s][jb][0], am[s][jb][1], am[s][jb][2], am[s][jb][3], b0[s], b1[s]);
     }
   }
 }
 
-// End of a shrink unit: partial products to scratch, count on the job; the last unit of the job adds them up in
-// unit order and publishes v as the fragments of the expand MMAs.
-__device__ __forceinline__ void shrink_finish(const StreamArgs& a, const UnitRec& r, float (&acc)[kImagePadMax / 16][4],
-                                              float (*vsum)[kImagePadMax], int lane) {
+// End of a shrink unit, first half: partial products to scratch and one count on the job.  The answer of the count
+// (lane 0) is not looked at here: the worker goes on with its next stage and calls shrink_finalize afterwards, so
+// the round trip of the atomic is not on its path.
+struct PendingCount {
+  uint32_t old;          // lane 0: units of the job that had arrived before this one
+  int32_t job, upj_s, jb;
+  float w;               // scale * gate of this lane's row of v (row t = lane / 8), 0 beyond the job's rows
+  bool valid;
+};
+template <int JB>
+__device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRec& r, float (&acc)[kAccSets][4],
+                                               PendingCount* pc, int lane) {
+  constexpr int SB = JB <= 2 ? 4 : 2;
   const int g = lane >> 2, q = lane & 3;
-  const int rp = r.rp, jblocks = rp >> 4;
   float* part = a.partial + ((size_t)r.job * a.kcmax + r.sub) * kR * a.rp;
   if (q < 2) {
 #pragma unroll
-    for (int jb = 0; jb < kImagePadMax / 16; ++jb) {
-      if (jb < jblocks) {
-        const int j = jb * 16 + g;
-        part[(2 * q) * a.rp + j] = acc[jb][0];
-        part[(2 * q + 1) * a.rp + j] = acc[jb][1];
-        part[(2 * q) * a.rp + j + 8] = acc[jb][2];
-        part[(2 * q + 1) * a.rp + j + 8] = acc[jb][3];
+    for (int jb = 0; jb < JB; ++jb) {
+      float c[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        c[e] = acc[jb][e];
+#pragma unroll
+        for (int s = 1; s < SB; ++s) c[e] += acc[s * JB + jb][e];      // fixed order: set 0, 1, ...
       }
+      const int j = jb * 16 + g;
+      part[(2 * q) * a.rp + j] = c[0];
+      part[(2 * q + 1) * a.rp + j] = c[1];
+      part[(2 * q) * a.rp + j + 8] = c[2];
+      part[(2 * q + 1) * a.rp + j + 8] = c[3];
     }
   }
+  const int t = g >> 1;
+  pc->job = r.job; pc->upj_s = r.upj_s; pc->jb = JB;
+  pc->w = (t < r.n) ? r.scale * r.gate[t] : 0.f;
+  pc->valid = true;
+  pc->old = 0;
   __syncwarp();
-  uint32_t* state = a.job_state + 2 * (size_t)r.job;
-  uint32_t old = 0;
-  if (lane == 0) {
-    __threadfence();
-    old = atomicAdd(state, 1u);
-    __threadfence();
-  }
-  old = __shfl_sync(0xffffffffu, old, 0);
-  if (old != (uint32_t)r.upj_s - 1) return;
-  // this unit arrived last: every partial of the job is visible now
-  const float* base = a.partial + (size_t)r.job * a.kcmax * kR * a.rp;
+  if (lane == 0) pc->old = atom_add_acq_rel(a.job_state + r.job, 1u);
+}
+
+// Second half: the unit that arrived last adds the job's partial sums in unit order (every one of them is visible
+// after its count), and publishes v as the fragments of the expand MMAs' second operand (K = rank rows, N = 8):
+// column n = g holds row t = g / 2 of v, as its bf16 value for even g and as the remainder after that rounding for
+// odd g.  Each lane computes the values of its own fragment.  The job's counter goes back to zero for the next launch.
+__device__ __forceinline__ void shrink_finalize(const StreamArgs& a, PendingCount* pc, int lane) {
+  if (!pc->valid) return;
+  pc->valid = false;
+  const uint32_t old = __shfl_sync(0xffffffffu, pc->old, 0);
+  if (old != (uint32_t)pc->upj_s - 1) return;
+  __syncwarp();          // lane 0's acquire covers the loads of the whole warp
+  const int g = lane >> 2, q = lane & 3;
+  const int t = g >> 1;
+  const bool rem = g & 1;
+  const float* base = a.partial + (size_t)pc->job * a.kcmax * kR * a.rp + t * a.rp;
   const size_t ustride = (size_t)kR * a.rp;
-  for (int idx = lane; idx < kR * rp; idx += 32) {
-    const int t = idx / rp, j = idx % rp;
-    const float* vp = base + t * a.rp + j;
-    float sum = 0.f;
-    for (int c0 = 0; c0 < r.upj_s; c0 += 8) {
-      float p8[8];
+  uint4* out = a.vfrag + (size_t)pc->job * (a.rp >> 4) * 32;
+  if (lane == 0) a.job_state[pc->job] = 0;
+  for (int ks = 0; ks < pc->jb; ++ks) {
+    const float* vp = base + ks * 16 + 2 * q;
+    float v4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int c0 = 0; c0 < pc->upj_s; c0 += 4) {
+      float2 lo[4], hi[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) p8[i] = (c0 + i < r.upj_s) ? __ldcg(vp + (size_t)(c0 + i) * ustride) : 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) sum += p8[i];
-    }
-    vsum[t][j] = (t < r.n) ? sum * r.scale * r.gate[t] : 0.f;
-  }
-  __syncwarp();
-  // fragment of the second MMA operand (K = rank rows, N = 8): column n = g holds row t = g / 2 of v, its bf16
-  // value for even g and the remainder after that rounding for odd g
-  {
-    const int t = g >> 1;
-    const bool rem = g & 1;
-    uint2* out = a.vfrag + (size_t)r.job * (a.rp >> 4) * 32;
-    for (int ks = 0; ks < jblocks; ++ks) {
-      float v4[4] = {vsum[t][ks * 16 + 2 * q], vsum[t][ks * 16 + 2 * q + 1], vsum[t][ks * 16 + 2 * q + 8],
-                     vsum[t][ks * 16 + 2 * q + 9]};
-      uint32_t w0 = pack_bf16(v4[0], v4[1]), w1 = pack_bf16(v4[2], v4[3]);
-      if (rem) {
-        const uint32_t h0 = w0, h1 = w1;
-        w0 = pack_bf16(v4[0] - bf16_lo(h0), v4[1] - bf16_hi(h0));
-        w1 = pack_bf16(v4[2] - bf16_lo(h1), v4[3] - bf16_hi(h1));
+      for (int i = 0; i < 4; ++i) {
+        lo[i] = hi[i] = make_float2(0.f, 0.f);
+        if (c0 + i < pc->upj_s) {
+          lo[i] = __ldcg(reinterpret_cast<const float2*>(vp + (size_t)(c0 + i) * ustride));
+          hi[i] = __ldcg(reinterpret_cast<const float2*>(vp + (size_t)(c0 + i) * ustride + 8));
+        }
       }
-      out[ks * 32 + lane] = make_uint2(w0, w1);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { v4[0] += lo[i].x; v4[1] += lo[i].y; v4[2] += hi[i].x; v4[3] += hi[i].y; }
     }
-  }
-  __syncwarp();
-  if (lane == 0) {
-    __threadfence();
-    st_release(state, kReady);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v4[i] *= pc->w;
+    uint32_t w0 = pack_bf16(v4[0], v4[1]), w1 = pack_bf16(v4[2], v4[3]);
+    if (rem) {
+      const uint32_t h0 = w0, h1 = w1;
+      w0 = pack_bf16(v4[0] - bf16_lo(h0), v4[1] - bf16_hi(h0));
+      w1 = pack_bf16(v4[2] - bf16_lo(h1), v4[3] - bf16_hi(h1));
+    }
+    st_tagged(out + ks * 32 + lane, w0, w1, a.epoch);
   }
 }
 
-// ---- expand: one stage, y updated in shared memory and stored back --------------------------------------------
+// ---- expand: one stage, added to y in global memory -----------------------------------------------------------
+// KS = rank blocks of 16.  NS steps of 16 columns are handled together, again grouped by kind of instruction.
+template <int KS>
 __device__ __forceinline__ void expand_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf,
                                              const uint2 (&vb)[kImagePadMax / 16], int lane) {
+  constexpr int NS = KS <= 2 ? 8 / KS : 2;
+  constexpr int rp = KS * 16;
   const int g = lane >> 2, q = lane & 3, mi = lane >> 3;
   const int c0 = (r.stage0 + stage_in_unit) * a.cols;
   const int ncols = min(a.cols, r.d - c0);
-  const int rp = r.rp, ksteps = rp >> 4;
-  const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
   const bool row_ok = q < r.n;
-  const uint32_t yrow = buf + kStageBytes + (row_ok ? q : 0) * rstride + 2 * g;
+  // The accumulators of a step give this lane column g and column g + 8 of row t = q.  Lanes g and g ^ 1 swap one
+  // of the two, so that the even lane holds columns (g, g + 1) and the odd lane columns (g + 7, g + 8): two
+  // neighbouring elements each, which one packed addition updates.
+  const bool odd = g & 1;
+  __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(const_cast<char*>(r.rows_base)) +
+                      (size_t)(row_ok ? r.rows[q] : 0) * r.d + c0 + (odd ? g + 7 : g);
   // ldmatrix row address inside a 128-column block for rank step 0, column step 0:
   // core matrix (n / 8, k / 8) at ((k / 8) * 16 + n / 8) * 128
   const uint32_t lane_off = (uint32_t)(((mi >> 1) * 16 + (mi & 1)) * 128 + (lane & 7) * 16);
   for (int nb = 0; nb < (ncols >> 7); ++nb) {
     const uint32_t blk = buf + (uint32_t)nb * rp * 256 + lane_off;
 #pragma unroll
-    for (int ns = 0; ns < 8; ++ns) {
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int n0 = 0; n0 < 8; n0 += NS) {
+      uint32_t am[NS][KS][4];
+      float c[NS][4];
 #pragma unroll
-      for (int ks = 0; ks < kImagePadMax / 16; ++ks) {
-        if (ks < ksteps) {
-          uint32_t a0, a1, a2, a3;
-          ldmatrix_x4(blk + (uint32_t)((2 * ks) * 16 + 2 * ns) * 128, a0, a1, a2, a3);
-          mma_16816(c, a0, a1, a2, a3, vb[ks].x, vb[ks].y);
-        }
+      for (int ns = 0; ns < NS; ++ns)
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+          ldmatrix_x4(blk + (uint32_t)((2 * ks) * 16 + 2 * (n0 + ns)) * 128, am[ns][ks][0], am[ns][ks][1], am[ns][ks][2],
+                      am[ns][ks][3]);
+#pragma unroll
+      for (int ns = 0; ns < NS; ++ns) {
+        c[ns][0] = c[ns][1] = c[ns][2] = c[ns][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+          mma_16816(c[ns], am[ns][ks][0], am[ns][ks][1], am[ns][ks][2], am[ns][ks][3], vb[ks].x, vb[ks].y);
       }
       // c0 + c1: column g of the step, row t = q (value part + remainder part); c2 + c3: column g + 8
-      if (row_ok) {
-        const uint32_t p = yrow + (nb * 128 + ns * 16) * 2;
-        const float y0 = __uint_as_float(lds16(p) << 16) + (c[0] + c[1]);
-        const float y1 = __uint_as_float(lds16(p + 16) << 16) + (c[2] + c[3]);
-        sts16(p, __bfloat16_as_ushort(__float2bfloat16_rn(y0)));
-        sts16(p + 16, __bfloat16_as_ushort(__float2bfloat16_rn(y1)));
+#pragma unroll
+      for (int ns = 0; ns < NS; ++ns) {
+        const float lo = c[ns][0] + c[ns][1], hi = c[ns][2] + c[ns][3];
+        const float got = __shfl_xor_sync(0xffffffffu, odd ? lo : hi, 4);
+        if (row_ok) red_add_bf16x2(yp + nb * 128 + (n0 + ns) * 16, odd ? got : lo, odd ? hi : got);
       }
     }
-  }
-  fence_proxy_async_smem();
-  __syncwarp();
-  if (lane == 0) {
-    for (int t = 0; t < r.n; ++t)
-      bulk_s2g(const_cast<char*>(r.rows_base) + ((size_t)r.rows[t] * r.d + c0) * 2, buf + kStageBytes + t * rstride,
-               (uint32_t)ncols * 2);
-    bulk_commit_group();
   }
 }
 
 // ---- the kernel --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a) {
+template <class SH>
+__global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamArgs a) {
+  constexpr int kWarps = SH::kWarps, kThreads = SH::kThreads;
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  Smem& sm = *reinterpret_cast<Smem*>(smem_raw + (size_t)kWarps * kBufs * kBufStride);
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw + (size_t)kWarps * kBufs * a.buf_stride);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int L = a.n_layers;
   const int n_seg = 2 * L * MILORA_NMOD;
@@ -439,62 +498,86 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a
   // ---- worker ----
   const int n_workers = (int)gridDim.x * kWarps;
   const int wid = warp * (int)gridDim.x + (int)blockIdx.x;     // neighbouring units go to different SMs
-  const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(warp * kBufs) * kBufStride;
+  const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(warp * kBufs) * a.buf_stride;
   UnitRec* ring = sm.unit[warp];
-  int n_fetched = 0;              // units this worker has taken so far
+  int n_fetched = 0;              // units this worker has asked for so far
   int n_kept = 0;                 // ... of which were valid (they take turns in the ring of unit records)
   int n_issued = 0, n_done = 0;   // stages issued / consumed (buffer = count % kBufs, parity = (count / kBufs) & 1)
   int iu = -1, is = 0;            // ring index and next stage of the unit being issued (-1: none)
-  bool dry = false, failed = false;
-  uint32_t next_dyn = 0;          // counter value fetched ahead
-  bool have_dyn = false;
-  float acc[kImagePadMax / 16][4];
+  bool failed = false, dry = false;
+  // Look-ahead: the two units after the one being issued are located and their records are on the way
+  // (pf0 is the next one); the counter value for the unit after those has been asked for (lane 0).
+  UnitLoc pf0, pf1;
+  bool pf0_valid = false, pf1_valid = false;
+  uint32_t next_dyn = 0;
+  float acc[kAccSets][4];
+  PendingCount pend;
+  pend.valid = false;
+  uint4 vb_pf[kImagePadMax / 16];   // fragments of the expand unit taken last, asked for when it was taken
+  int vb_pf_unit = -1;
   uint2 vb[kImagePadMax / 16];
-  int cu_loaded = -1;             // ring index of the unit whose fragments are in vb
+  int cu_loaded = -1;               // ring index of the unit whose fragments are in vb
 
+  // asks for one more unit (index, place in the lists, record load) into pf1
+  auto look_ahead = [&]() {
+    pf1_valid = false;
+    if (dry) return;
+    int u;
+    if (n_fetched < kStaticRounds) {
+      u = wid + n_fetched * n_workers;
+    } else {
+      u = kStaticRounds * n_workers + (int)__shfl_sync(0xffffffffu, next_dyn, 0);
+      if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);    // for the call after this one
+    }
+    ++n_fetched;
+    if (u >= total) { dry = true; return; }
+    pf1 = locate_unit(a, sm, n_seg, u, lane);
+    pf1_valid = true;
+  };
+  // makes the next located unit the one being issued (skipping damaged records) and looks one further ahead
   auto take_unit = [&]() {
-    // next unit of this worker into the ring; sets iu (or dry)
-    while (!dry) {
-      int u;
-      if (n_fetched < kStaticRounds) {
-        u = wid + n_fetched * n_workers;
-      } else {
-        if (!have_dyn) {
-          if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);
-          have_dyn = true;
-        }
-        u = kStaticRounds * n_workers + (int)__shfl_sync(0xffffffffu, next_dyn, 0);
-        have_dyn = false;
-      }
-      ++n_fetched;
-      if (u >= total) { dry = true; break; }
-      if (n_fetched >= kStaticRounds) {      // ask for the one after it now; the answer is used at the next call
-        if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);
-        have_dyn = true;
-      }
+    iu = -1;
+    while (pf0_valid) {
       // at most kBufs earlier units still have stages in a buffer, so the record after the last kept one is free
       const int slot = n_kept % kUnitRing;
-      decode_unit(a, sm, n_seg, u, &ring[slot], lane);
+      fill_unit(a, sm, pf0, &ring[slot], lane);
       __syncwarp();
-      if (ring[slot].ok) { ++n_kept; iu = slot; is = 0; return; }
-      if (ring[slot].sub == 0 && ring[slot].phase == 0 && lane == 0) atomicOr(a.err, ERR_BAD_ITEM);
+      const bool ok = ring[slot].ok != 0;
+      if (!ok && ring[slot].sub == 0 && ring[slot].phase == 0 && lane == 0) atomicOr(a.err, ERR_BAD_ITEM);
+      pf0 = pf1;
+      pf0_valid = pf1_valid;
+      look_ahead();
+      if (ok) {
+        ++n_kept; iu = slot; is = 0;
+        if (ring[slot].phase == 1) {
+          // an expand unit: ask for its fragments now; they are checked (and asked for again if the job's shrink
+          // units have not all finished yet) when its first stage is consumed
+          const uint4* vf = a.vfrag + (size_t)ring[slot].job * (a.rp >> 4) * 32;
+#pragma unroll
+          for (int ks = 0; ks < kImagePadMax / 16; ++ks)
+            if (ks < (ring[slot].rp >> 4)) vb_pf[ks] = ld_tagged(vf + ks * 32 + lane);
+          vb_pf_unit = slot;
+        }
+        return;
+      }
     }
-    iu = -1;
   };
 
+  if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);
+  look_ahead();
+  pf0 = pf1;
+  pf0_valid = pf1_valid;
+  look_ahead();
   take_unit();
   while (true) {
     // issue while a buffer is free
     while (iu >= 0 && n_issued - n_done < kBufs) {
       const int b = n_issued % kBufs;
-      const uint32_t buf = buf0 + b * kBufStride, bar = smem_u32(&sm.full[warp][b]);
+      const uint32_t buf = buf0 + b * a.buf_stride, bar = smem_u32(&sm.full[warp][b]);
       if (lane == 0) {
         sm.buf_unit[warp][b] = iu;
         sm.buf_stage[warp][b] = is;
-        issue_stage(a, ring[iu], is, buf, bar, false);
-        // the rows of this buffer may still be read by the bulk store of the stage that used it last
-        bulk_wait_group_read0();
-        issue_stage(a, ring[iu], is, buf, bar, true);
+        issue_stage(a, ring[iu], is, buf, bar);
       }
       ++n_issued;
       if (++is == ring[iu].n_stages) take_unit();
@@ -502,15 +585,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a
     if (n_done == n_issued) break;
     // consume the oldest stage
     const int b = n_done % kBufs;
-    const uint32_t buf = buf0 + b * kBufStride, bar = smem_u32(&sm.full[warp][b]);
+    const uint32_t buf = buf0 + b * a.buf_stride, bar = smem_u32(&sm.full[warp][b]);
     __syncwarp();
     const int cu = sm.buf_unit[warp][b], cs = sm.buf_stage[warp][b];
     const UnitRec& r = ring[cu];
+    const int jb = r.rp >> 4;
     if (!mbar_wait(bar, (uint32_t)(n_done / kBufs) & 1u)) {
-      // the copies did not arrive: report, stop taking work, let what is in flight land (bounded again below)
+      // the copies did not arrive: report, stop taking work, and give what is in flight a second (bounded) wait
+      // so that nothing lands in shared memory after the CTA has gone
       if (lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
       failed = true;
       iu = -1;
+      pf0_valid = pf1_valid = false;
       dry = true;
       mbar_wait(bar, (uint32_t)(n_done / kBufs) & 1u);
       ++n_done;
@@ -519,26 +605,52 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a
     if (r.phase == 0) {
       if (cs == 0) {
 #pragma unroll
-        for (int jb = 0; jb < kImagePadMax / 16; ++jb)
+        for (int i = 0; i < kAccSets; ++i)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[jb][e] = 0.f;
+          for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
       }
-      shrink_stage(a, r, cs, buf, acc, lane);
-      if (cs == r.n_stages - 1 && !failed) shrink_finish(a, r, acc, sm.vsum[warp], lane);
-    } else {
-      bool ready = true;
-      if (cs == 0 || cu_loaded != cu) {
-        const uint32_t* state = a.job_state + 2 * (size_t)r.job;
-        uint32_t spins = 0;
-        while (ld_acquire(state) != kReady) {
-          if (++spins >= kDepSpin) { ready = false; break; }
-          __nanosleep(64);
+      switch (jb) {
+        case 1: shrink_stage<1>(a, r, cs, buf, acc, lane); break;
+        case 2: shrink_stage<2>(a, r, cs, buf, acc, lane); break;
+        case 3: shrink_stage<3>(a, r, cs, buf, acc, lane); break;
+        default: shrink_stage<4>(a, r, cs, buf, acc, lane); break;
+      }
+      shrink_finalize(a, &pend, lane);      // the count of the unit before this one has had a stage's time to answer
+      if (cs == r.n_stages - 1 && !failed) {
+        switch (jb) {
+          case 1: shrink_publish<1>(a, r, acc, &pend, lane); break;
+          case 2: shrink_publish<2>(a, r, acc, &pend, lane); break;
+          case 3: shrink_publish<3>(a, r, acc, &pend, lane); break;
+          default: shrink_publish<4>(a, r, acc, &pend, lane); break;
         }
-        if (ready) {
-          const uint2* vf = a.vfrag + (size_t)r.job * (a.rp >> 4) * 32;
+      }
+    } else {
+      if (cs == 0 || cu_loaded != cu) {
+        // fragments of v: those asked for when the unit was taken, unless another unit was taken since
+        const uint4* vf = a.vfrag + (size_t)r.job * (a.rp >> 4) * 32;
+        uint4 f[kImagePadMax / 16];
+#pragma unroll
+        for (int ks = 0; ks < kImagePadMax / 16; ++ks) {
+          f[ks] = make_uint4(0, a.epoch, 0, a.epoch);
+          if (ks < jb) f[ks] = (vb_pf_unit == cu) ? vb_pf[ks] : ld_tagged(vf + ks * 32 + lane);
+        }
+        uint32_t spins = 0;
+        while (true) {
+          bool mine = true;
+#pragma unroll
+          for (int ks = 0; ks < kImagePadMax / 16; ++ks) mine = mine && f[ks].y == a.epoch && f[ks].w == a.epoch;
+          if (__all_sync(0xffffffffu, mine)) break;
+          if (++spins >= kDepSpin) break;
+          // the job's shrink units are not all done: its last one may be waiting behind this very stage
+          shrink_finalize(a, &pend, lane);
+          __nanosleep(100);
 #pragma unroll
           for (int ks = 0; ks < kImagePadMax / 16; ++ks)
-            vb[ks] = (ks < (r.rp >> 4)) ? __ldcg(vf + ks * 32 + lane) : make_uint2(0, 0);
+            if (ks < jb) f[ks] = ld_tagged(vf + ks * 32 + lane);
+        }
+        if (spins < kDepSpin) {
+#pragma unroll
+          for (int ks = 0; ks < kImagePadMax / 16; ++ks) vb[ks] = make_uint2(f[ks].x, f[ks].z);
           cu_loaded = cu;
         } else {
           if (lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
@@ -546,22 +658,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a
           cu_loaded = -1;
         }
       }
-      if (ready && cu_loaded == cu) expand_stage(a, r, cs, buf, vb, lane);
-      if (cs == r.n_stages - 1 && !failed && lane == 0) {
-        uint32_t* state = a.job_state + 2 * (size_t)r.job;
-        const uint32_t old = atomicAdd(state + 1, 1u);
-        if (old == (uint32_t)r.upj_e - 1) {      // every expand unit of the job has read v: reset for the next launch
-          state[0] = 0;
-          state[1] = 0;
+      if (cu_loaded == cu) {
+        switch (jb) {
+          case 1: expand_stage<1>(a, r, cs, buf, vb, lane); break;
+          case 2: expand_stage<2>(a, r, cs, buf, vb, lane); break;
+          case 3: expand_stage<3>(a, r, cs, buf, vb, lane); break;
+          default: expand_stage<4>(a, r, cs, buf, vb, lane); break;
         }
       }
+      shrink_finalize(a, &pend, lane);
     }
     __syncwarp();
     ++n_done;
   }
-  // stores of y must have left shared memory before the CTA may go; the counter is reset by the last worker
+  shrink_finalize(a, &pend, lane);
+  // the counter is reset by the worker that finishes last
   if (lane == 0) {
-    bulk_wait_group0();
     __threadfence();        // a counter request that was never used must not pass the line below
     const uint32_t old = atomicAdd(&a.ctrl[1], 1u);
     if (old == (uint32_t)n_workers - 1) {
@@ -571,10 +683,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stream_kernel(StreamArgs a
   }
 }
 
-__host__ __device__ inline int stage_cols(int rp) {
-  int c = (kStageBytes / (2 * rp)) & ~127;
-  return c < 128 ? 128 : c;
-}
+// Columns of d1 / d2 per stage: as many 128-column blocks as the stage holds at this padded rank.
+inline int stage_cols(int stage_bytes, int rp) { return (stage_bytes / (2 * rp)) & ~127; }
 
 }  // namespace
 
@@ -593,13 +703,19 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
   std::memset(&a, 0, sizeof(a));
   a.err = ctx->d_err;
   a.rp = (ctx->desc.max_rank + 15) & ~15;
-  a.cols = stage_cols(a.rp);
+  const bool small = stage_cols(ShapeSmall::kStageBytes, a.rp) >= 128;
+  const int n_warps = small ? ShapeSmall::kWarps : ShapeLarge::kWarps;
+  a.stage_bytes = small ? ShapeSmall::kStageBytes : ShapeLarge::kStageBytes;
+  a.cols = stage_cols(a.stage_bytes, a.rp);
+  if (a.cols < 128) return MILORA_E_SHAPE;
+  // a buffer: the stage, then kR rows of x; the smallest padded rank (16) gives the widest rows
+  a.buf_stride = (a.stage_bytes + kR * (a.cols * 2 + kRowPad) + 127) & ~127;
   double stages_per_job = 0;
   for (int m = 0; m < MILORA_NMOD; ++m) {
     module_dims(ctx->desc, m, &a.d1[m], &a.d2[m]);
     stages_per_job += ((a.d1[m] + a.cols - 1) / a.cols + (a.d2[m] + a.cols - 1) / a.cols) / (double)MILORA_NMOD;
   }
-  const int workers = ctx->sm_count * kWarps;
+  const int workers = ctx->sm_count * n_warps;
   int us = ctx->stream_unit_stages;
   if (us < 1) {
     // enough units that every worker gets several; long units save partial sums and look-ups
@@ -612,16 +728,19 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
   for (int m = 0; m < MILORA_NMOD; ++m)
     kcmax = std::max(kcmax, ((a.d1[m] + a.cols - 1) / a.cols + us - 1) / us);
   a.kcmax = kcmax;
-  const size_t frag_bytes = (size_t)(a.rp >> 4) * 32 * sizeof(uint2);
+  const size_t frag_bytes = (size_t)(a.rp >> 4) * 32 * sizeof(uint4);
   const size_t part_bytes = (size_t)kcmax * kR * a.rp * sizeof(float);
   // scratch of a launch: control words | job states | fragments | partial sums
   auto scratch_bytes = [&](size_t jobs) { return 256 + align256(jobs * 8) + align256(jobs * frag_bytes) + jobs * part_bytes; };
   const size_t cap_bytes = (size_t)512 << 20;
-  const size_t smem = (size_t)kWarps * kBufs * kBufStride + sizeof(Smem);
+  const size_t smem = (size_t)n_warps * kBufs * a.buf_stride + sizeof(Smem);
   if (!ctx->stream_attr_set) {
-    MILORA_CUDA(ctx, cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int top = 227 * 1024;
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(decode_stream_kernel<ShapeSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, top));
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(decode_stream_kernel<ShapeLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, top));
     ctx->stream_attr_set = true;
   }
+  if (smem > 227 * 1024) return MILORA_E_SHAPE;
 
   for (int l0 = 0; l0 < n_layers;) {
     // a launch takes as many layers as the record table and the scratch cap allow
@@ -635,9 +754,9 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
       ++l1;
     }
     const int n = l1 - l0;
-    // The buffer is laid out for its capacity (jobs, bytes per job), not for the batch at hand, so a job's state
-    // words never serve as anything else; every launch leaves them at zero, and they are cleared by the host only
-    // when the buffer is new or after a launch that failed or timed out.
+    // The buffer is laid out for its capacity (jobs, bytes per job), not for the batch at hand, so a job's counter
+    // never serves as anything else; every launch leaves the counters at zero, and they are cleared by the host only
+    // when the buffer is new or after a launch that failed or timed out.  Fragments carry the launch's tag.
     if (jobs > ctx->stream_jobs_cap || frag_bytes > ctx->stream_frag_bytes || part_bytes > ctx->stream_part_bytes) {
       const size_t jc = std::max(jobs, ctx->stream_jobs_cap);
       const size_t fb = std::max(frag_bytes, ctx->stream_frag_bytes), pb = std::max(part_bytes, ctx->stream_part_bytes);
@@ -647,6 +766,8 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
       ctx->d_stream = nullptr;
       ctx->stream_jobs_cap = 0;
       MILORA_CUDA(ctx, cudaMalloc(&ctx->d_stream, need));
+      // fresh memory may hold anything, also words that look like a later launch's tag
+      MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_stream, 0, need, s));
       ctx->stream_jobs_cap = jc;
       ctx->stream_frag_bytes = fb;
       ctx->stream_part_bytes = pb;
@@ -656,7 +777,7 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
     const size_t state_bytes = align256(ctx->stream_jobs_cap * 8);
     a.ctrl = reinterpret_cast<uint32_t*>(base);
     a.job_state = reinterpret_cast<uint32_t*>(base + 256);
-    a.vfrag = reinterpret_cast<uint2*>(base + 256 + state_bytes);
+    a.vfrag = reinterpret_cast<uint4*>(base + 256 + state_bytes);
     a.partial = reinterpret_cast<float*>(base + 256 + state_bytes + align256(ctx->stream_jobs_cap * ctx->stream_frag_bytes));
     if (ctx->stream_dirty) MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_stream, 0, 256 + state_bytes, s));
     a.n_layers = n;
@@ -689,8 +810,14 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
       }
       a.layers = static_cast<const StreamLayer*>(ctx->d_stream_layers);
     }
+    if (++ctx->stream_epoch == 0) ++ctx->stream_epoch;      // 0 is what a cleared buffer holds
+    a.epoch = ctx->stream_epoch;
     ctx->stream_dirty = true;       // stays set if the launch fails
-    MILORA_CUDA(ctx, launch_pdl(decode_stream_kernel, dim3((unsigned)ctx->sm_count), dim3(kThreads), smem, s, a));
+    if (small) {
+      MILORA_CUDA(ctx, launch_pdl(decode_stream_kernel<ShapeSmall>, dim3((unsigned)ctx->sm_count), dim3(ShapeSmall::kThreads), smem, s, a));
+    } else {
+      MILORA_CUDA(ctx, launch_pdl(decode_stream_kernel<ShapeLarge>, dim3((unsigned)ctx->sm_count), dim3(ShapeLarge::kThreads), smem, s, a));
+    }
     ctx->stream_dirty = false;
     l0 = l1;
   }

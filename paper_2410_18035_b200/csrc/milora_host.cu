@@ -173,7 +173,7 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->dsplit_occ_s = 0; ctx->dsplit_occ_e = 0; ctx->decode_path = MILORA_DECODE_AUTO;
   ctx->copy_stream = nullptr; ctx->ev_done = nullptr; ctx->copy_ready = false;
   ctx->d_stream = nullptr; ctx->stream_jobs_cap = 0; ctx->stream_frag_bytes = 0; ctx->stream_part_bytes = 0;
-  ctx->stream_dirty = true; ctx->stream_attr_set = false; ctx->stream_unit_stages = 0;
+  ctx->stream_dirty = true; ctx->stream_attr_set = false; ctx->stream_epoch = 0; ctx->stream_unit_stages = 0;
   ctx->d_stream_layers = nullptr; ctx->h_stream_stage = nullptr; ctx->stream_stage_next = 0; ctx->stream_layers_cached = 0;
   for (int i = 0; i < 4; ++i) ctx->stream_stage_ev[i] = nullptr;
   for (int m = 0; m < MILORA_NMOD; ++m) ctx->ev_site[m] = nullptr;

@@ -164,6 +164,7 @@ struct milora_ctx {
   size_t stream_jobs_cap, stream_frag_bytes, stream_part_bytes;   // what d_stream is laid out for
   bool stream_dirty;                            // job states must be cleared before the next launch
   bool stream_attr_set;
+  uint32_t stream_epoch;                        // tag of the last launch (marks the fragments it wrote)
   int stream_unit_stages;                       // stages per unit; 0 = chosen from the batch size
   void* d_stream_layers;                        // layer records of a multi-layer launch
   void* h_stream_stage;                         // pinned: four staging copies of those records
