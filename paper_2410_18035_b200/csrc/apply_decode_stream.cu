@@ -75,7 +75,7 @@ struct StreamArgs {
   uint32_t* ctrl;              // [0] units handed out beyond the static rounds, [1] workers that have finished
   uint32_t* job_state;         // [jobs]: shrink units of the job that have delivered their partial sums
   uint32_t epoch;              // tag of this launch (never 0): marks the fragments written by it
-  float* partial;              // [jobs][kcmax][kR][rp]
+  uint2* partial;              // [jobs][kcmax][kR][rp] of {value, epoch}
   uint4* vfrag;                // [jobs][rp / 16][32] of {word 0, epoch, word 1, epoch}
 };
 
@@ -128,11 +128,15 @@ __device__ __forceinline__ void red_add_bf16x2(void* addr, float v0, float v1) {
   const uint32_t h = pack_bf16(v0, v1);
   asm volatile("red.global.add.noftz.bf16x2 [%0], %1;" ::"l"(addr), "r"(h) : "memory");
 }
-// counts on a job; release for this warp's earlier writes, acquire for the other units' partial sums
-__device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
-  uint32_t old;
-  asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-  return old;
+// A value that travels together with the tag of the launch that wrote it, as one 8-byte access (8-byte accesses
+// are single-copy atomic): whoever reads the right tag has the right value, without a flag or a fence.
+__device__ __forceinline__ void st_tagged1(uint2* p, uint32_t w, uint32_t tag) {
+  asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(w), "r"(tag) : "memory");
+}
+__device__ __forceinline__ uint2 ld_tagged1(const uint2* p) {
+  uint2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  return v;
 }
 // A fragment word travels together with the tag of the launch that wrote it, as one 8-byte access (8-byte
 // accesses are single-copy atomic): whoever reads the right tag has the right word, without a flag or a fence.
@@ -304,7 +308,7 @@ __device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRe
                                                PendingCount* pc, int lane) {
   constexpr int SB = JB <= 2 ? 4 : 2;
   const int g = lane >> 2, q = lane & 3;
-  float* part = a.partial + ((size_t)r.job * a.kcmax + r.sub) * kR * a.rp;
+  uint2* part = a.partial + ((size_t)r.job * a.kcmax + r.sub) * kR * a.rp;
   if (q < 2) {
 #pragma unroll
     for (int jb = 0; jb < JB; ++jb) {
@@ -316,10 +320,10 @@ __device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRe
         for (int s = 1; s < SB; ++s) c[e] += acc[s * JB + jb][e];      // fixed order: set 0, 1, ...
       }
       const int j = jb * 16 + g;
-      part[(2 * q) * a.rp + j] = c[0];
-      part[(2 * q + 1) * a.rp + j] = c[1];
-      part[(2 * q) * a.rp + j + 8] = c[2];
-      part[(2 * q + 1) * a.rp + j + 8] = c[3];
+      st_tagged1(part + (2 * q) * a.rp + j, __float_as_uint(c[0]), a.epoch);
+      st_tagged1(part + (2 * q + 1) * a.rp + j, __float_as_uint(c[1]), a.epoch);
+      st_tagged1(part + (2 * q) * a.rp + j + 8, __float_as_uint(c[2]), a.epoch);
+      st_tagged1(part + (2 * q + 1) * a.rp + j + 8, __float_as_uint(c[3]), a.epoch);
     }
   }
   const int t = g >> 1;
@@ -327,42 +331,60 @@ __device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRe
   pc->w = (t < r.n) ? r.scale * r.gate[t] : 0.f;
   pc->valid = true;
   pc->old = 0;
-  __syncwarp();
-  if (lane == 0) pc->old = atom_add_acq_rel(a.job_state + r.job, 1u);
+  // The count only decides who adds the job up; the partial sums carry this launch's tag, so no fence is needed
+  // (a fence here would wait for every addition into y that this warp still has under way).
+  if (lane == 0) pc->old = atomicAdd(a.job_state + r.job, 1u);
 }
 
-// Second half: the unit that arrived last adds the job's partial sums in unit order (every one of them is visible
-// after its count), and publishes v as the fragments of the expand MMAs' second operand (K = rank rows, N = 8):
-// column n = g holds row t = g / 2 of v, as its bf16 value for even g and as the remainder after that rounding for
-// odd g.  Each lane computes the values of its own fragment.  The job's counter goes back to zero for the next launch.
-__device__ __forceinline__ void shrink_finalize(const StreamArgs& a, PendingCount* pc, int lane) {
-  if (!pc->valid) return;
+// Second half: the unit that arrived last adds the job's partial sums in unit order and publishes v as the
+// fragments of the expand MMAs' second operand (K = rank rows, N = 8): column n = g holds row t = g / 2 of v, as its
+// bf16 value for even g and as the remainder after that rounding for odd g.  Each lane computes the values of its
+// own fragment.  A partial sum whose tag is not this launch's yet (its store is still on the way) is asked for
+// again, a bounded number of times.  The job's counter goes back to zero for the next launch.
+// Returns false when a partial sum never arrived.
+__device__ __forceinline__ bool shrink_finalize(const StreamArgs& a, PendingCount* pc, int lane) {
+  if (!pc->valid) return true;
   pc->valid = false;
   const uint32_t old = __shfl_sync(0xffffffffu, pc->old, 0);
-  if (old != (uint32_t)pc->upj_s - 1) return;
-  __syncwarp();          // lane 0's acquire covers the loads of the whole warp
+  if (old != (uint32_t)pc->upj_s - 1) return true;
   const int g = lane >> 2, q = lane & 3;
   const int t = g >> 1;
   const bool rem = g & 1;
-  const float* base = a.partial + (size_t)pc->job * a.kcmax * kR * a.rp + t * a.rp;
+  const uint2* base = a.partial + (size_t)pc->job * a.kcmax * kR * a.rp + t * a.rp;
   const size_t ustride = (size_t)kR * a.rp;
   uint4* out = a.vfrag + (size_t)pc->job * (a.rp >> 4) * 32;
   if (lane == 0) a.job_state[pc->job] = 0;
+  bool all_ok = true;
   for (int ks = 0; ks < pc->jb; ++ks) {
-    const float* vp = base + ks * 16 + 2 * q;
+    const uint2* vp = base + ks * 16 + 2 * q;
     float v4[4] = {0.f, 0.f, 0.f, 0.f};
     for (int c0 = 0; c0 < pc->upj_s; c0 += 4) {
-      float2 lo[4], hi[4];
+      uint2 p[4][4];
+      uint32_t spins = 0;
+      while (true) {
+        bool ok = true;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        lo[i] = hi[i] = make_float2(0.f, 0.f);
-        if (c0 + i < pc->upj_s) {
-          lo[i] = __ldcg(reinterpret_cast<const float2*>(vp + (size_t)(c0 + i) * ustride));
-          hi[i] = __ldcg(reinterpret_cast<const float2*>(vp + (size_t)(c0 + i) * ustride + 8));
+        for (int i = 0; i < 4; ++i) {
+          const uint2* u = vp + (size_t)min(c0 + i, pc->upj_s - 1) * ustride;
+          p[i][0] = ld_tagged1(u);
+          p[i][1] = ld_tagged1(u + 1);
+          p[i][2] = ld_tagged1(u + 8);
+          p[i][3] = ld_tagged1(u + 9);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) ok = ok && p[i][e].y == a.epoch;
+        if (__all_sync(0xffffffffu, ok)) break;
+        if (++spins >= kDepSpin) { all_ok = false; break; }
+        __nanosleep(100);
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { v4[0] += lo[i].x; v4[1] += lo[i].y; v4[2] += hi[i].x; v4[3] += hi[i].y; }
+      for (int i = 0; i < 4; ++i)
+        if (c0 + i < pc->upj_s) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) v4[e] += __uint_as_float(p[i][e].x);
+        }
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) v4[i] *= pc->w;
@@ -372,8 +394,9 @@ __device__ __forceinline__ void shrink_finalize(const StreamArgs& a, PendingCoun
       w0 = pack_bf16(v4[0] - bf16_lo(h0), v4[1] - bf16_hi(h0));
       w1 = pack_bf16(v4[2] - bf16_lo(h1), v4[3] - bf16_hi(h1));
     }
-    st_tagged(out + ks * 32 + lane, w0, w1, a.epoch);
+    if (all_ok) st_tagged(out + ks * 32 + lane, w0, w1, a.epoch);
   }
+  return all_ok;
 }
 
 // ---- expand: one stage, added to y in global memory -----------------------------------------------------------
@@ -387,15 +410,15 @@ __device__ __forceinline__ void expand_stage(const StreamArgs& a, const UnitRec&
   const int c0 = (r.stage0 + stage_in_unit) * a.cols;
   const int ncols = min(a.cols, r.d - c0);
   const bool row_ok = q < r.n;
-  // The accumulators of a step give this lane column g and column g + 8 of row t = q.  Lanes g and g ^ 1 swap one
-  // of the two, so that the even lane holds columns (g, g + 1) and the odd lane columns (g + 7, g + 8): two
-  // neighbouring elements each, which one packed addition updates.
-  const bool odd = g & 1;
+  // ldmatrix takes any eight rows for a matrix: the first M half of a step is given the step's even columns and
+  // the second half the odd ones, so that the accumulators of this lane are columns 2g and 2g + 1 of row t = q:
+  // two neighbouring elements of y, which one packed addition updates.
   __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(const_cast<char*>(r.rows_base)) +
-                      (size_t)(row_ok ? r.rows[q] : 0) * r.d + c0 + (odd ? g + 7 : g);
-  // ldmatrix row address inside a 128-column block for rank step 0, column step 0:
-  // core matrix (n / 8, k / 8) at ((k / 8) * 16 + n / 8) * 128
-  const uint32_t lane_off = (uint32_t)(((mi >> 1) * 16 + (mi & 1)) * 128 + (lane & 7) * 16);
+                      (size_t)(row_ok ? r.rows[q] : 0) * r.d + c0 + 2 * g;
+  // row address inside a 128-column block for rank step 0, column step 0: column n of the block sits in
+  // core matrix (n / 8, k / 8) at ((k / 8) * 16 + n / 8) * 128, row n % 8
+  const int n_loc = 2 * (lane & 7) + (mi & 1);
+  const uint32_t lane_off = (uint32_t)(((mi >> 1) * 16 + (n_loc >> 3)) * 128 + (n_loc & 7) * 16);
   for (int nb = 0; nb < (ncols >> 7); ++nb) {
     const uint32_t blk = buf + (uint32_t)nb * rp * 256 + lane_off;
 #pragma unroll
@@ -415,12 +438,11 @@ __device__ __forceinline__ void expand_stage(const StreamArgs& a, const UnitRec&
         for (int ks = 0; ks < KS; ++ks)
           mma_16816(c[ns], am[ns][ks][0], am[ns][ks][1], am[ns][ks][2], am[ns][ks][3], vb[ks].x, vb[ks].y);
       }
-      // c0 + c1: column g of the step, row t = q (value part + remainder part); c2 + c3: column g + 8
+      // c0 + c1: column 2g of the step, row t = q (value part + remainder part); c2 + c3: column 2g + 1
+      if (row_ok) {
 #pragma unroll
-      for (int ns = 0; ns < NS; ++ns) {
-        const float lo = c[ns][0] + c[ns][1], hi = c[ns][2] + c[ns][3];
-        const float got = __shfl_xor_sync(0xffffffffu, odd ? lo : hi, 4);
-        if (row_ok) red_add_bf16x2(yp + nb * 128 + (n0 + ns) * 16, odd ? got : lo, odd ? hi : got);
+        for (int ns = 0; ns < NS; ++ns)
+          red_add_bf16x2(yp + nb * 128 + (n0 + ns) * 16, c[ns][0] + c[ns][1], c[ns][2] + c[ns][3]);
       }
     }
   }
@@ -615,7 +637,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
         case 3: shrink_stage<3>(a, r, cs, buf, acc, lane); break;
         default: shrink_stage<4>(a, r, cs, buf, acc, lane); break;
       }
-      shrink_finalize(a, &pend, lane);      // the count of the unit before this one has had a stage's time to answer
+      if (!shrink_finalize(a, &pend, lane)) failed = true;      // the count of the unit before this one has had a stage's time to answer
       if (cs == r.n_stages - 1 && !failed) {
         switch (jb) {
           case 1: shrink_publish<1>(a, r, acc, &pend, lane); break;
@@ -642,7 +664,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
           if (__all_sync(0xffffffffu, mine)) break;
           if (++spins >= kDepSpin) break;
           // the job's shrink units are not all done: its last one may be waiting behind this very stage
-          shrink_finalize(a, &pend, lane);
+          if (!shrink_finalize(a, &pend, lane)) failed = true;
           __nanosleep(100);
 #pragma unroll
           for (int ks = 0; ks < kImagePadMax / 16; ++ks)
@@ -666,12 +688,13 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
           default: expand_stage<4>(a, r, cs, buf, vb, lane); break;
         }
       }
-      shrink_finalize(a, &pend, lane);
+      if (!shrink_finalize(a, &pend, lane)) failed = true;
     }
     __syncwarp();
     ++n_done;
   }
-  shrink_finalize(a, &pend, lane);
+  if (!shrink_finalize(a, &pend, lane)) failed = true;
+  if (failed && lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
   // the counter is reset by the worker that finishes last
   if (lane == 0) {
     __threadfence();        // a counter request that was never used must not pass the line below
@@ -729,7 +752,7 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
     kcmax = std::max(kcmax, ((a.d1[m] + a.cols - 1) / a.cols + us - 1) / us);
   a.kcmax = kcmax;
   const size_t frag_bytes = (size_t)(a.rp >> 4) * 32 * sizeof(uint4);
-  const size_t part_bytes = (size_t)kcmax * kR * a.rp * sizeof(float);
+  const size_t part_bytes = (size_t)kcmax * kR * a.rp * sizeof(uint2);
   // scratch of a launch: control words | job states | fragments | partial sums
   auto scratch_bytes = [&](size_t jobs) { return 256 + align256(jobs * 8) + align256(jobs * frag_bytes) + jobs * part_bytes; };
   const size_t cap_bytes = (size_t)512 << 20;
@@ -778,7 +801,7 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
     a.ctrl = reinterpret_cast<uint32_t*>(base);
     a.job_state = reinterpret_cast<uint32_t*>(base + 256);
     a.vfrag = reinterpret_cast<uint4*>(base + 256 + state_bytes);
-    a.partial = reinterpret_cast<float*>(base + 256 + state_bytes + align256(ctx->stream_jobs_cap * ctx->stream_frag_bytes));
+    a.partial = reinterpret_cast<uint2*>(base + 256 + state_bytes + align256(ctx->stream_jobs_cap * ctx->stream_frag_bytes));
     if (ctx->stream_dirty) MILORA_CUDA(ctx, cudaMemsetAsync(ctx->d_stream, 0, 256 + state_bytes, s));
     a.n_layers = n;
     if (n == 1) {
