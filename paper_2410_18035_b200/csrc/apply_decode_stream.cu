@@ -5,29 +5,33 @@
 // Section 3.3: the route is fixed per request, so the lists stay valid from step to step).
 //
 // Shape of the kernel
-//   * One CTA per SM, kWarps independent worker warps per CTA.  A worker owns kBufs shared-memory buffers and runs
-//     its own software pipeline: it asks for the next piece of adapter (a "stage": up to kStageBytes of the A or B
-//     operand image, one contiguous cp.async.bulk, plus the job's rows of x or y, one bulk copy per row) while it
-//     computes on the one that has arrived.  Workers never synchronise with each other inside the CTA.
+//   * One CTA per SM: W worker warps and one scheduler warp.  A worker owns kBufs shared-memory buffers and does
+//     nothing but wait for a buffer to fill, contract it and hand it back.  Lane w of the scheduler warp is the
+//     state machine of worker w: it takes units from the queue, reads their job records (two units ahead), and,
+//     whenever one of the worker's buffers is free, writes the stage's descriptor and starts its copies (a "stage":
+//     up to 8 KB of the A or B operand image as one contiguous cp.async.bulk, plus, for a shrink stage, the job's
+//     rows of x, one bulk copy per row).  All bookkeeping of the ten workers thus costs one warp's instructions, and
+//     none of its round trips to memory sits on a worker's path.
 //   * Work is cut into units: `unit_stages` consecutive stages of one job's shrink or expand.  Units are numbered
 //     so that every shrink unit of a job precedes all of its expand units, and the expand units of layer l come
 //     after the shrink units of layer l + 1.  The first units are assigned by worker index, later ones come from a
-//     counter (fetched ahead), so unequal units balance.
+//     counter (asked for ahead of time), so unequal units balance.
 //   * A shrink unit leaves its partial x . A^T in global scratch and counts itself on the job; the unit that
 //     arrives last adds the partials in unit order (deterministic), applies scale and gate, and publishes v as
-//     ready-made mma.sync fragments (bf16 value + bf16 remainder, i.e. v to 2^-17).  An expand unit waits
-//     (bounded) for that flag.  Since units are handed out in order and a worker issues its units in order, the
-//     unit with the smallest number that is not finished can always proceed: no deadlock while all CTAs are
-//     resident (grid = number of SMs, one CTA per SM).
+//     ready-made mma.sync fragments (bf16 value + bf16 remainder, i.e. v to 2^-17).  Partial sums and fragments
+//     travel as 8-byte {value, tag of this launch} pairs, so neither side needs a fence: an expand unit asks for
+//     its job's fragments and repeats the request (bounded) until every tag is this launch's.  Units are handed out
+//     in order and every worker is fed its units in order, so the unit with the smallest number that is not
+//     finished can always proceed: no deadlock while all CTAs are resident (grid = number of SMs, one CTA per SM).
 //   * Both contractions run on mma.sync m16n8k16 fed by ldmatrix from the operand images (the images are
-//     8 x 16-byte core matrices, exactly what ldmatrix reads without bank conflicts).  The path is bound by the
-//     adapter stream; the tensor cores are used for the instruction count.
+//     8 x 16-byte core matrices, exactly what ldmatrix reads).  The path is bound by the adapter stream; the tensor
+//     cores are used for the instruction count.
 //     shrink: M = rank rows, N = rows of x, K = columns of d1.
 //     expand: M = columns of d2, N = (row t, value | remainder), K = rank rows; the products are added to y with
-//     red.global.add.noftz.bf16: y never travels to the SM, every element of y receives exactly one addition
+//     red.global.add.noftz.bf16x2: y never travels to the SM, every element of y receives exactly one addition
 //     (deterministic), and its error is half an ulp of y plus the bf16 rounding of the term (2^-9 of it).
-//   * The job states and the unit counter clean themselves up (last expand unit of a job, last worker of the grid),
-//     so a launch leaves the scratch ready for the next one.
+//   * The job counters and the unit counter clean themselves up (the unit that adds a job up, the scheduler that
+//     finishes last), so a launch leaves the scratch ready for the next one.
 #include <algorithm>
 #include <cstring>
 
@@ -43,19 +47,19 @@ constexpr int kR = kGatherRows;
 constexpr int kBufs = 2;                         // buffers (stages in flight) per worker
 constexpr int kRowPad = 16;                      // keeps the rows of one stage on different banks
 constexpr int kStaticRounds = 2;                 // units per worker assigned by index before the counter is used
-constexpr int kUnitRing = 4;                     // unit records a worker keeps (issue runs ahead of compute)
 constexpr int kMaxSeg = 2 * kMaxStreamLayers * MILORA_NMOD;
-constexpr uint32_t kDepSpin = 1u << 22;          // polls of a job's ready flag before an expand unit gives up
+constexpr uint32_t kDepSpin = 1u << 22;          // repeats of a request for fragments or partial sums
+constexpr uint32_t kSchedSpin = 1u << 26;        // rounds of the scheduler loop
 constexpr int kMaxWarps = 10;
 
-// Two shapes of the kernel: many warps on small stages for the usual ranks (the warps hide each other's
-// latencies; 20 stages of 8 KB in flight per SM), fewer warps on 16 KB stages for padded ranks of 48 and 64,
-// whose smallest stage (one 128-column block of B) no longer fits 8 KB.
+// Two shapes of the kernel: ten workers on 8 KB stages for the usual ranks (the warps hide each other's
+// latencies; 20 stages in flight per SM), six on 16 KB stages for padded ranks of 48 and 64, whose smallest stage
+// (one 128-column block of B) no longer fits 8 KB.
 template <int WARPS, int STAGE>
 struct Shape {
-  static constexpr int kWarps = WARPS;
+  static constexpr int kWarps = WARPS;           // workers; the scheduler is one more warp
   static constexpr int kStageBytes = STAGE;
-  static constexpr int kThreads = WARPS * 32;
+  static constexpr int kThreads = (WARPS + 1) * 32;
 };
 using ShapeSmall = Shape<10, 8192>;
 using ShapeLarge = Shape<6, 16384>;
@@ -72,34 +76,35 @@ struct StreamArgs {
   int buf_stride;              // bytes from one buffer to the next: stage + kR rows of x, rounded up
   int unit_stages;             // stages per unit
   int kcmax;                   // most shrink units per job over the modules
-  uint32_t* ctrl;              // [0] units handed out beyond the static rounds, [1] workers that have finished
+  uint32_t* ctrl;              // [0] units handed out beyond the static rounds, [1] schedulers that have finished
   uint32_t* job_state;         // [jobs]: shrink units of the job that have delivered their partial sums
-  uint32_t epoch;              // tag of this launch (never 0): marks the fragments written by it
+  uint32_t epoch;              // tag of this launch (never 0): marks the values written by it
   uint2* partial;              // [jobs][kcmax][kR][rp] of {value, epoch}
   uint4* vfrag;                // [jobs][rp / 16][32] of {word 0, epoch, word 1, epoch}
 };
 
-struct UnitRec {               // what a worker needs to know about a unit, in shared memory
-  const char* img;             // operand image of the phase (A image for shrink, B image for expand)
-  const char* rows_base;       // X or Y of the module
-  int32_t rows[kR];
-  float gate[kR];
-  float scale;
-  int32_t n, rp, rank;
-  int32_t d, phase, module;
-  int32_t stage0, n_stages;    // stage range of the job's phase covered by this unit
-  int32_t job, sub, upj_s, upj_e;
-  int32_t ok;
+// What a worker needs to know about the stage in one of its buffers; written by the scheduler before it starts
+// the stage's copies, read by the worker after the buffer's barrier has completed.
+enum StageKind { STAGE_SHRINK = 0, STAGE_EXPAND = 1, STAGE_STOP = 2 };
+struct StageDesc {
+  char* y_base;                // expand: first element of the module's Y
+  int32_t rows[kR];            // expand: rows of y
+  float w[kR];                 // shrink: scale * gate of each row of the job (used when the unit ends)
+  int32_t kind, n, jb, ncols;  // rows of the job, rank blocks of 16, columns of this stage
+  int32_t c0, d;               // expand: first column of the stage, row length of y
+  int32_t first, last;         // first / last stage of its unit
+  int32_t job, sub, upj_s, pad;
 };
+static_assert(sizeof(StageDesc) == 88, "StageDesc layout");
 
 struct Smem {
   StreamLayer layers[kMaxStreamLayers];
   int32_t seg_base[kMaxSeg + 1];
   int32_t first[kMaxStreamLayers][MILORA_NMOD + 1];
   int32_t upj[2][MILORA_NMOD];
-  UnitRec unit[kMaxWarps][kUnitRing];
-  uint64_t full[kMaxWarps][kBufs];
-  int32_t buf_unit[kMaxWarps][kBufs], buf_stage[kMaxWarps][kBufs];
+  StageDesc desc[kMaxWarps][kBufs];
+  uint64_t full[kMaxWarps][kBufs], empty[kMaxWarps][kBufs];
+  volatile int32_t hint[kMaxWarps];   // job of the expand unit taken last for each worker (-1: none): what to ask fragments for
 };
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -161,110 +166,120 @@ __device__ __forceinline__ void pos_to_layer(int p, int L, int* li, int* phase) 
   else { *li = (p >> 1) - 1; *phase = 1; }
 }
 
-// ---- unit look-up ------------------------------------------------------------------------------------
-// In two halves, so that the 64-byte job record travels while the worker does something else: locate_unit finds
-// the unit's place in the work lists and asks for the record (lanes 0..3, 16 bytes each); fill_unit, called when the
-// worker needs the unit, hands the pieces around the warp, checks the record and writes the unit record.
+// ---- scheduler: one lane per worker -------------------------------------------------------------------------
+// A unit that has been found in the work lists and whose 64-byte job record is on its way (four 16-byte loads).
 struct UnitLoc {
   int li, phase, m, job_local, sub;
-  uint4 piece;
+  uint4 p0, p1, p2, p3;
+  bool valid;
 };
-__device__ __forceinline__ UnitLoc locate_unit(const StreamArgs& a, const Smem& sm, int n_seg, int u, int lane) {
+__device__ __forceinline__ UnitLoc locate_unit(const StreamArgs& a, const Smem& sm, int n_seg, int u) {
+  UnitLoc loc;
+  UnitLoc* x = &loc;
   // segment = (queue position, module): binary search over the prefix table
   int lo = 0, hi = n_seg;
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (sm.seg_base[mid] <= u) lo = mid; else hi = mid;
   }
-  UnitLoc x;
   const int p = lo / MILORA_NMOD;
-  x.m = lo % MILORA_NMOD;
-  pos_to_layer(p, a.n_layers, &x.li, &x.phase);
+  x->m = lo % MILORA_NMOD;
+  pos_to_layer(p, a.n_layers, &x->li, &x->phase);
   const int local = u - sm.seg_base[lo];
-  const int upj = sm.upj[x.phase][x.m];
-  x.job_local = sm.first[x.li][x.m] + local / upj;
-  x.sub = local % upj;
-  const StreamLayer& L = sm.layers[x.li];
-  const uint4* jp = reinterpret_cast<const uint4*>(L.ws + L.off_gather) + (size_t)x.job_local * (kJobInts / 4);
-  x.piece = make_uint4(0, 0, 0, 0);
-  if (lane < 4) x.piece = jp[lane];
-  return x;
+  const int upj = sm.upj[x->phase][x->m];
+  x->job_local = sm.first[x->li][x->m] + local / upj;
+  x->sub = local % upj;
+  const StreamLayer& L = sm.layers[x->li];
+  const uint4* jp = reinterpret_cast<const uint4*>(L.ws + L.off_gather) + (size_t)x->job_local * (kJobInts / 4);
+  x->p0 = jp[0]; x->p1 = jp[1]; x->p2 = jp[2]; x->p3 = jp[3];
+  x->valid = true;
+  return loc;
 }
-__device__ __forceinline__ void fill_unit(const StreamArgs& a, const Smem& sm, const UnitLoc& x, UnitRec* r, int lane) {
-  GatherJob job;
-  uint32_t* jw = reinterpret_cast<uint32_t*>(&job);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    jw[4 * i + 0] = __shfl_sync(0xffffffffu, x.piece.x, i);
-    jw[4 * i + 1] = __shfl_sync(0xffffffffu, x.piece.y, i);
-    jw[4 * i + 2] = __shfl_sync(0xffffffffu, x.piece.z, i);
-    jw[4 * i + 3] = __shfl_sync(0xffffffffu, x.piece.w, i);
-  }
+
+// A unit as the scheduler lane keeps it while it issues the unit's stages.
+struct Unit {
+  const char* img;             // operand image of the phase, at the unit's first stage
+  const char* rows0;           // shrink: X of the module at the unit's first column; expand: Y of the module
+  int32_t rows[kR];
+  float w[kR];
+  int32_t n, rp, d, phase, c_begin, n_stages, job, sub, upj_s;
+};
+// Checks the job record (a damaged one is skipped by its shrink and its expand units alike) and derives the unit.
+__device__ __forceinline__ bool decode_unit(const StreamArgs& a, const Smem& sm, const UnitLoc& x, Unit* un) {
   const StreamLayer& L = sm.layers[x.li];
-  const int m = x.m, phase = x.phase;
-  const int d1 = a.d1[m], d2 = a.d2[m];
-  const int rpj = (job.rank + 15) & ~15;
-  bool ok = job.rank > 0 && rpj <= a.rp && job.count > 0 && job.count <= kR && job.At != nullptr && job.module == m &&
+  const int m = x.m;
+  const char* At = reinterpret_cast<const char*>(((uint64_t)x.p0.y << 32) | x.p0.x);
+  const int rank = (int)x.p1.x, count = (int)x.p1.w;
+  const float scale = __uint_as_float(x.p1.y);
+  const int rows[kR] = {(int)x.p2.x, (int)x.p2.y, (int)x.p2.z, (int)x.p2.w};
+  const float gate[kR] = {__uint_as_float(x.p3.x), __uint_as_float(x.p3.y), __uint_as_float(x.p3.z), __uint_as_float(x.p3.w)};
+  const int rpj = (rank + 15) & ~15;
+  bool ok = rank > 0 && rpj <= a.rp && count > 0 && count <= kR && At != nullptr && (int)x.p1.z == m &&
             L.X[m] != nullptr && L.Y[m] != nullptr;
 #pragma unroll
   for (int t = 0; t < kR; ++t)
-    if (t < job.count && (job.rows[t] < 0 || job.rows[t] >= L.T)) ok = false;
-  if (lane == 0) {
-    const int d = phase ? d2 : d1;
-    const int stages = (d + a.cols - 1) / a.cols;
-    const AdapterLayout al = adapter_layout(d1, d2, ok ? job.rank : 1, 2);
-    r->img = static_cast<const char*>(job.At) + (phase ? al.off_b_img : al.off_a_img);
-    r->rows_base = static_cast<const char*>(phase ? L.Y[m] : L.X[m]);
+    if (t < count && (rows[t] < 0 || rows[t] >= L.T)) ok = false;
+  if (!ok) return false;
+  const int d1 = a.d1[m], d2 = a.d2[m];
+  const int d = x.phase ? d2 : d1;
+  const int stages = (d + a.cols - 1) / a.cols;
+  const AdapterLayout al = adapter_layout(d1, d2, rank, 2);
+  un->c_begin = x.sub * a.unit_stages * a.cols;
+  // both images are contiguous in column order: rp * 2 bytes per column
+  un->img = At + (x.phase ? al.off_b_img : al.off_a_img) + (size_t)un->c_begin * rpj * 2;
+  un->rows0 = x.phase ? static_cast<const char*>(L.Y[m]) : static_cast<const char*>(L.X[m]) + (size_t)un->c_begin * 2;
 #pragma unroll
-    for (int t = 0; t < kR; ++t) { r->rows[t] = job.rows[t]; r->gate[t] = job.gate[t]; }
-    r->scale = job.scale;
-    r->n = job.count; r->rp = rpj; r->rank = job.rank;
-    r->d = d; r->phase = phase; r->module = m;
-    r->stage0 = x.sub * a.unit_stages;
-    r->n_stages = min(a.unit_stages, stages - x.sub * a.unit_stages);
-    r->job = L.job_base + x.job_local; r->sub = x.sub;
-    r->upj_s = sm.upj[0][m]; r->upj_e = sm.upj[1][m];
-    r->ok = ok ? 1 : 0;
+  for (int t = 0; t < kR; ++t) {
+    un->rows[t] = rows[t];
+    un->w[t] = t < count ? scale * gate[t] : 0.f;
   }
+  un->n = count; un->rp = rpj; un->d = d; un->phase = x.phase;
+  un->n_stages = min(a.unit_stages, stages - x.sub * a.unit_stages);
+  un->job = L.job_base + x.job_local; un->sub = x.sub; un->upj_s = sm.upj[0][m];
+  return true;
 }
 
-// ---- issue: the copies of one stage -------------------------------------------------------------------
-// Lane 0 only.  buf: shared address of the buffer; bar: its mbarrier.  A shrink stage also brings the job's rows
-// of x; an expand stage needs nothing but its piece of the B image (y is updated in place in global memory).
-__device__ __forceinline__ void issue_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf, uint32_t bar) {
-  const int c0 = (r.stage0 + stage_in_unit) * a.cols;
-  const int ncols = min(a.cols, r.d - c0);
-  // both images are contiguous in column order: rp * 2 bytes per column
-  const uint32_t bytes_img = (uint32_t)ncols * r.rp * 2;
-  const uint32_t bytes_row = (uint32_t)ncols * 2;
-  const int n_rows = r.phase == 0 ? r.n : 0;
+// Descriptor and copies of stage `is` of the unit into a free buffer of the worker.
+__device__ __forceinline__ void issue_stage(const StreamArgs& a, const Unit& un, int is, StageDesc* dsc, uint32_t buf,
+                                            uint32_t bar) {
+  const int c_off = is * a.cols;                       // columns from the unit's first one
+  const int ncols = min(a.cols, un.d - un.c_begin - c_off);
+  dsc->y_base = const_cast<char*>(un.rows0);
+#pragma unroll
+  for (int t = 0; t < kR; ++t) { dsc->rows[t] = un.rows[t]; dsc->w[t] = un.w[t]; }
+  dsc->kind = un.phase; dsc->n = un.n; dsc->jb = un.rp >> 4; dsc->ncols = ncols;
+  dsc->c0 = un.c_begin + c_off; dsc->d = un.d;
+  dsc->first = is == 0; dsc->last = is == un.n_stages - 1;
+  dsc->job = un.job; dsc->sub = un.sub; dsc->upj_s = un.upj_s; dsc->pad = 0;
+  const uint32_t bytes_img = (uint32_t)ncols * un.rp * 2, bytes_row = (uint32_t)ncols * 2;
+  const int n_rows = un.phase == 0 ? un.n : 0;
+  // the arrive releases the descriptor to the worker, whose wait on the barrier acquires it
   mbar_expect_tx(bar, bytes_img + (uint32_t)n_rows * bytes_row);
-  bulk_g2s(buf, r.img + (size_t)c0 * r.rp * 2, bytes_img, bar);
+  bulk_g2s(buf, un.img + (size_t)c_off * un.rp * 2, bytes_img, bar);
   const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
   for (int t = 0; t < n_rows; ++t)
-    bulk_g2s(buf + a.stage_bytes + t * rstride, r.rows_base + ((size_t)r.rows[t] * r.d + c0) * 2, bytes_row, bar);
+    bulk_g2s(buf + a.stage_bytes + t * rstride, un.rows0 + ((size_t)un.rows[t] * un.d + c_off) * 2, bytes_row, bar);
 }
 
-// ---- shrink: one stage into the unit's accumulators ---------------------------------------------------------
-// JB = rank blocks of 16.  The instructions of one 64-column chunk are grouped by kind (x fragments, ldmatrix, MMA)
-// so that independent ones follow each other: the asm statements keep their order, and a chain
-// ldmatrix -> mma -> next ldmatrix would run at one latency per step.  Consecutive k steps go to kAcc independent
-// accumulator sets, which are added when the unit ends.
+// ---- worker: shrink -------------------------------------------------------------------------------------------
+// One stage into the unit's accumulators.  JB = rank blocks of 16.  The instructions of one 64-column chunk are
+// grouped by kind (x fragments, ldmatrix, MMA) so that independent ones follow each other: the asm statements keep
+// their order, and a chain ldmatrix -> mma -> next ldmatrix would run at one latency per step.  Consecutive k steps
+// go to independent accumulator sets, which are added when the unit ends.
 // acc[s * JB + jb] is a 16 x 8 tile (rank rows jb*16.., rows of x): c0, c1 = (rank row g, x rows 2q, 2q+1),
 // c2, c3 = (rank row g + 8, same x rows).
 constexpr int kAccSets = 8;     // accumulator tiles a worker holds: steps-per-batch x JB
 template <int JB>
-__device__ __forceinline__ void shrink_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf,
-                                             float (&acc)[kAccSets][4], int lane) {
+__device__ __forceinline__ void shrink_stage(const StreamArgs& a, int n, int ncols, uint32_t buf, float (&acc)[kAccSets][4],
+                                             int lane) {
   constexpr int SB = JB <= 2 ? 4 : 2;          // k steps whose loads are issued together
   const int g = lane >> 2, q = lane & 3, mi = lane >> 3;
-  const int c0 = (r.stage0 + stage_in_unit) * a.cols;
-  const int ncols = min(a.cols, r.d - c0);
   constexpr int rp = JB * 16;
   const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
-  const bool x_ok = g < r.n;
+  const bool x_ok = g < n;
   const uint32_t xrow = buf + a.stage_bytes + (x_ok ? g : 0) * rstride + 4 * q;
-  // ldmatrix row address of this lane inside a 64-column chunk, for k step 0 and rank block 0
+  // ldmatrix row address of this lane inside a 64-column chunk, for k step 0 and rank block 0:
+  // core matrix (j / 8, k / 8) at ((k / 8) * (rp / 8) + j / 8) * 128
   const uint32_t lane_off = (uint32_t)(((mi >> 1) * (rp >> 3) + (mi & 1)) * 128 + (lane & 7) * 16);
   for (int kc = 0; kc < (ncols >> 6); ++kc) {
     const uint32_t chunk = buf + (uint32_t)kc * rp * 128 + lane_off;
@@ -304,11 +319,12 @@ struct PendingCount {
   bool valid;
 };
 template <int JB>
-__device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRec& r, float (&acc)[kAccSets][4],
+__device__ __forceinline__ void shrink_publish(const StreamArgs& a, const StageDesc& dsc, float (&acc)[kAccSets][4],
                                                PendingCount* pc, int lane) {
   constexpr int SB = JB <= 2 ? 4 : 2;
   const int g = lane >> 2, q = lane & 3;
-  uint2* part = a.partial + ((size_t)r.job * a.kcmax + r.sub) * kR * a.rp;
+  const int job = dsc.job;
+  uint2* part = a.partial + ((size_t)job * a.kcmax + dsc.sub) * kR * a.rp;
   if (q < 2) {
 #pragma unroll
     for (int jb = 0; jb < JB; ++jb) {
@@ -326,14 +342,13 @@ __device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRe
       st_tagged1(part + (2 * q + 1) * a.rp + j + 8, __float_as_uint(c[3]), a.epoch);
     }
   }
-  const int t = g >> 1;
-  pc->job = r.job; pc->upj_s = r.upj_s; pc->jb = JB;
-  pc->w = (t < r.n) ? r.scale * r.gate[t] : 0.f;
+  pc->job = job; pc->upj_s = dsc.upj_s; pc->jb = JB;
+  pc->w = dsc.w[g >> 1];
   pc->valid = true;
   pc->old = 0;
   // The count only decides who adds the job up; the partial sums carry this launch's tag, so no fence is needed
   // (a fence here would wait for every addition into y that this warp still has under way).
-  if (lane == 0) pc->old = atomicAdd(a.job_state + r.job, 1u);
+  if (lane == 0) pc->old = atomicAdd(a.job_state + job, 1u);
 }
 
 // Second half: the unit that arrived last adds the job's partial sums in unit order and publishes v as the
@@ -399,22 +414,20 @@ __device__ __forceinline__ bool shrink_finalize(const StreamArgs& a, PendingCoun
   return all_ok;
 }
 
-// ---- expand: one stage, added to y in global memory -----------------------------------------------------------
-// KS = rank blocks of 16.  NS steps of 16 columns are handled together, again grouped by kind of instruction.
+// ---- worker: expand -------------------------------------------------------------------------------------------
+// One stage, added to y in global memory.  KS = rank blocks of 16.  NS steps of 16 columns are handled together,
+// again grouped by kind of instruction.
 template <int KS>
-__device__ __forceinline__ void expand_stage(const StreamArgs& a, const UnitRec& r, int stage_in_unit, uint32_t buf,
-                                             const uint2 (&vb)[kImagePadMax / 16], int lane) {
+__device__ __forceinline__ void expand_stage(const StageDesc& dsc, uint32_t buf, const uint2 (&vb)[kImagePadMax / 16], int lane) {
   constexpr int NS = KS <= 2 ? 8 / KS : 2;
   constexpr int rp = KS * 16;
   const int g = lane >> 2, q = lane & 3, mi = lane >> 3;
-  const int c0 = (r.stage0 + stage_in_unit) * a.cols;
-  const int ncols = min(a.cols, r.d - c0);
-  const bool row_ok = q < r.n;
+  const int ncols = dsc.ncols;
+  const bool row_ok = q < dsc.n;
   // ldmatrix takes any eight rows for a matrix: the first M half of a step is given the step's even columns and
   // the second half the odd ones, so that the accumulators of this lane are columns 2g and 2g + 1 of row t = q:
   // two neighbouring elements of y, which one packed addition updates.
-  __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(const_cast<char*>(r.rows_base)) +
-                      (size_t)(row_ok ? r.rows[q] : 0) * r.d + c0 + 2 * g;
+  __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(dsc.y_base) + (size_t)(row_ok ? dsc.rows[q] : 0) * dsc.d + dsc.c0 + 2 * g;
   // row address inside a 128-column block for rank step 0, column step 0: column n of the block sits in
   // core matrix (n / 8, k / 8) at ((k / 8) * 16 + n / 8) * 128, row n % 8
   const int n_loc = 2 * (lane & 7) + (mi & 1);
@@ -451,210 +464,225 @@ __device__ __forceinline__ void expand_stage(const StreamArgs& a, const UnitRec&
 // ---- the kernel --------------------------------------------------------------------------------------------
 template <class SH>
 __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamArgs a) {
-  constexpr int kWarps = SH::kWarps, kThreads = SH::kThreads;
+  constexpr int kWarps = SH::kWarps;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw + (size_t)kWarps * kBufs * a.buf_stride);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int L = a.n_layers;
-  const int n_seg = 2 * L * MILORA_NMOD;
   if (tid == 0) {
-    for (int w = 0; w < kWarps; ++w)
-      for (int b = 0; b < kBufs; ++b) mbar_init(smem_u32(&sm.full[w][b]), 1);
+    for (int w = 0; w < kWarps; ++w) {
+      for (int b = 0; b < kBufs; ++b) {
+        mbar_init(smem_u32(&sm.full[w][b]), 1);
+        mbar_init(smem_u32(&sm.empty[w][b]), 1);
+      }
+      sm.hint[w] = -1;
+    }
     fence_barrier_init();
   }
   pdl_launch_dependents();
+  __syncthreads();
   pdl_wait();
 
-  // ---- layer records and the unit table (every CTA builds the same one) ----
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(a.layers ? a.layers : &a.one);
-    uint4* dst = reinterpret_cast<uint4*>(sm.layers);
-    if (a.layers) {
-      for (int i = tid; i < L * (int)(sizeof(StreamLayer) / 16); i += kThreads) dst[i] = src[i];
-    } else if (tid == 0) {
-      sm.layers[0] = a.one;
-    }
-    if (tid < MILORA_NMOD) {
-      const int ss = (a.d1[tid] + a.cols - 1) / a.cols, se = (a.d2[tid] + a.cols - 1) / a.cols;
-      sm.upj[0][tid] = (ss + a.unit_stages - 1) / a.unit_stages;
-      sm.upj[1][tid] = (se + a.unit_stages - 1) / a.unit_stages;
-    }
-  }
-  __syncthreads();
-  for (int i = tid; i < L * (MILORA_NMOD + 1); i += kThreads) {
-    const int li = i / (MILORA_NMOD + 1), m = i % (MILORA_NMOD + 1);
-    const StreamLayer& Ly = sm.layers[li];
-    const int n_jobs = max(0, min(Ly.ws[Ly.off_header + H_NGATHER], Ly.max_gather));
-    sm.first[li][m] = max(0, min(Ly.ws[Ly.off_mod_gather + m], n_jobs));
-  }
-  __syncthreads();
-  for (int i = tid; i < n_seg; i += kThreads) {
-    const int p = i / MILORA_NMOD, m = i % MILORA_NMOD;
-    int li, phase;
-    pos_to_layer(p, L, &li, &phase);
-    const StreamLayer& Ly = sm.layers[li];
-    int cnt = max(0, sm.first[li][m + 1] - sm.first[li][m]) * sm.upj[phase][m];
-    if (Ly.X[m] == nullptr || Ly.Y[m] == nullptr) cnt = 0;
-    sm.seg_base[i + 1] = cnt;       // counts first, prefix sums below
-  }
-  __syncthreads();
-  if (warp == 0) {
-    // inclusive scan of seg_base[1..n_seg] by one warp, 32 entries per pass
-    int carry = 0;
-    for (int b = 0; b < n_seg; b += 32) {
-      const int i = b + lane;
-      int v = (i < n_seg) ? sm.seg_base[i + 1] : 0;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= o) v += t;
+  if (warp == kWarps) {
+    // ================= scheduler =================
+    const int L = a.n_layers;
+    const int n_seg = 2 * L * MILORA_NMOD;
+    // layer records and the unit table
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(a.layers);
+      uint4* dst = reinterpret_cast<uint4*>(sm.layers);
+      if (a.layers) {
+        for (int i = lane; i < L * (int)(sizeof(StreamLayer) / 16); i += 32) dst[i] = src[i];
+      } else if (lane == 0) {
+        sm.layers[0] = a.one;
       }
-      if (i < n_seg) sm.seg_base[i + 1] = carry + v;
-      carry += __shfl_sync(0xffffffffu, v, 31);
+      if (lane < MILORA_NMOD) {
+        const int ss = (a.d1[lane] + a.cols - 1) / a.cols, se = (a.d2[lane] + a.cols - 1) / a.cols;
+        sm.upj[0][lane] = (ss + a.unit_stages - 1) / a.unit_stages;
+        sm.upj[1][lane] = (se + a.unit_stages - 1) / a.unit_stages;
+      }
     }
-    if (lane == 0) sm.seg_base[0] = 0;
-  }
-  __syncthreads();
-  const int total = sm.seg_base[n_seg];
+    __syncwarp();
+    for (int i = lane; i < L * (MILORA_NMOD + 1); i += 32) {
+      const int li = i / (MILORA_NMOD + 1), m = i % (MILORA_NMOD + 1);
+      const StreamLayer& Ly = sm.layers[li];
+      const int n_jobs = max(0, min(Ly.ws[Ly.off_header + H_NGATHER], Ly.max_gather));
+      sm.first[li][m] = max(0, min(Ly.ws[Ly.off_mod_gather + m], n_jobs));
+    }
+    __syncwarp();
+    {
+      // unit counts per (queue position, module), then their prefix sums, 32 entries per pass
+      int carry = 0;
+      if (lane == 0) sm.seg_base[0] = 0;
+      for (int b = 0; b < n_seg; b += 32) {
+        const int i = b + lane;
+        int v = 0;
+        if (i < n_seg) {
+          const int p = i / MILORA_NMOD, m = i % MILORA_NMOD;
+          int li, phase;
+          pos_to_layer(p, L, &li, &phase);
+          const StreamLayer& Ly = sm.layers[li];
+          v = max(0, sm.first[li][m + 1] - sm.first[li][m]) * sm.upj[phase][m];
+          if (Ly.X[m] == nullptr || Ly.Y[m] == nullptr) v = 0;
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, v, o);
+          if (lane >= o) v += t;
+        }
+        if (i < n_seg) sm.seg_base[i + 1] = carry + v;
+        carry += __shfl_sync(0xffffffffu, v, 31);
+      }
+    }
+    __syncwarp();
+    const int total = sm.seg_base[n_seg];
 
-  // ---- worker ----
-  const int n_workers = (int)gridDim.x * kWarps;
-  const int wid = warp * (int)gridDim.x + (int)blockIdx.x;     // neighbouring units go to different SMs
+    bool timed_out = false;
+    if (lane < kWarps) {
+      const int w = lane;
+      const int n_workers = (int)gridDim.x * kWarps;
+      const int wid = w * (int)gridDim.x + (int)blockIdx.x;     // neighbouring units go to different SMs
+      const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(w * kBufs) * a.buf_stride;
+      int n_fetched = 0, n_issued = 0, is = 0;
+      bool dry = false, have_cur = false, stop_sent = false;
+      uint32_t next_dyn = atomicAdd(&a.ctrl[0], 1u);     // used by the third look-ahead; the answer has time to come
+      UnitLoc q0, q1;
+      Unit cur;
+      auto fetch = [&]() -> UnitLoc {
+        UnitLoc none;
+        none.valid = false;
+        if (dry) return none;
+        int u;
+        if (n_fetched < kStaticRounds) {
+          u = wid + n_fetched * n_workers;
+        } else {
+          u = kStaticRounds * n_workers + (int)next_dyn;
+          next_dyn = atomicAdd(&a.ctrl[0], 1u);          // for the call after this one
+        }
+        ++n_fetched;
+        if (u >= total) { dry = true; return none; }
+        return locate_unit(a, sm, n_seg, u);
+      };
+      q0 = fetch();
+      q1 = fetch();
+      uint32_t round = 0;
+      for (; round < kSchedSpin && !stop_sent; ++round) {
+        if (!have_cur && q0.valid) {
+          const bool ok = decode_unit(a, sm, q0, &cur);
+          if (!ok && q0.sub == 0 && q0.phase == 0) atomicOr(a.err, ERR_BAD_ITEM);
+          q0 = q1;
+          q1 = fetch();
+          if (ok) {
+            have_cur = true;
+            is = 0;
+            if (cur.phase == 1) sm.hint[w] = cur.job;
+          }
+        }
+        if (have_cur || !q0.valid) {
+          // a stage of the current unit, or, when nothing is left, the descriptor that ends the worker
+          const int b = n_issued % kBufs, k = n_issued / kBufs;
+          const bool is_free = k == 0 || mbar_test_wait(smem_u32(&sm.empty[w][b]), (uint32_t)(k - 1) & 1u);
+          if (is_free) {
+            const uint32_t bar = smem_u32(&sm.full[w][b]);
+            if (have_cur) {
+              issue_stage(a, cur, is, &sm.desc[w][b], buf0 + b * a.buf_stride, bar);
+              if (++is == cur.n_stages) have_cur = false;
+            } else {
+              sm.desc[w][b].kind = STAGE_STOP;
+              mbar_arrive(bar);
+              stop_sent = true;
+            }
+            ++n_issued;
+          } else {
+            __nanosleep(32);
+          }
+        }
+      }
+      timed_out = !stop_sent;
+      __threadfence();        // a counter request that was never used must not pass the count of finished CTAs
+    }
+    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
+    __syncwarp();
+    // the unit counter is reset by the scheduler that finishes last
+    if (lane == 0) {
+      const uint32_t old = atomicAdd(&a.ctrl[1], 1u);
+      if (old == gridDim.x - 1) {
+        a.ctrl[0] = 0;
+        a.ctrl[1] = 0;
+      }
+    }
+    return;
+  }
+
+  // ================= worker =================
   const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(warp * kBufs) * a.buf_stride;
-  UnitRec* ring = sm.unit[warp];
-  int n_fetched = 0;              // units this worker has asked for so far
-  int n_kept = 0;                 // ... of which were valid (they take turns in the ring of unit records)
-  int n_issued = 0, n_done = 0;   // stages issued / consumed (buffer = count % kBufs, parity = (count / kBufs) & 1)
-  int iu = -1, is = 0;            // ring index and next stage of the unit being issued (-1: none)
-  bool failed = false, dry = false;
-  // Look-ahead: the two units after the one being issued are located and their records are on the way
-  // (pf0 is the next one); the counter value for the unit after those has been asked for (lane 0).
-  UnitLoc pf0, pf1;
-  bool pf0_valid = false, pf1_valid = false;
-  uint32_t next_dyn = 0;
   float acc[kAccSets][4];
   PendingCount pend;
   pend.valid = false;
-  uint4 vb_pf[kImagePadMax / 16];   // fragments of the expand unit taken last, asked for when it was taken
-  int vb_pf_unit = -1;
+  uint4 vb_pf[kImagePadMax / 16];      // fragments asked for ahead of time, and the job they belong to
+  int pf_job = -1;
   uint2 vb[kImagePadMax / 16];
-  int cu_loaded = -1;               // ring index of the unit whose fragments are in vb
-
-  // asks for one more unit (index, place in the lists, record load) into pf1
-  auto look_ahead = [&]() {
-    pf1_valid = false;
-    if (dry) return;
-    int u;
-    if (n_fetched < kStaticRounds) {
-      u = wid + n_fetched * n_workers;
-    } else {
-      u = kStaticRounds * n_workers + (int)__shfl_sync(0xffffffffu, next_dyn, 0);
-      if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);    // for the call after this one
-    }
-    ++n_fetched;
-    if (u >= total) { dry = true; return; }
-    pf1 = locate_unit(a, sm, n_seg, u, lane);
-    pf1_valid = true;
-  };
-  // makes the next located unit the one being issued (skipping damaged records) and looks one further ahead
-  auto take_unit = [&]() {
-    iu = -1;
-    while (pf0_valid) {
-      // at most kBufs earlier units still have stages in a buffer, so the record after the last kept one is free
-      const int slot = n_kept % kUnitRing;
-      fill_unit(a, sm, pf0, &ring[slot], lane);
-      __syncwarp();
-      const bool ok = ring[slot].ok != 0;
-      if (!ok && ring[slot].sub == 0 && ring[slot].phase == 0 && lane == 0) atomicOr(a.err, ERR_BAD_ITEM);
-      pf0 = pf1;
-      pf0_valid = pf1_valid;
-      look_ahead();
-      if (ok) {
-        ++n_kept; iu = slot; is = 0;
-        if (ring[slot].phase == 1) {
-          // an expand unit: ask for its fragments now; they are checked (and asked for again if the job's shrink
-          // units have not all finished yet) when its first stage is consumed
-          const uint4* vf = a.vfrag + (size_t)ring[slot].job * (a.rp >> 4) * 32;
-#pragma unroll
-          for (int ks = 0; ks < kImagePadMax / 16; ++ks)
-            if (ks < (ring[slot].rp >> 4)) vb_pf[ks] = ld_tagged(vf + ks * 32 + lane);
-          vb_pf_unit = slot;
-        }
-        return;
-      }
-    }
-  };
-
-  if (lane == 0) next_dyn = atomicAdd(&a.ctrl[0], 1u);
-  look_ahead();
-  pf0 = pf1;
-  pf0_valid = pf1_valid;
-  look_ahead();
-  take_unit();
-  while (true) {
-    // issue while a buffer is free
-    while (iu >= 0 && n_issued - n_done < kBufs) {
-      const int b = n_issued % kBufs;
-      const uint32_t buf = buf0 + b * a.buf_stride, bar = smem_u32(&sm.full[warp][b]);
-      if (lane == 0) {
-        sm.buf_unit[warp][b] = iu;
-        sm.buf_stage[warp][b] = is;
-        issue_stage(a, ring[iu], is, buf, bar);
-      }
-      ++n_issued;
-      if (++is == ring[iu].n_stages) take_unit();
-    }
-    if (n_done == n_issued) break;
-    // consume the oldest stage
+  bool failed = false;
+  const int ks_ctx = a.rp >> 4;
+  for (int n_done = 0;; ++n_done) {
     const int b = n_done % kBufs;
-    const uint32_t buf = buf0 + b * a.buf_stride, bar = smem_u32(&sm.full[warp][b]);
-    __syncwarp();
-    const int cu = sm.buf_unit[warp][b], cs = sm.buf_stage[warp][b];
-    const UnitRec& r = ring[cu];
-    const int jb = r.rp >> 4;
-    if (!mbar_wait(bar, (uint32_t)(n_done / kBufs) & 1u)) {
-      // the copies did not arrive: report, stop taking work, and give what is in flight a second (bounded) wait
-      // so that nothing lands in shared memory after the CTA has gone
-      if (lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
-      failed = true;
-      iu = -1;
-      pf0_valid = pf1_valid = false;
-      dry = true;
-      mbar_wait(bar, (uint32_t)(n_done / kBufs) & 1u);
-      ++n_done;
-      continue;
+    const uint32_t buf = buf0 + b * a.buf_stride;
+    // the scheduler says which job's expand unit comes next: ask for its fragments while waiting
+    {
+      const int hj = sm.hint[warp];
+      if (hj >= 0 && hj != pf_job) {
+        const uint4* vf = a.vfrag + (size_t)hj * ks_ctx * 32;
+#pragma unroll
+        for (int ks = 0; ks < kImagePadMax / 16; ++ks)
+          if (ks < ks_ctx) vb_pf[ks] = ld_tagged(vf + ks * 32 + lane);
+        pf_job = hj;
+      }
     }
-    if (r.phase == 0) {
-      if (cs == 0) {
+    if (!mbar_wait(smem_u32(&sm.full[warp][b]), (uint32_t)(n_done / kBufs) & 1u)) {
+      // nothing arrived within the limit: report and leave (the scheduler gives up on its own limit; copies that
+      // were started have had the same time to land)
+      failed = true;
+      break;
+    }
+    const StageDesc& dsc = sm.desc[warp][b];
+    const int kind = dsc.kind;
+    if (kind == STAGE_STOP) break;
+    const int jb = dsc.jb;
+    if (kind == STAGE_SHRINK) {
+      if (dsc.first) {
 #pragma unroll
         for (int i = 0; i < kAccSets; ++i)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
       }
+      const int n = dsc.n, ncols = dsc.ncols;
       switch (jb) {
-        case 1: shrink_stage<1>(a, r, cs, buf, acc, lane); break;
-        case 2: shrink_stage<2>(a, r, cs, buf, acc, lane); break;
-        case 3: shrink_stage<3>(a, r, cs, buf, acc, lane); break;
-        default: shrink_stage<4>(a, r, cs, buf, acc, lane); break;
+        case 1: shrink_stage<1>(a, n, ncols, buf, acc, lane); break;
+        case 2: shrink_stage<2>(a, n, ncols, buf, acc, lane); break;
+        case 3: shrink_stage<3>(a, n, ncols, buf, acc, lane); break;
+        default: shrink_stage<4>(a, n, ncols, buf, acc, lane); break;
       }
-      if (!shrink_finalize(a, &pend, lane)) failed = true;      // the count of the unit before this one has had a stage's time to answer
-      if (cs == r.n_stages - 1 && !failed) {
+      if (!shrink_finalize(a, &pend, lane)) failed = true;      // the count of the unit before this one has had time to answer
+      if (dsc.last) {
         switch (jb) {
-          case 1: shrink_publish<1>(a, r, acc, &pend, lane); break;
-          case 2: shrink_publish<2>(a, r, acc, &pend, lane); break;
-          case 3: shrink_publish<3>(a, r, acc, &pend, lane); break;
-          default: shrink_publish<4>(a, r, acc, &pend, lane); break;
+          case 1: shrink_publish<1>(a, dsc, acc, &pend, lane); break;
+          case 2: shrink_publish<2>(a, dsc, acc, &pend, lane); break;
+          case 3: shrink_publish<3>(a, dsc, acc, &pend, lane); break;
+          default: shrink_publish<4>(a, dsc, acc, &pend, lane); break;
         }
       }
     } else {
-      if (cs == 0 || cu_loaded != cu) {
-        // fragments of v: those asked for when the unit was taken, unless another unit was taken since
-        const uint4* vf = a.vfrag + (size_t)r.job * (a.rp >> 4) * 32;
+      bool have = true;
+      if (dsc.first) {
+        // fragments of v: those asked for ahead of time when they are this job's, asked for again until every tag
+        // is this launch's (the job's shrink units may not all have finished; the last of them may even be the
+        // count this very warp has not looked at yet)
+        const int job = dsc.job;
+        const uint4* vf = a.vfrag + (size_t)job * ks_ctx * 32;
         uint4 f[kImagePadMax / 16];
 #pragma unroll
         for (int ks = 0; ks < kImagePadMax / 16; ++ks) {
           f[ks] = make_uint4(0, a.epoch, 0, a.epoch);
-          if (ks < jb) f[ks] = (vb_pf_unit == cu) ? vb_pf[ks] : ld_tagged(vf + ks * 32 + lane);
+          if (ks < jb) f[ks] = (pf_job == job) ? vb_pf[ks] : ld_tagged(vf + ks * 32 + lane);
         }
         uint32_t spins = 0;
         while (true) {
@@ -662,48 +690,35 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
 #pragma unroll
           for (int ks = 0; ks < kImagePadMax / 16; ++ks) mine = mine && f[ks].y == a.epoch && f[ks].w == a.epoch;
           if (__all_sync(0xffffffffu, mine)) break;
-          if (++spins >= kDepSpin) break;
-          // the job's shrink units are not all done: its last one may be waiting behind this very stage
+          if (++spins >= kDepSpin) { have = false; break; }
           if (!shrink_finalize(a, &pend, lane)) failed = true;
           __nanosleep(100);
 #pragma unroll
           for (int ks = 0; ks < kImagePadMax / 16; ++ks)
             if (ks < jb) f[ks] = ld_tagged(vf + ks * 32 + lane);
         }
-        if (spins < kDepSpin) {
 #pragma unroll
-          for (int ks = 0; ks < kImagePadMax / 16; ++ks) vb[ks] = make_uint2(f[ks].x, f[ks].z);
-          cu_loaded = cu;
-        } else {
-          if (lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
+        for (int ks = 0; ks < kImagePadMax / 16; ++ks) vb[ks] = make_uint2(f[ks].x, f[ks].z);
+        if (!have) {
           failed = true;
-          cu_loaded = -1;
+#pragma unroll
+          for (int ks = 0; ks < kImagePadMax / 16; ++ks) vb[ks] = make_uint2(0, 0);     // the unit adds nothing
         }
       }
-      if (cu_loaded == cu) {
-        switch (jb) {
-          case 1: expand_stage<1>(a, r, cs, buf, vb, lane); break;
-          case 2: expand_stage<2>(a, r, cs, buf, vb, lane); break;
-          case 3: expand_stage<3>(a, r, cs, buf, vb, lane); break;
-          default: expand_stage<4>(a, r, cs, buf, vb, lane); break;
-        }
+      switch (jb) {
+        case 1: expand_stage<1>(dsc, buf, vb, lane); break;
+        case 2: expand_stage<2>(dsc, buf, vb, lane); break;
+        case 3: expand_stage<3>(dsc, buf, vb, lane); break;
+        default: expand_stage<4>(dsc, buf, vb, lane); break;
       }
       if (!shrink_finalize(a, &pend, lane)) failed = true;
     }
+    // every lane's reads of the buffer and of the descriptor are done (the MMAs needed them): hand it back
     __syncwarp();
-    ++n_done;
+    if (lane == 0) mbar_arrive(smem_u32(&sm.empty[warp][b]));
   }
   if (!shrink_finalize(a, &pend, lane)) failed = true;
   if (failed && lane == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
-  // the counter is reset by the worker that finishes last
-  if (lane == 0) {
-    __threadfence();        // a counter request that was never used must not pass the line below
-    const uint32_t old = atomicAdd(&a.ctrl[1], 1u);
-    if (old == (uint32_t)n_workers - 1) {
-      a.ctrl[0] = 0;
-      a.ctrl[1] = 0;
-    }
-  }
 }
 
 // Columns of d1 / d2 per stage: as many 128-column blocks as the stage holds at this padded rank.
