@@ -59,7 +59,8 @@ template <int WARPS, int STAGE>
 struct Shape {
   static constexpr int kWarps = WARPS;           // workers; the scheduler is one more warp
   static constexpr int kStageBytes = STAGE;
-  static constexpr int kThreads = (WARPS + 1) * 32;
+  static constexpr int kSched = 2;               // scheduler warps; each serves half of the workers
+  static constexpr int kThreads = (WARPS + kSched) * 32;
 };
 using ShapeSmall = Shape<10, 8192>;
 using ShapeLarge = Shape<6, 16384>;
@@ -83,27 +84,36 @@ struct StreamArgs {
   uint4* vfrag;                // [jobs][rp / 16][32] of {word 0, epoch, word 1, epoch}
 };
 
-// What a worker needs to know about the stage in one of its buffers; written by the scheduler before it starts
-// the stage's copies, read by the worker after the buffer's barrier has completed.
+// What a worker needs to know about its work.  The scheduler writes a unit's record when it takes the unit and
+// two words per stage before it starts the stage's copies; the worker reads both after the buffer's barrier has
+// completed (the scheduler's arrive on that barrier releases them).  A worker has at most kBufs + 1 units alive
+// (one per buffer, one being issued), so kUnitRing records take turns.
 enum StageKind { STAGE_SHRINK = 0, STAGE_EXPAND = 1, STAGE_STOP = 2 };
-struct StageDesc {
+constexpr int kUnitRing = 4;
+struct UnitRec {
   char* y_base;                // expand: first element of the module's Y
   int32_t rows[kR];            // expand: rows of y
   float w[kR];                 // shrink: scale * gate of each row of the job (used when the unit ends)
-  int32_t kind, n, jb, ncols;  // rows of the job, rank blocks of 16, columns of this stage
-  int32_t c0, d;               // expand: first column of the stage, row length of y
-  int32_t first, last;         // first / last stage of its unit
-  int32_t job, sub, upj_s, pad;
+  int32_t n, jb, d;            // rows of the job, rank blocks of 16, row length of y
+  int32_t job, sub, upj_s;
 };
-static_assert(sizeof(StageDesc) == 88, "StageDesc layout");
+struct StageWord {             // ncols | slot << 16 | first << 20 | last << 21 | kind << 22, then the first column
+  uint32_t bits;
+  int32_t c0;
+};
+__host__ __device__ inline uint32_t stage_bits(int ncols, int slot, bool first, bool last, int kind) {
+  return (uint32_t)ncols | (uint32_t)slot << 16 | (uint32_t)first << 20 | (uint32_t)last << 21 | (uint32_t)kind << 22;
+}
 
 struct Smem {
   StreamLayer layers[kMaxStreamLayers];
   int32_t seg_base[kMaxSeg + 1];
   int32_t first[kMaxStreamLayers][MILORA_NMOD + 1];
   int32_t upj[2][MILORA_NMOD];
-  StageDesc desc[kMaxWarps][kBufs];
+  UnitRec unit[kMaxWarps][kUnitRing];
+  StageWord stage[kMaxWarps][kBufs];
   uint64_t full[kMaxWarps][kBufs], empty[kMaxWarps][kBufs];
+  uint4 rec[kMaxWarps][3][4];         // job records of the units a scheduler lane has located (cp.async targets)
   volatile int32_t hint[kMaxWarps];   // job of the expand unit taken last for each worker (-1: none): what to ask fragments for
 };
 
@@ -167,54 +177,65 @@ __device__ __forceinline__ void pos_to_layer(int p, int L, int* li, int* phase) 
 }
 
 // ---- scheduler: one lane per worker -------------------------------------------------------------------------
-// A unit that has been found in the work lists and whose 64-byte job record is on its way (four 16-byte loads).
+// A unit that has been found in the work lists and whose 64-byte job record is on its way to shared memory
+// (cp.async: the lane holds no register for it and never waits when it asks).
 struct UnitLoc {
-  int li, phase, m, job_local, sub;
-  uint4 p0, p1, p2, p3;
+  int li, phase, m, job_local, sub, slot;      // slot: which of the lane's three record buffers the record goes to
   bool valid;
 };
-__device__ __forceinline__ UnitLoc locate_unit(const StreamArgs& a, const Smem& sm, int n_seg, int u) {
-  UnitLoc loc;
-  UnitLoc* x = &loc;
-  // segment = (queue position, module): binary search over the prefix table
-  int lo = 0, hi = n_seg;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (sm.seg_base[mid] <= u) lo = mid; else hi = mid;
-  }
-  const int p = lo / MILORA_NMOD;
-  x->m = lo % MILORA_NMOD;
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// `seg` is the lane's cursor into the prefix table: unit numbers only grow, so the search starts where the last
+// one ended.
+__device__ __forceinline__ void locate_unit(const StreamArgs& a, Smem& sm, int n_seg, int u, int w, int slot, int* seg,
+                                            UnitLoc* x) {
+  int sg = *seg;
+  while (sg + 1 < n_seg && sm.seg_base[sg + 1] <= u) ++sg;
+  *seg = sg;
+  const int p = sg / MILORA_NMOD;
+  x->m = sg - p * MILORA_NMOD;
   pos_to_layer(p, a.n_layers, &x->li, &x->phase);
-  const int local = u - sm.seg_base[lo];
+  const int local = u - sm.seg_base[sg];
   const int upj = sm.upj[x->phase][x->m];
-  x->job_local = sm.first[x->li][x->m] + local / upj;
-  x->sub = local % upj;
+  // local / upj for small non-negative numbers: the float quotient of (local + 0.5) is never close to an integer
+  const int jq = __float2int_rz(__fdividef((float)local + 0.5f, (float)upj));
+  x->job_local = sm.first[x->li][x->m] + jq;
+  x->sub = local - jq * upj;
   const StreamLayer& L = sm.layers[x->li];
   const uint4* jp = reinterpret_cast<const uint4*>(L.ws + L.off_gather) + (size_t)x->job_local * (kJobInts / 4);
-  x->p0 = jp[0]; x->p1 = jp[1]; x->p2 = jp[2]; x->p3 = jp[3];
+  const uint32_t dst = smem_u32(&sm.rec[w][slot][0]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) cp_async16(dst + 16 * i, jp + i);
+  cp_async_commit();
+  x->slot = slot;
   x->valid = true;
-  return loc;
 }
 
 // A unit as the scheduler lane keeps it while it issues the unit's stages.
 struct Unit {
   const char* img;             // operand image of the phase, at the unit's first stage
-  const char* rows0;           // shrink: X of the module at the unit's first column; expand: Y of the module
+  const char* x0;              // shrink: X of the module at the unit's first column
   int32_t rows[kR];
-  float w[kR];
-  int32_t n, rp, d, phase, c_begin, n_stages, job, sub, upj_s;
+  int32_t n, rp, d, phase, c_begin, n_stages, slot;
 };
-// Checks the job record (a damaged one is skipped by its shrink and its expand units alike) and derives the unit.
-__device__ __forceinline__ bool decode_unit(const StreamArgs& a, const Smem& sm, const UnitLoc& x, Unit* un) {
+// Checks the job record (a damaged one is skipped by its shrink and its expand units alike), derives the unit and
+// writes its record for the worker.
+__device__ __forceinline__ bool decode_unit(const StreamArgs& a, const Smem& sm, const UnitLoc& x, const uint4* piece,
+                                            Unit* un, UnitRec* rec) {
   const StreamLayer& L = sm.layers[x.li];
   const int m = x.m;
-  const char* At = reinterpret_cast<const char*>(((uint64_t)x.p0.y << 32) | x.p0.x);
-  const int rank = (int)x.p1.x, count = (int)x.p1.w;
-  const float scale = __uint_as_float(x.p1.y);
-  const int rows[kR] = {(int)x.p2.x, (int)x.p2.y, (int)x.p2.z, (int)x.p2.w};
-  const float gate[kR] = {__uint_as_float(x.p3.x), __uint_as_float(x.p3.y), __uint_as_float(x.p3.z), __uint_as_float(x.p3.w)};
+  const uint4 p0 = piece[0], p1 = piece[1], p2 = piece[2], p3 = piece[3];
+  const char* At = reinterpret_cast<const char*>(((uint64_t)p0.y << 32) | p0.x);
+  const int rank = (int)p1.x, count = (int)p1.w;
+  const float scale = __uint_as_float(p1.y);
+  const int rows[kR] = {(int)p2.x, (int)p2.y, (int)p2.z, (int)p2.w};
+  const float gate[kR] = {__uint_as_float(p3.x), __uint_as_float(p3.y), __uint_as_float(p3.z), __uint_as_float(p3.w)};
   const int rpj = (rank + 15) & ~15;
-  bool ok = rank > 0 && rpj <= a.rp && count > 0 && count <= kR && At != nullptr && (int)x.p1.z == m &&
+  bool ok = rank > 0 && rpj <= a.rp && count > 0 && count <= kR && At != nullptr && (int)p1.z == m &&
             L.X[m] != nullptr && L.Y[m] != nullptr;
 #pragma unroll
   for (int t = 0; t < kR; ++t)
@@ -224,41 +245,41 @@ __device__ __forceinline__ bool decode_unit(const StreamArgs& a, const Smem& sm,
   const int d = x.phase ? d2 : d1;
   const int stages = (d + a.cols - 1) / a.cols;
   const AdapterLayout al = adapter_layout(d1, d2, rank, 2);
+  const size_t off = x.phase ? al.off_b_img : al.off_a_img;
   un->c_begin = x.sub * a.unit_stages * a.cols;
   // both images are contiguous in column order: rp * 2 bytes per column
-  un->img = At + (x.phase ? al.off_b_img : al.off_a_img) + (size_t)un->c_begin * rpj * 2;
-  un->rows0 = x.phase ? static_cast<const char*>(L.Y[m]) : static_cast<const char*>(L.X[m]) + (size_t)un->c_begin * 2;
+  un->img = At + off + (size_t)un->c_begin * rpj * 2;
+  un->x0 = static_cast<const char*>(L.X[m]) + (size_t)un->c_begin * 2;
 #pragma unroll
-  for (int t = 0; t < kR; ++t) {
-    un->rows[t] = rows[t];
-    un->w[t] = t < count ? scale * gate[t] : 0.f;
-  }
+  for (int t = 0; t < kR; ++t) un->rows[t] = rows[t];
   un->n = count; un->rp = rpj; un->d = d; un->phase = x.phase;
   un->n_stages = min(a.unit_stages, stages - x.sub * a.unit_stages);
-  un->job = L.job_base + x.job_local; un->sub = x.sub; un->upj_s = sm.upj[0][m];
+  rec->y_base = static_cast<char*>(L.Y[m]);
+#pragma unroll
+  for (int t = 0; t < kR; ++t) {
+    rec->rows[t] = rows[t];
+    rec->w[t] = t < count ? scale * gate[t] : 0.f;
+  }
+  rec->n = count; rec->jb = rpj >> 4; rec->d = d;
+  rec->job = L.job_base + x.job_local; rec->sub = x.sub; rec->upj_s = sm.upj[0][m];
   return true;
 }
 
-// Descriptor and copies of stage `is` of the unit into a free buffer of the worker.
-__device__ __forceinline__ void issue_stage(const StreamArgs& a, const Unit& un, int is, StageDesc* dsc, uint32_t buf,
+// Stage `is` of the unit into a free buffer of the worker: its two words, then its copies.
+__device__ __forceinline__ void issue_stage(const StreamArgs& a, const Unit& un, int is, StageWord* sw, uint32_t buf,
                                             uint32_t bar) {
   const int c_off = is * a.cols;                       // columns from the unit's first one
   const int ncols = min(a.cols, un.d - un.c_begin - c_off);
-  dsc->y_base = const_cast<char*>(un.rows0);
-#pragma unroll
-  for (int t = 0; t < kR; ++t) { dsc->rows[t] = un.rows[t]; dsc->w[t] = un.w[t]; }
-  dsc->kind = un.phase; dsc->n = un.n; dsc->jb = un.rp >> 4; dsc->ncols = ncols;
-  dsc->c0 = un.c_begin + c_off; dsc->d = un.d;
-  dsc->first = is == 0; dsc->last = is == un.n_stages - 1;
-  dsc->job = un.job; dsc->sub = un.sub; dsc->upj_s = un.upj_s; dsc->pad = 0;
+  sw->bits = stage_bits(ncols, un.slot, is == 0, is == un.n_stages - 1, un.phase);
+  sw->c0 = un.c_begin + c_off;
   const uint32_t bytes_img = (uint32_t)ncols * un.rp * 2, bytes_row = (uint32_t)ncols * 2;
   const int n_rows = un.phase == 0 ? un.n : 0;
-  // the arrive releases the descriptor to the worker, whose wait on the barrier acquires it
+  // the arrive releases the words and the unit's record to the worker, whose wait on the barrier acquires them
   mbar_expect_tx(bar, bytes_img + (uint32_t)n_rows * bytes_row);
   bulk_g2s(buf, un.img + (size_t)c_off * un.rp * 2, bytes_img, bar);
   const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
   for (int t = 0; t < n_rows; ++t)
-    bulk_g2s(buf + a.stage_bytes + t * rstride, un.rows0 + ((size_t)un.rows[t] * un.d + c_off) * 2, bytes_row, bar);
+    bulk_g2s(buf + a.stage_bytes + t * rstride, un.x0 + ((size_t)un.rows[t] * un.d + c_off) * 2, bytes_row, bar);
 }
 
 // ---- worker: shrink -------------------------------------------------------------------------------------------
@@ -319,7 +340,7 @@ struct PendingCount {
   bool valid;
 };
 template <int JB>
-__device__ __forceinline__ void shrink_publish(const StreamArgs& a, const StageDesc& dsc, float (&acc)[kAccSets][4],
+__device__ __forceinline__ void shrink_publish(const StreamArgs& a, const UnitRec& dsc, float (&acc)[kAccSets][4],
                                                PendingCount* pc, int lane) {
   constexpr int SB = JB <= 2 ? 4 : 2;
   const int g = lane >> 2, q = lane & 3;
@@ -418,16 +439,16 @@ __device__ __forceinline__ bool shrink_finalize(const StreamArgs& a, PendingCoun
 // One stage, added to y in global memory.  KS = rank blocks of 16.  NS steps of 16 columns are handled together,
 // again grouped by kind of instruction.
 template <int KS>
-__device__ __forceinline__ void expand_stage(const StageDesc& dsc, uint32_t buf, const uint2 (&vb)[kImagePadMax / 16], int lane) {
+__device__ __forceinline__ void expand_stage(const UnitRec& dsc, int ncols, int c0, uint32_t buf,
+                                             const uint2 (&vb)[kImagePadMax / 16], int lane) {
   constexpr int NS = KS <= 2 ? 8 / KS : 2;
   constexpr int rp = KS * 16;
   const int g = lane >> 2, q = lane & 3, mi = lane >> 3;
-  const int ncols = dsc.ncols;
   const bool row_ok = q < dsc.n;
   // ldmatrix takes any eight rows for a matrix: the first M half of a step is given the step's even columns and
   // the second half the odd ones, so that the accumulators of this lane are columns 2g and 2g + 1 of row t = q:
   // two neighbouring elements of y, which one packed addition updates.
-  __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(dsc.y_base) + (size_t)(row_ok ? dsc.rows[q] : 0) * dsc.d + dsc.c0 + 2 * g;
+  __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(dsc.y_base) + (size_t)(row_ok ? dsc.rows[q] : 0) * dsc.d + c0 + 2 * g;
   // row address inside a 128-column block for rank step 0, column step 0: column n of the block sits in
   // core matrix (n / 8, k / 8) at ((k / 8) * 16 + n / 8) * 128, row n % 8
   const int n_loc = 2 * (lane & 7) + (mi & 1);
@@ -482,10 +503,13 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
   __syncthreads();
   pdl_wait();
 
-  if (warp == kWarps) {
+  if (warp >= kWarps) {
     // ================= scheduler =================
+    const int sched = warp - kWarps;
+    constexpr int kPerSched = (kWarps + SH::kSched - 1) / SH::kSched;
     const int L = a.n_layers;
     const int n_seg = 2 * L * MILORA_NMOD;
+    if (sched == 0) {
     // layer records and the unit table
     {
       const uint4* src = reinterpret_cast<const uint4*>(a.layers);
@@ -534,23 +558,25 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       }
     }
     __syncwarp();
+    }
+    // the other scheduler warps wait for the table
+    named_barrier(1, SH::kSched * 32);
     const int total = sm.seg_base[n_seg];
 
     bool timed_out = false;
-    if (lane < kWarps) {
-      const int w = lane;
+    if (lane < kPerSched && sched * kPerSched + lane < kWarps) {
+      const int w = sched * kPerSched + lane;
       const int n_workers = (int)gridDim.x * kWarps;
       const int wid = w * (int)gridDim.x + (int)blockIdx.x;     // neighbouring units go to different SMs
       const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(w * kBufs) * a.buf_stride;
-      int n_fetched = 0, n_issued = 0, is = 0;
+      int n_fetched = 0, n_located = 0, n_issued = 0, n_kept = 0, is = 0, seg = 0;
       bool dry = false, have_cur = false, stop_sent = false;
       uint32_t next_dyn = atomicAdd(&a.ctrl[0], 1u);     // used by the third look-ahead; the answer has time to come
       UnitLoc q0, q1;
       Unit cur;
-      auto fetch = [&]() -> UnitLoc {
-        UnitLoc none;
-        none.valid = false;
-        if (dry) return none;
+      auto fetch_q1 = [&]() {
+        q1.valid = false;
+        if (dry) return;
         int u;
         if (n_fetched < kStaticRounds) {
           u = wid + n_fetched * n_workers;
@@ -559,43 +585,52 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
           next_dyn = atomicAdd(&a.ctrl[0], 1u);          // for the call after this one
         }
         ++n_fetched;
-        if (u >= total) { dry = true; return none; }
-        return locate_unit(a, sm, n_seg, u);
+        if (u >= total) { dry = true; return; }
+        locate_unit(a, sm, n_seg, u, w, n_located % 3, &seg, &q1);
+        ++n_located;
       };
-      q0 = fetch();
-      q1 = fetch();
+      fetch_q1();
+      q0 = q1;
+      fetch_q1();
       uint32_t round = 0;
       for (; round < kSchedSpin && !stop_sent; ++round) {
         if (!have_cur && q0.valid) {
-          const bool ok = decode_unit(a, sm, q0, &cur);
+          // at most kBufs earlier units still have stages in a buffer, so the record after the last kept one is free
+          const int slot = n_kept % kUnitRing;
+          // the record of q0 was asked for before that of q1: all but the newest request must have landed
+          if (q1.valid) cp_async_wait<1>(); else cp_async_wait<0>();
+          const bool ok = decode_unit(a, sm, q0, sm.rec[w][q0.slot], &cur, &sm.unit[w][slot]);
           if (!ok && q0.sub == 0 && q0.phase == 0) atomicOr(a.err, ERR_BAD_ITEM);
           q0 = q1;
-          q1 = fetch();
+          fetch_q1();
           if (ok) {
             have_cur = true;
             is = 0;
-            if (cur.phase == 1) sm.hint[w] = cur.job;
+            cur.slot = slot;
+            ++n_kept;
+            if (cur.phase == 1) sm.hint[w] = sm.unit[w][slot].job;
           }
         }
-        if (have_cur || !q0.valid) {
-          // a stage of the current unit, or, when nothing is left, the descriptor that ends the worker
+        // stages of the current unit into every free buffer, or, when nothing is left, the word that ends the worker
+        bool progress = false;
+#pragma unroll
+        for (int rep = 0; rep < kBufs; ++rep) {
+          if (!(have_cur || (!q0.valid && !stop_sent))) break;
           const int b = n_issued % kBufs, k = n_issued / kBufs;
-          const bool is_free = k == 0 || mbar_test_wait(smem_u32(&sm.empty[w][b]), (uint32_t)(k - 1) & 1u);
-          if (is_free) {
-            const uint32_t bar = smem_u32(&sm.full[w][b]);
-            if (have_cur) {
-              issue_stage(a, cur, is, &sm.desc[w][b], buf0 + b * a.buf_stride, bar);
-              if (++is == cur.n_stages) have_cur = false;
-            } else {
-              sm.desc[w][b].kind = STAGE_STOP;
-              mbar_arrive(bar);
-              stop_sent = true;
-            }
-            ++n_issued;
+          if (k > 0 && !mbar_test_wait(smem_u32(&sm.empty[w][b]), (uint32_t)(k - 1) & 1u)) break;
+          const uint32_t bar = smem_u32(&sm.full[w][b]);
+          if (have_cur) {
+            issue_stage(a, cur, is, &sm.stage[w][b], buf0 + b * a.buf_stride, bar);
+            if (++is == cur.n_stages) have_cur = false;
           } else {
-            __nanosleep(32);
+            sm.stage[w][b].bits = stage_bits(0, 0, false, false, STAGE_STOP);
+            mbar_arrive(bar);
+            stop_sent = true;
           }
+          ++n_issued;
+          progress = true;
         }
+        if (!progress && have_cur) __nanosleep(32);
       }
       timed_out = !stop_sent;
       __threadfence();        // a counter request that was never used must not pass the count of finished CTAs
@@ -605,7 +640,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
     // the unit counter is reset by the scheduler that finishes last
     if (lane == 0) {
       const uint32_t old = atomicAdd(&a.ctrl[1], 1u);
-      if (old == gridDim.x - 1) {
+      if (old == gridDim.x * SH::kSched - 1) {
         a.ctrl[0] = 0;
         a.ctrl[1] = 0;
       }
@@ -643,18 +678,21 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       failed = true;
       break;
     }
-    const StageDesc& dsc = sm.desc[warp][b];
-    const int kind = dsc.kind;
+    const uint32_t bits = sm.stage[warp][b].bits;
+    const int kind = (int)(bits >> 22);
     if (kind == STAGE_STOP) break;
+    const int ncols = (int)(bits & 0xFFFFu), c0 = sm.stage[warp][b].c0;
+    const bool first = (bits >> 20) & 1u, last = (bits >> 21) & 1u;
+    const UnitRec& dsc = sm.unit[warp][(bits >> 16) & 15u];
     const int jb = dsc.jb;
     if (kind == STAGE_SHRINK) {
-      if (dsc.first) {
+      if (first) {
 #pragma unroll
         for (int i = 0; i < kAccSets; ++i)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
       }
-      const int n = dsc.n, ncols = dsc.ncols;
+      const int n = dsc.n;
       switch (jb) {
         case 1: shrink_stage<1>(a, n, ncols, buf, acc, lane); break;
         case 2: shrink_stage<2>(a, n, ncols, buf, acc, lane); break;
@@ -662,7 +700,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
         default: shrink_stage<4>(a, n, ncols, buf, acc, lane); break;
       }
       if (!shrink_finalize(a, &pend, lane)) failed = true;      // the count of the unit before this one has had time to answer
-      if (dsc.last) {
+      if (last) {
         switch (jb) {
           case 1: shrink_publish<1>(a, dsc, acc, &pend, lane); break;
           case 2: shrink_publish<2>(a, dsc, acc, &pend, lane); break;
@@ -672,7 +710,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       }
     } else {
       bool have = true;
-      if (dsc.first) {
+      if (first) {
         // fragments of v: those asked for ahead of time when they are this job's, asked for again until every tag
         // is this launch's (the job's shrink units may not all have finished; the last of them may even be the
         // count this very warp has not looked at yet)
@@ -706,10 +744,10 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
         }
       }
       switch (jb) {
-        case 1: expand_stage<1>(dsc, buf, vb, lane); break;
-        case 2: expand_stage<2>(dsc, buf, vb, lane); break;
-        case 3: expand_stage<3>(dsc, buf, vb, lane); break;
-        default: expand_stage<4>(dsc, buf, vb, lane); break;
+        case 1: expand_stage<1>(dsc, ncols, c0, buf, vb, lane); break;
+        case 2: expand_stage<2>(dsc, ncols, c0, buf, vb, lane); break;
+        case 3: expand_stage<3>(dsc, ncols, c0, buf, vb, lane); break;
+        default: expand_stage<4>(dsc, ncols, c0, buf, vb, lane); break;
       }
       if (!shrink_finalize(a, &pend, lane)) failed = true;
     }
