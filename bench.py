@@ -456,7 +456,7 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
             "by_decode_path": by_path, "one_call_all_layers": one_call}
 
 
-def run_decode_stack(step, device, peaks, n_layers=8, rounds=20):
+def run_decode_stack(step, device, peaks, n_layers=32, rounds=10):
     """The decode kernel in the setting it serves in: one launch per Transformer layer, back to back, each layer with
     its own routes and adapters (here the first `n_layers` layers of a LLaMA-2-7B stack; 7 call sites per launch).
     One round touches n_layers x ~27 MB of distinct adapters (more than L2), so every launch reads from HBM.
@@ -508,7 +508,7 @@ def run_mixed_step(step, device, iters=50):
             "device_error_flag": err}
 
 
-def run_decode_13b(device, peaks, n_layers=2, rounds=20):
+def run_decode_13b(device, peaks, n_layers=8, rounds=10):
     """The same chain on the LLaMA-2-13B shapes of the skewed-reuse workload (rank 32, 256 decode requests whose
     tenants follow Zipf(1.1) over 1000 ids, routes from 256-token prompts): ~100 MB of adapters per layer, two
     layers alternating so that a launch never finds its adapters in L2."""
@@ -530,7 +530,7 @@ def run_decode_13b(device, peaks, n_layers=2, rounds=20):
     return out
 
 
-def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=2, rounds=20):
+def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=8, rounds=10):
     """Decode-only batch sweep on the LLaMA-3-8B shapes (GQA k/v, rank 16, tenants = batch size): the same replayed
     chain as above for each batch size, two layers alternating, with either decode kernel set and with the
     library's own choice.  Small batches are bound by the launch, large ones by the adapter stream."""
@@ -554,6 +554,7 @@ def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=2
                     "algorithmic_bytes_per_layer": r["algorithmic_bytes_per_layer"],
                     "chosen": "split" if lw.ml.decode_path_for(b, b) == 2 else "cluster",
                     "us_per_layer_by_path": {k: v["us_per_layer"] for k, v in r["by_decode_path"].items()},
+                    "one_call_all_layers": r["one_call_all_layers"],
                     "device_error_flag": r["device_error_flag"]})
         lw.close()
         del Xd, Yd

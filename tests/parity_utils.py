@@ -56,7 +56,8 @@ def assert_apply_close(y_gpu, y_oracle, y_base, dtype: str, active_rows=None, wh
     if changed.any():
         d = delta_ref[changed]
         rms = np.sqrt(np.mean(d * d))
-        allowed = tol * np.maximum(np.abs(d), rms) + 2.0 * half_ulp(yr[changed], dtype)
+        # the stored y is rounded once (half an ulp); 1 % on top for the fp32 sums behind it
+        allowed = tol * np.maximum(np.abs(d), rms) + 1.01 * half_ulp(yr[changed], dtype)
         err = np.abs(yg[changed] - yr[changed])
         worst = float((err / allowed).max())
         assert worst <= 1.0, f"{what}: delta error is {worst:.3f}x the allowed bound"

@@ -38,22 +38,12 @@ def _sample_rows(cu, rng, per_seq=6):
     return np.array(sorted(set(rows)), dtype=np.int64)
 
 
-def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True, decode_path="auto"):
-    """One step in the bench's configuration: group, multi-site prefill apply, multi-site decode apply
-    (decode_path: which kernel set milora_apply_decode uses)."""
+def _apply_and_check(lw, li, groups, cu_h, token_slot, table_col, T, tag, rng, multi=True, decode_path="auto"):
+    """Multi-site prefill apply and decode apply of one layer on a grouped step; outputs against the oracle on
+    sampled rows, untouched rows bit for bit on the whole tensors."""
     w, ml = lw.w, lw.ml
     ml.set_decode_path(decode_path)
     layer = lw.layers[li]
-    cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
-    n_seq = slots.numel()
-    ws = ml.alloc_group_ws(1, n_seq, T)
-    ml.group(li, 1, cu, slots, n_seq, T, ws)
-    cu_h = cu.cpu().numpy()
-    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
-    g_o = R.group_layer(w, token_slot, table_col)
-    g_o["max_tenants"] = w.n_tenants
-    assert_groups_equal(read_group_block(ml, ws[0], n_seq, T), g_o, cu_h)
-    groups = ml.groups(ws[0], n_seq, T)
     Xs = [w.module_input(layer, m, T, tag, "cuda") for m in range(7)]
     Ybs = [w.base_output(layer, m, T, tag, "cuda") for m in range(7)]
     Ys = [y.clone() for y in Ybs]
@@ -67,9 +57,13 @@ def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True
             ml.apply_decode(li, m, Xs[m], Ys[m], groups)
     torch.cuda.synchronize()
     assert ml.poll_error() == 0
+    _check_outputs(w, layer, Xs, Ybs, Ys, cu_h, token_slot, table_col, rng)
+
+
+def _check_outputs(w, layer, Xs, Ybs, Ys, cu_h, token_slot, table_col, rng):
     rows = _sample_rows(cu_h, rng)
     slot_module = np.asarray(table_col)
-    for m in mods:
+    for m in range(7):
         active = torch.from_numpy(slot_module[token_slot] == m).cuda()
         # rows whose request routes elsewhere: bit-identical over the whole tensor
         assert torch.equal(Ys[m][~active], Ybs[m][~active]), f"module {m}: an unrouted row changed"
@@ -83,6 +77,94 @@ def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True
         idx = torch.from_numpy(sel).cuda()
         y_o = R.apply_site(w, layer, m, Xs[m][idx].cpu(), Ybs[m][idx].cpu(), token_slot, table_col, rows=sel)
         assert_apply_close(Ys[m][idx], y_o, Ybs[m][idx], w.dtype, what=f"{w.name} layer {layer} module {m}")
+
+
+def _check_step(lw, li, prefill_ids, decode_ids, table_col, tag, rng, multi=True, decode_path="auto"):
+    """One step in the bench's configuration: group, multi-site prefill apply, multi-site decode apply
+    (decode_path: which kernel set milora_apply_decode uses)."""
+    w, ml = lw.w, lw.ml
+    cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
+    n_seq = slots.numel()
+    ws = ml.alloc_group_ws(1, n_seq, T)
+    ml.group(li, 1, cu, slots, n_seq, T, ws)
+    cu_h = cu.cpu().numpy()
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
+    g_o = R.group_layer(w, token_slot, table_col)
+    g_o["max_tenants"] = w.n_tenants
+    assert_groups_equal(read_group_block(ml, ws[0], n_seq, T), g_o, cu_h)
+    _apply_and_check(lw, li, ml.groups(ws[0], n_seq, T), cu_h, token_slot, table_col, T, tag, rng, multi, decode_path)
+
+
+def _spread(n_layers):
+    """First, last and two layers inside the stack."""
+    return sorted({0, n_layers // 3, (2 * n_layers) // 3, n_layers - 1})
+
+
+def _full_stack(lw, prefill_ids, decode_ids, rng, max_excused, decode_path="auto"):
+    """Every layer of the workload: routes against the oracle in full, one grouping call for all layers compared
+    block by block, the step applied on four layers spread over the stack, and (when the step has decode rows) the
+    decode rows of ALL layers in one milora_apply_decode_layers call, checked on the same four layers against the
+    oracle and on every layer for rows that must stay untouched.  Returns the number of excused near-tie routes."""
+    w, ml = lw.w, lw.ml
+    L = len(lw.layers)
+    ids = sorted(set(int(i) for i in prefill_ids) | set(int(i) for i in decode_ids))
+    table = np.full((w.n_requests, L), -1, dtype=np.int32)
+    excused = 0
+    for li in range(L):
+        for i0 in range(0, len(ids), 64):
+            lw.route(li, ids[i0:i0 + 64])
+        tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+        _, margins = R.route_requests(w, lw.layers[li], ids, tmp)
+        col = ml.route_table_read(0, w.n_requests).numpy()[:, li]
+        excused += compare_routes(col[ids], tmp[ids, lw.layers[li]], margins)
+        table[:, li] = col          # the GPU's decisions downstream, so that an excused near tie cannot cascade
+    assert excused <= max_excused, f"{excused} near-tie route mismatches over {L} layers"
+    cu, slots, T = lw.seq_arrays(prefill_ids, decode_ids)
+    n_seq = slots.numel()
+    ws = ml.alloc_group_ws(L, n_seq, T)
+    ml.group(0, L, cu, slots, n_seq, T, ws)
+    cu_h = cu.cpu().numpy()
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
+    for li in range(L):
+        g_o = R.group_layer(w, token_slot, table[:, li])
+        g_o["max_tenants"] = w.n_tenants
+        assert_groups_equal(read_group_block(ml, ws[li], n_seq, T), g_o, cu_h)
+    for li in _spread(L):
+        _apply_and_check(lw, li, ml.groups(ws[li], n_seq, T), cu_h, token_slot, table[:, li], T, 50 + li, rng,
+                         decode_path=decode_path)
+    if len(decode_ids):
+        # the decode rows alone, every layer in one launch, every layer its own outputs
+        ml.set_decode_path("auto")
+        cu_d, slots_d, T_d = lw.seq_arrays([], decode_ids)
+        n_d = slots_d.numel()
+        ws_d = ml.alloc_group_ws(L, n_d, T_d)
+        ml.group(0, L, cu_d, slots_d, n_d, T_d, ws_d)
+        slot_d = slots_d.cpu().numpy()
+        Xs = [w.module_input(lw.layers[0], m, T_d, 90, "cuda") for m in range(7)]          # inputs shared by the layers
+        Ybs = [w.base_output(lw.layers[0], m, T_d, 90, "cuda") for m in range(7)]
+        Ys = [[y.clone() for y in Ybs] for _ in range(L)]
+        entries = [(li, ml.groups(ws_d[li], n_d, T_d), {m: (Xs[m], Ys[li][m]) for m in range(7)}) for li in range(L)]
+        ml.apply_decode_layers(ml.decode_layers(entries))
+        torch.cuda.synchronize()
+        assert ml.poll_error() == 0
+        cu_dh = cu_d.cpu().numpy()
+        for li in range(L):
+            if li in _spread(L):
+                # the adapters differ per layer; x and y_base are those of tag 90 for every layer
+                rows = np.arange(T_d)
+                for m in range(7):
+                    sel = rows[table[slot_d, li] == m]
+                    if sel.size == 0:
+                        continue
+                    idx = torch.from_numpy(sel).cuda()
+                    y_o = R.apply_site(w, lw.layers[li], m, Xs[m][idx].cpu(), Ybs[m][idx].cpu(), slot_d, table[:, li], rows=sel)
+                    assert_apply_close(Ys[li][m][idx], y_o, Ybs[m][idx], w.dtype, what=f"{w.name} one call, layer {li} module {m}")
+            for m in range(7):
+                active = torch.from_numpy(table[slot_d, li] == m).cuda()
+                assert torch.equal(Ys[li][m][~active], Ybs[m][~active]), f"layer {li} module {m}: an unrouted row changed"
+                if active.any():
+                    assert bool((Ys[li][m][active] != Ybs[m][active]).any(dim=1).all()), f"layer {li} module {m}: a routed row was not updated"
+    return excused
 
 
 def _route_and_check(lw, li, ids):
@@ -107,59 +189,52 @@ def test_config2_full_size_bench_configuration():
     _check_step(lw, 0, ids, [], table, tag=0, rng=rng)          # prefill rows (dense tiles)
     _check_step(lw, 0, [], ids, table, tag=1, rng=rng)          # decode rows (gathered)
     _check_step(lw, 0, [], ids, table, tag=4, rng=rng, decode_path="split")
+    _check_step(lw, 0, [], ids, table, tag=5, rng=rng, decode_path="stream")
     _check_step(lw, 0, ids[:8], ids[8:], table, tag=2, rng=rng, multi=False)   # mixed, per-site calls
     _check_step(lw, 0, ids, ids, table, tag=3, rng=rng)         # all prompts and all decode rows as one batch
     lw.close()
 
 
-def test_config3_shape_ragged_prefill_two_layers():
-    """LLaMA-2-7B prefill with prompt lengths U[128, 2048] and repeated tenants (2 of the 32 layers)."""
+def test_config3_full_stack_ragged_prefill():
+    """LLaMA-2-7B, all 32 layers registered: 32 prompts with lengths U[128, 2048] and repeated tenants; routes and
+    groupings on every layer, the segmented apply on four layers spread over the stack."""
     w = get_workload("c3")
-    w = scaled_workload(w, n_layers=2)
     w.gen_device = "cuda"
     lw = _loaded(w)
     ids = list(range(w.n_requests))
-    rng = np.random.default_rng(1)
-    for li in range(2):
-        table, excused = _route_and_check(lw, li, ids)
-        assert excused <= 3
-        _check_step(lw, li, ids, [], table, tag=li, rng=rng)
+    _full_stack(lw, ids, [], np.random.default_rng(1), max_excused=32)
     lw.close()
 
 
-def test_config4_shape_zipf_decode_one_layer():
-    """LLaMA-2-13B shapes, rank 32, 256 decode requests whose tenants follow Zipf(1.1) over 1000 ids
-    (only the drawn tenants are registered), 256-token prompts."""
+def test_config4_full_stack_zipf_decode():
+    """LLaMA-2-13B shapes, all 40 layers registered, rank 32, 256 decode requests whose tenants follow Zipf(1.1) over
+    1000 ids (every drawn tenant gets backing: about 110 tenants x 40 layers x 7 adapters), 256-token prompts:
+    routes (40 x 256) and groupings on every layer, the gathered apply on four layers with the two-launch kernels,
+    and the whole stack in one milora_apply_decode_layers call."""
     w = get_workload("c4")
-    w = scaled_workload(w, n_layers=1)
     w.gen_device = "cuda"
+    free, _ = torch.cuda.mem_get_info()
+    per_tenant = w.n_layers * sum(2 * 2 * w.rank * sum(w.dims(m)) for m in range(7))      # row-major + images, bf16
+    n_active = len(w.active_tenants())
+    assert per_tenant * n_active < 0.8 * free, f"{n_active} tenants x {per_tenant >> 20} MB do not fit this device"
     lw = _loaded(w)
     ids = list(range(w.n_requests))
-    table, excused = _route_and_check(lw, 0, ids)
-    assert excused <= 8
-    rng = np.random.default_rng(2)
     assert lw.ml.decode_path_for(len(ids), len(ids)) == 2       # a batch of this size takes the two-launch kernels
-    _check_step(lw, 0, [], ids, table, tag=0, rng=rng, decode_path="split")
-    _check_step(lw, 0, [], ids, table, tag=1, rng=rng, decode_path="cluster")
+    _full_stack(lw, [], ids, np.random.default_rng(2), max_excused=120, decode_path="auto")
+    rng = np.random.default_rng(22)
+    table = lw.ml.route_table_read(0, w.n_requests).numpy()
+    _check_step(lw, 0, [], ids, table[:, 0], tag=1, rng=rng, decode_path="cluster")
+    _check_step(lw, 39, [], ids, table[:, 39], tag=2, rng=rng, decode_path="stream")
     lw.close()
 
 
-def test_config5_shape_mixed_step_one_layer():
-    """LLaMA-3-8B GQA shapes: 8 prompts U[256, 4096] plus 192 decode rows in one step."""
+def test_config5_full_stack_mixed_step():
+    """LLaMA-3-8B GQA shapes, all 32 layers registered: 8 prompts U[256, 4096] plus 192 decode rows in one step."""
     w = get_workload("c5")
-    w = scaled_workload(w, n_layers=1)
     w.gen_device = "cuda"
     lw = _loaded(w)
-    ids = list(range(w.n_requests))
-    for i0 in range(0, len(ids), 64):
-        lw.route(0, ids[i0:i0 + 64])
-    table = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0].copy()
-    tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
-    pre = [int(i) for i in w.prefill_ids]
-    _, margins = R.route_requests(w, 0, pre, tmp)
-    assert compare_routes(table[pre], tmp[pre, 0], margins) <= 1
-    rng = np.random.default_rng(3)
-    _check_step(lw, 0, pre, [int(i) for i in w.decode_ids], table, tag=0, rng=rng)
+    _full_stack(lw, [int(i) for i in w.prefill_ids], [int(i) for i in w.decode_ids], np.random.default_rng(3),
+                max_excused=80)
     lw.close()
 
 
@@ -176,6 +251,7 @@ def test_decode_batch_sweep_small_batches():
             lw.route(0, ids[i0:i0 + 64])
         table = lw.ml.route_table_read(0, w.n_requests).numpy()[:, 0].copy()
         _check_step(lw, 0, [], ids, table, tag=b, rng=rng)
+        _check_step(lw, 0, [], ids, table, tag=b + 1, rng=rng, decode_path="stream")
         lw.close()
 
 
