@@ -152,7 +152,24 @@ struct RouteArgs {
   float* stats;       // [total_chunks][2]  (self-attention pooler: chunk max, chunk sum of exp)
   int32_t* sched;     // next dynamic unit; zero on entry, put back to zero by pass 2
   int layer, P, d, n_strips, rows;
+  int T_total;        // rows of H: every row range read from cu is checked against it
+  int max_chunks;     // rows of `partial` / `stats`: no unit beyond them is touched
 };
+
+// Row range of prompt p.  cu is a device array the host never sees: a range that is negative, reversed or beyond the
+// rows of H is treated as empty and raises ERR_BAD_ROW (both passes take the same decision, so the chunk numbering
+// stays consistent), and no chunk beyond the scratch the host sized from T_total is touched.
+__device__ __forceinline__ void prompt_rows(const RouteArgs& a, int p, int* lo, int* hi) {
+  const int l = a.cu[p], h = a.cu[p + 1];
+  if (l < 0 || h < l || h > a.T_total) {
+    atomicOr(a.tab.err, ERR_BAD_ROW);
+    *lo = 0;
+    *hi = 0;
+  } else {
+    *lo = l;
+    *hi = h;
+  }
+}
 
 // Router entry of prompt p, or nullptr when its slot is closed / its tenant has no router at this layer.
 __device__ __forceinline__ const RouterEntry* router_of(const RouteArgs& a, int p, int* slot_out) {
@@ -194,7 +211,9 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
     const int p = base + tid;
     int chunks = 0;
     if (p < a.P) {
-      const int n_p = a.cu[p + 1] - a.cu[p];
+      int row_lo, row_hi;
+      prompt_rows(a, p, &row_lo, &row_hi);
+      const int n_p = row_hi - row_lo;
       if (n_p > 0) chunks = (n_p + kRows - 1) / kRows;
       int slot;
       const RouterEntry* r = router_of(a, p, &slot);
@@ -238,9 +257,10 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
     }
     const int p = lo;
     const int pool = pool_sm[p];
-    if (pool < 0) continue;
+    if (pool < 0 || cg >= a.max_chunks) continue;
     const int rc = cg - chunk_start[p];
-    const int row_lo = a.cu[p], row_hi = a.cu[p + 1];
+    int row_lo, row_hi;
+    prompt_rows(a, p, &row_lo, &row_hi);
     int r0 = row_lo + rc * kRows;
     int nr = min(kRows, row_hi - r0);
     if (pool == MILORA_POOL_LAST) {             // only the prompt's last row is pooled; its last chunk holds it
@@ -324,7 +344,9 @@ __global__ void __launch_bounds__(kFinThreads) route_finalize_kernel(RouteArgs a
   // first scratch row of this prompt = number of chunks of the prompts before it
   int mine = 0;
   for (int q = tid; q < p; q += kFinThreads) {
-    const int n_q = a.cu[q + 1] - a.cu[q];
+    int q_lo, q_hi;
+    prompt_rows(a, q, &q_lo, &q_hi);
+    const int n_q = q_hi - q_lo;
     if (n_q > 0) mine += (n_q + kRows - 1) / kRows;
   }
 #pragma unroll
@@ -333,8 +355,12 @@ __global__ void __launch_bounds__(kFinThreads) route_finalize_kernel(RouteArgs a
   __syncthreads();
   int chunk0 = 0;
   for (int w = 0; w < kFinWarps; ++w) chunk0 += wsum[w];
-  const int n_p = a.cu[p + 1] - a.cu[p];
+  int p_lo, p_hi;
+  prompt_rows(a, p, &p_lo, &p_hi);
+  const int n_p = p_hi - p_lo;
   int n_chunks = n_p > 0 ? (n_p + kRows - 1) / kRows : 0;
+  // chunks beyond the scratch do not exist for pass 1 either: such a prompt stays "not routed"
+  if (chunk0 + n_chunks > a.max_chunks) n_chunks = 0;
   int slot;
   const RouterEntry* rp = router_of(a, p, &slot);
   if (!rp || n_chunks == 0) {
@@ -484,6 +510,7 @@ milora_status transpose(milora_ctx* ctx, const void* in, void* out, int rows, in
 struct RoutePlan {
   int n_strips, rows;
   size_t max_chunks, scratch_floats, max_units;
+  int T_total;
 };
 
 RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
@@ -500,6 +527,7 @@ RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
   pl.max_chunks = (size_t)T_total / kRows + P;
   pl.scratch_floats = pl.max_chunks * d + 2 * pl.max_chunks;
   pl.max_units = pl.max_chunks * pl.n_strips;
+  pl.T_total = T_total;
   return pl;
 }
 
@@ -515,6 +543,7 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   a.stats = scratch + pl.max_chunks * ctx->desc.d_model;
   a.sched = sched;
   a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_strips = pl.n_strips; a.rows = pl.rows;
+  a.T_total = pl.T_total; a.max_chunks = (int)pl.max_chunks;
   const size_t smem = (size_t)(2 * P + 1) * sizeof(int32_t);
   const bool f32 = ctx->desc.dtype == MILORA_F32;
   // pass 1: one wave of resident CTAs (a warp's first unit is assigned by index, so every CTA must start at once)

@@ -471,8 +471,15 @@ def test_route_is_fixed_by_the_prompt_alone():
         assert table[0, 0] == route0
         gen = _rand(rng, 4, d) * 3
         snapshot = table.copy()
-        # decode steps only read the table
+        # decode steps only read the table: each generated token gets its term on the module the PROMPT selected,
+        # whatever its own hidden state would have selected, and applying never writes the table
+        A, B = _rand(rng, d, 2), _rand(rng, 2, d)
         for step in range(4):
+            x = gen[step:step + 1]
+            y_base = _rand(rng, 1, d)
+            for module in range(O.N_MOD):
+                y = O.apply_module(y_base, x, [0], [0], table[:, 0], module, lambda t, m: (A, B, 2.0))
+                assert np.array_equal(y != y_base, np.full_like(y_base, module == route0, dtype=bool))
             assert np.array_equal(table, snapshot)
         if O.route_prompt(np.vstack([H, gen]), W)["route"] != route0:
             flips += 1

@@ -1,5 +1,6 @@
 """The oracle run over the tiny synthetic stack (config 1) and structure checks of the larger workloads."""
 import numpy as np
+import torch
 
 from oracle import milora_oracle as O
 from oracle import reference_run as R
@@ -64,3 +65,75 @@ def test_config1_full_stack_invariants():
     g = R.group_layer(w, token_slot, table[:, 0])
     assert g["n_excluded"] == 0 and len(g["perm"]) == T
     assert sorted(g["perm"].tolist()) == list(range(T))
+
+
+class _HandWorkload:
+    """Just enough of a workload for reference_run.route_requests, with hand-built tensors that differ per
+    tenant, layer and request, so that a mix-up of any index changes the logits."""
+    n_tenants, n_layers, d = 3, 2, 6
+    request_tenant = np.array([2, 0, 1, 2], dtype=np.int32)
+
+    def _t(self, *ids, shape):
+        base = sum((i + 1) * f for i, f in zip(ids, (0.37, 0.11, 0.05)))
+        n = int(np.prod(shape))
+        return torch.tensor(np.sin(base + 0.7 * np.arange(n)).reshape(shape), dtype=torch.float64)
+
+    def hidden(self, layer, request):
+        return self._t(layer, request, 5, shape=(3 + request, self.d))
+
+    def router(self, tenant, layer):
+        return self._t(tenant, layer, 1, shape=(self.d, 7))
+
+    def w_sa(self, tenant, layer):
+        return self._t(tenant, layer, 2, shape=(self.d,))
+
+    def router_bias(self, tenant, layer):
+        return self._t(tenant, layer, 3, shape=(7,))
+
+    def rational_coef(self, tenant, layer):
+        c = self._t(tenant, layer, 4, shape=(12,)) * 0.3
+        return c[:7].clone(), c[7:].clone()
+
+
+def test_route_requests_hands_the_right_tensors_to_the_oracle():
+    """The variant branches of reference_run.route_requests (self-attention pooling, rational activation, bias,
+    top-k table) against direct calls of the oracle with the tensors picked by hand for each request's tenant and
+    the layer; picking another tenant's or layer's tensor changes the logits, so the comparison has power."""
+    w = _HandWorkload()
+    layer, ids, k = 1, [3, 0, 2], 3
+    table = np.full((4, 2), -1, dtype=np.int32)
+    topk = np.full((4, 2, k), -1, dtype=np.int32)
+    logits, margins = R.route_requests(w, layer, ids, table, pooler=O.POOL_SELFATTN, activation=O.ACT_RATIONAL,
+                                       with_bias=True, k=k, topk_table=topk)
+    for p, i in enumerate(ids):
+        t = int(w.request_tenant[i])
+        a, b = w.rational_coef(t, layer)
+        want = O.route_prompt(w.hidden(layer, i).numpy(), w.router(t, layer).numpy(), pooler=O.POOL_SELFATTN,
+                              activation=O.ACT_RATIONAL, k=k, w_sa=w.w_sa(t, layer).numpy(), coef_a=a.numpy(),
+                              coef_b=b.numpy(), bias=w.router_bias(t, layer).numpy())
+        assert np.array_equal(logits[p], want["logits"]) and margins[p] == want["margin"]
+        assert table[i, layer] == want["route"] and topk[i, layer].tolist() == list(want["topk"])
+        assert topk[i, layer, 0] == table[i, layer]
+        # each ingredient matters: another tenant's query column, coefficients or bias, or another layer's router
+        other = (t + 1) % 3
+        for kw in ({"w_sa": w.w_sa(other, layer).numpy()}, {"coef_a": w.rational_coef(other, layer)[0].numpy()},
+                   {"bias": w.router_bias(other, layer).numpy()}):
+            args = dict(w_sa=w.w_sa(t, layer).numpy(), coef_a=a.numpy(), coef_b=b.numpy(), bias=w.router_bias(t, layer).numpy())
+            args.update(kw)
+            wrong = O.route_prompt(w.hidden(layer, i).numpy(), w.router(t, layer).numpy(), pooler=O.POOL_SELFATTN,
+                                   activation=O.ACT_RATIONAL, k=k, **args)
+            assert not np.allclose(wrong["logits"], logits[p])
+        wrong = O.route_prompt(w.hidden(layer, i).numpy(), w.router(t, 0).numpy(), pooler=O.POOL_SELFATTN,
+                               activation=O.ACT_RATIONAL, k=k, w_sa=w.w_sa(t, layer).numpy(), coef_a=a.numpy(),
+                               coef_b=b.numpy(), bias=w.router_bias(t, layer).numpy())
+        assert not np.allclose(wrong["logits"], logits[p])
+    # rows of requests that were not routed, and the other layer, stay untouched
+    assert table[1, layer] == -1 and (table[:, 0] == -1).all() and (topk[:, 0] == -1).all()
+    # the plain branch: no bias, mean pooling, tanh, top-1 (no top-k table)
+    table2 = np.full((4, 2), -1, dtype=np.int32)
+    lo2, _ = R.route_requests(w, 0, [1], table2)
+    want = O.route_prompt(w.hidden(0, 1).numpy(), w.router(0, 0).numpy())
+    assert np.array_equal(lo2[0], want["logits"]) and table2[1, 0] == want["route"]
+    # a caller-supplied hidden-state function replaces the workload's own
+    lo3, _ = R.route_requests(w, 0, [1], table2, hidden=lambda i: w.hidden(1, 2))
+    assert np.array_equal(lo3[0], O.route_prompt(w.hidden(1, 2).numpy(), w.router(0, 0).numpy())["logits"])

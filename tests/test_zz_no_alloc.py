@@ -1,12 +1,15 @@
-"""milora_route_static against milora_route.
+"""milora_route_static against milora_route and against the oracle, and that it allocates nothing.
 
 Some callers of this library cannot allocate device memory while they serve: an inference engine whose
 memory pool has taken the whole GPU, code running while the allocator is frozen, or a latency path that
 cannot afford the device-wide synchronisation a cudaMalloc/cudaFree implies.  milora_route may grow a
 scratch buffer; milora_route_static keeps its scratch in a fixed array inside the library instead.  Both
-must write the same route table, logits and probabilities.  The fixed array is shared by all calls and
-keeps the previous call's contents, so the comparison is made on two calls in a row, with different
-prompts, and the second call must not be disturbed by what the first one left behind.
+must write the same route table, logits and probabilities, and both are compared with the fp64 oracle (the
+two entry points share their kernels, so agreeing with each other alone would not show a fault in what they
+share).  The fixed array is shared by all calls and keeps the previous call's contents, so the comparison is
+made on two calls in a row, with different prompts, and the second call must not be disturbed by what the first
+one left behind.  The static call is also made first on a fresh context, with a batch larger than any before,
+and the device's free memory must be the same before and after it.
 
 This file sorts last on purpose: a run that stops at the first failure has then run every other test.
 """
@@ -14,8 +17,12 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import milora_oracle as O
+from oracle import reference_run as R
 from synth import get_workload
 from synth.workloads import scaled_workload
+
+from parity_utils import compare_routes
 
 pytestmark = pytest.mark.gpu
 
@@ -59,6 +66,44 @@ def test_route_static_matches_route_on_two_calls_in_a_row(dtype):
         scale = max(1e-3, float(np.abs(logits_d).max()))
         assert np.abs(logits_s - logits_d).max() <= TOL * scale
         assert np.abs(probs_s - probs_d).max() <= TOL
+        # and against the oracle: routes bit-exact (near ties excused and counted), logits to fp32 accumulation
+        tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+        lo, margins = R.route_requests(w, lw.layers[li], ids, tmp)
+        assert compare_routes(table_s[ids, li], tmp[ids, lw.layers[li]], margins) <= 1
+        assert np.abs(logits_s - lo).max() <= 2e-4 * max(1e-3, float(np.abs(lo).max()))
+        np.testing.assert_allclose(probs_s, O.softmax(lo), atol=2e-4)
+    assert lw.ml.poll_error() == 0
+    lw.close()
+
+
+def test_route_static_allocates_nothing():
+    """The static call first on a fresh context, with a batch larger than any this context has seen: the free
+    memory of the device is the same before and after (every tensor of the test exists before the first reading)."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    base = get_workload("c1")
+    lens = np.array([900, 700, 64, 1], dtype=np.int32)
+    w = scaled_workload(base, name="no_alloc_fresh", dtype="bf16", d_model=1024, d_ff=2816, d_kv=256, n_tenants=2,
+                        request_tenant=np.array([0, 1, 0, 1], dtype=np.int32), prompt_len=lens, prefill_ids=np.arange(4),
+                        decode_ids=np.zeros(0, dtype=np.int64), has_base_weights=False, n_layers=1)
+    lw = LoadedWorkload(w, "cuda", register_adapters=False)
+    ids = [0, 1, 2, 3]
+    H = w.hidden_batch(0, ids, "cuda")
+    cu = torch.from_numpy(w.cu_seqlens(ids)).cuda()
+    slots = torch.tensor(ids, dtype=torch.int32, device="cuda")
+    logits = torch.zeros((4, 7), device="cuda")
+    probs = torch.zeros((4, 7), device="cuda")
+    lw.ml.route_static(0, H[:64], cu[:2].clone().fill_(0), slots[:1], logits[:1], probs[:1])   # set-up call (looks the array up)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    lw.ml.route_static(0, H, cu, slots, logits, probs)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "milora_route_static changed the device's free memory"
+    tmp = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
+    lo, margins = R.route_requests(w, 0, ids, tmp)
+    table = lw.ml.route_table_read(0, w.n_requests).numpy()
+    assert compare_routes(table[ids, 0], tmp[ids, 0], margins) == 0
+    assert np.abs(logits.cpu().numpy() - lo).max() <= 2e-4 * max(1e-3, float(np.abs(lo).max()))
     assert lw.ml.poll_error() == 0
     lw.close()
 
