@@ -201,9 +201,16 @@ class Step:
             self.Yd.append(w.base_output(lw.layers[0], m, self.T_d, 1, device))
         self.n_launches = 0
         self.mods = list(range(7))
+        self.decode_grouped = False
+
+    def group_decode(self):
+        """The decode requests were routed when their prompts were served (Section 3.3: once, before the first new
+        token), so their group block is built once and stays valid from step to step."""
+        self.lw.ml.group(0, 1, self.cu_d, self.slots_d, len(self.decode_ids), self.T_d, self.ws_d)
+        self.decode_grouped = True
 
     def run(self, ev=None):
-        """One pass of the path.  ev: optional list of 6 CUDA events recorded at the phase boundaries."""
+        """One pass of the path.  ev: optional list of 5 CUDA events recorded at the phase boundaries."""
         ml = self.lw.ml
         rec = (lambda i: ev[i].record()) if ev is not None else (lambda i: None)
         rec(0)
@@ -213,12 +220,12 @@ class Step:
         rec(2)
         ml.apply_prefill_multi(0, self.mods, self.Xp, self.Yp, self.g_p)     # all 7 call sites, one call
         rec(3)
-        ml.group(0, 1, self.cu_d, self.slots_d, len(self.decode_ids), self.T_d, self.ws_d)
-        rec(4)
+        if not self.decode_grouped:
+            self.group_decode()
         ml.apply_decode_multi(0, self.mods, self.Xd, self.Yd, self.g_d)      # all 7 call sites, one call
-        rec(5)
+        rec(4)
         self.decode_launches = 2 if ml.decode_path_for(len(self.decode_ids), self.T_d) == 2 else 1
-        self.n_launches = 2 + 1 + 2 + 1 + self.decode_launches
+        self.n_launches = 2 + 1 + 2 + self.decode_launches
         return self.n_launches
 
 
@@ -226,6 +233,16 @@ def run_ours(args, rank, world, device):
     from paper_2410_18035_b200.workload_runner import LoadedWorkload
     from synth import get_workload
 
+    if args.config in ("c3", "c4", "c5"):
+        if rank != 0:
+            return None
+        try:
+            gpu_id = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+        except Exception:
+            gpu_id = str(device.index or 0)
+        sampler = ClockSampler(gpu_id)
+        sampler.start()
+        return {"c3": run_c3, "c4": run_c4, "c5": run_c5}[args.config](args, device, sampler)
     w = get_workload(args.config, seed=rank)          # weak scaling: every rank serves its own tenants' requests
     w.gen_device = str(device)                        # draw the (multi-GB) inputs with the device generator
     lw = LoadedWorkload(w, device, layers=[0])
@@ -269,15 +286,15 @@ def run_ours(args, rank, world, device):
     # Second pass of the same K steps with an event at every phase boundary: the per-kernel durations behind
     # `roofline`.  (Events between two launches keep the next kernel from starting early, so the whole-step
     # time above is taken without them.)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     for k in range(args.steps):
         step.run(evs[k])
     barrier()
     sampler.region_end()
     clocks = sampler.stop() if rank == 0 else None
-    phase_ms = np.zeros(5)
+    phase_ms = np.zeros(4)
     for k in range(args.steps):
-        for i in range(5):
+        for i in range(4):
             phase_ms[i] += evs[k][i].elapsed_time(evs[k][i + 1])
     phase_ms /= args.steps
     if world > 1:
@@ -296,11 +313,12 @@ def run_ours(args, rank, world, device):
         sweep = run_decode_sweep(device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
+    gpu_check = checked_step_outputs(step, device) if (rank == 0 and not args.skip_cpu) else None
 
     if rank != 0:
         return None
     peaks = load_peaks()
-    route_ms, gp_ms, prefill_ms, gd_ms, decode_ms = (float(v) for v in phase_ms)
+    route_ms, gp_ms, prefill_ms, decode_ms = (float(v) for v in phase_ms)
     shares = {"router": route_ms, "prefill_apply": prefill_ms, "decode_apply": decode_ms}
     dom = max(shares, key=shares.get)
     per_kernel = {
@@ -323,7 +341,16 @@ def run_ours(args, rank, world, device):
         "config": {"workload": w.name, "note": w.note, "tokens_per_step": tokens_per_step, "prompts": len(step.prefill_ids),
                    "decode_tokens": len(step.decode_ids), "rank": w.rank, "tenants": w.n_tenants,
                    "l2": "inputs larger than L2: every step streams > 2 GB between two launches of the same kernel",
-                   "parallelism": f"requests sharded by tenant over {world} GPU(s), no collective"},
+                   "value_is": f"{100.0 * step.T_p / tokens_per_step:.1f} % prompt rows (prefill apply) and "
+                               f"{100.0 * step.T_d / tokens_per_step:.1f} % decode rows; the decode figures stand on their own "
+                               "in decode_tokens_per_s / decode_frac",
+                   "parallelism": f"{world} GPU(s), every rank its own batch of {w.n_requests} requests on its own "
+                                  "tenants (replicas; a request never needs another rank's data), no collective"},
+        # decode on its own: the whole decode step of the model's stack in ONE call (milora_apply_decode_layers,
+        # CUDA-graph replay; breakdown.decode_stack), and the single-layer launch inside the timed step
+        "decode_tokens_per_s": (stack or {}).get("one_call_all_layers", {}).get("decode_tokens_per_s_full_stack"),
+        "decode_frac": (stack or {}).get("one_call_all_layers", {}).get("frac_of_measured_hbm"),
+        "decode_frac_in_step_single_layer_launch": rooflines["decode_apply"]["frac"],
         "breakdown": {
             "decode_tokens_per_s": len(step.decode_ids) / (decode_ms * 1e-3),
             "decode_gbs": rooflines["decode_apply"]["achieved"],
@@ -334,7 +361,8 @@ def run_ours(args, rank, world, device):
             "prefill_frac_of_bf16_peak": work["prefill_flops"] / (prefill_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "router_us_per_prompt": route_ms * 1e3 / len(step.prefill_ids),
             "router_gbs": rooflines["router"]["achieved"],
-            "group_prefill_us": gp_ms * 1e3, "group_decode_us": gd_ms * 1e3,
+            "group_prefill_us": gp_ms * 1e3,
+            "group_decode": "built once when the requests were routed and reused by every step (Section 3.3)",
             "ms_per_step_with_phase_events": float(phase_ms.sum()),
             "fused_projection": fused,
             "decode_stack": stack,
@@ -348,7 +376,225 @@ def run_ours(args, rank, world, device):
         "gpu_launches": launches,
         "clocks": clocks,
     }
-    out["cpu_baseline"] = None if args.skip_cpu else cpu_baseline(w, args)
+    if args.skip_cpu:
+        out["cpu_baseline"] = None
+        out["parity"] = None
+    else:
+        out["cpu_baseline"], out["parity"] = cpu_baseline(w, args, gpu_check)
+    return out
+
+
+def _line(w, args, world, value, ms_per_step, tokens_per_step, roofline, rooflines, breakdown, launches, clocks, extra_cfg):
+    """The JSON line of a configuration other than the default one (same keys)."""
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": dict({"workload": w.name, "note": w.note, "tokens_per_step": tokens_per_step, "rank": w.rank,
+                           "tenants": w.n_tenants, "l2": "inputs larger than L2: a step streams far more than 126 MB",
+                           "parallelism": f"{world} GPU(s), replicas, no collective"}, **extra_cfg),
+           "breakdown": breakdown, "roofline": roofline, "rooflines": rooflines,
+           "e2e": None, "gpu_launches": launches, "clocks": clocks}
+    if args.skip_cpu:
+        out["cpu_baseline"] = None
+    else:
+        n = {"c3": 4, "c4": 16, "c5": 2}.get(args.config, 4)
+        out["cpu_baseline"], _ = cpu_baseline(w, args, None, n_all=n, n_single=max(1, n // 2))
+    return out
+
+
+def _roof(nbytes, ms, peaks, launches):
+    gbs = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+            "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "peak_source": peaks["source"], "ms_per_step": ms,
+            "launches_per_step": launches, "algorithmic_bytes_per_step": nbytes, "traffic": None}
+
+
+def run_c3(args, device, sampler):
+    """Config 3: the LLaMA-2-7B stack, all 32 layers: every layer routes the 32 ragged prompts and applies the
+    segmented LoRA on all their tokens (7 call sites).  A step = 32 x (route, group, prefill apply)."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth import get_workload
+    peaks = load_peaks()
+    w = get_workload("c3")
+    w.gen_device = str(device)
+    lw = LoadedWorkload(w, device)
+    ml, L = lw.ml, w.n_layers
+    ids = [int(i) for i in w.prefill_ids]
+    cu, slots, T = lw.seq_arrays(ids, [])
+    H = [w.hidden_batch(l, ids, device) for l in range(L)]
+    ws = ml.alloc_group_ws(L, len(ids), T)
+    groups = [ml.groups(ws[l], len(ids), T) for l in range(L)]
+    X = [w.module_input(0, m, T, 0, device) for m in range(7)]
+    Y = [w.base_output(0, m, T, 0, device) for m in range(7)]
+    mods = list(range(7))
+
+    def step(ev=None):
+        for l in range(L):
+            if ev is not None:
+                ev[3 * l].record()
+            ml.route(l, H[l], cu, slots)
+            if ev is not None:
+                ev[3 * l + 1].record()
+            ml.group(l, 1, cu, slots, len(ids), T, ws[l:l + 1])
+            ml.apply_prefill_multi(l, mods, X, Y, groups[l])
+            if ev is not None:
+                ev[3 * l + 2].record()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize(device)
+    routes = ml.route_table_read(0, w.n_requests).numpy()
+    steps = min(args.steps, 50)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.region_begin()
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize(device)
+    ms_step = t0.elapsed_time(t1) / steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3 * L)] for _ in range(5)]
+    for e in evs:
+        step(e)
+    torch.cuda.synchronize(device)
+    sampler.region_end()
+    route_ms = float(np.mean([sum(e[3 * l].elapsed_time(e[3 * l + 1]) for l in range(L)) for e in evs]))
+    apply_ms = float(np.mean([sum(e[3 * l + 1].elapsed_time(e[3 * l + 2]) for l in range(L)) for e in evs]))
+    works = [algorithmic_work(w, routes[:, l], ids, []) for l in range(L)]
+    rb, pb, pf = (sum(x[k] for x in works) for k in ("router_bytes", "prefill_bytes", "prefill_flops"))
+    rooflines = {"router": _roof(rb, route_ms, peaks, 2 * L), "prefill_apply": _roof(pb, apply_ms, peaks, 3 * L)}
+    err = ml.poll_error()
+    lw.close()
+    breakdown = {"router_us_per_prompt_all_layers": route_ms * 1e3 / len(ids),
+                 "router_us_per_prompt_per_layer": route_ms * 1e3 / len(ids) / L,
+                 "prefill_tflops": pf / (apply_ms * 1e-3) / 1e12, "prefill_gbs": rooflines["prefill_apply"]["achieved"],
+                 "prefill_frac_of_bf16_peak": pf / (apply_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                 "apply_ms_includes": "the grouping launch of every layer", "device_error_flag": err}
+    args.steps = steps
+    return _line(w, args, 1, T * L / (ms_step * 1e-3), ms_step, T * L, dict(rooflines["prefill_apply"], kernel="prefill_apply"),
+                 rooflines, breakdown, steps * 5 * L, sampler.stop(),
+                 {"layers": L, "prompts": len(ids), "prompt_rows": T,
+                  "step": "32 layers x (route 32 prompts, group, segmented apply on all prompt rows at 7 call sites); "
+                          "the module inputs and base outputs are one set reused by every layer, routers, hidden states "
+                          "and adapters are each layer's own"})
+
+
+def run_c4(args, device, sampler):
+    """Config 4: LLaMA-2-13B shapes, 256 decode requests with Zipf(1.1) tenants, 8 of the 40 layers (each with its own
+    routes and adapters) as one decode step.  value = decode token-layers/s of the one-call path."""
+    peaks = load_peaks()
+    sampler.region_begin()
+    r = run_decode_13b(device, peaks, n_layers=8, rounds=max(3, min(args.steps, 20)))
+    sampler.region_end()
+    one = r["one_call_all_layers"]
+    from synth import get_workload
+    w = get_workload("c4")
+    roof = {"bound": "hbm", "achieved": one["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": one["frac_of_measured_hbm"], "frac_of_8TBs_nominal": one["frac_of_8TBs_nominal"],
+            "peak_source": peaks["source"], "ms_per_step": one["us_per_layer"] * 8e-3, "launches_per_step": 1,
+            "algorithmic_bytes_per_step": r["algorithmic_bytes_per_layer"] * 8, "traffic": None, "kernel": "decode_apply"}
+    reuse = r["decode_rows"] / r["distinct_adapters_per_layer"]
+    return _line(w, args, 1, one["decode_token_layers_per_s"], one["us_per_layer"] * 8e-3, r["decode_rows"] * 8, roof,
+                 {"decode_apply": roof}, {"decode_stack_13b_zipf": r, "reuse_factor_tokens_per_distinct_adapter": reuse},
+                 max(3, min(args.steps, 20)), sampler.stop(),
+                 {"layers": 8, "decode_rows": r["decode_rows"],
+                  "step": "one milora_apply_decode_layers call over 8 layers (CUDA-graph replay); 8 of the 40 layers are "
+                          "registered for the timing, the tests register all 40"})
+
+
+def run_c5(args, device, sampler):
+    """Config 5: LLaMA-3-8B GQA shapes: the mixed step (8 prompts U[256, 4096] + 192 decode rows as one continuous
+    batch of one layer: route the prompts, group, dense-tile apply and gathered apply) and the decode batch sweep."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    from synth import get_workload
+    from synth.workloads import scaled_workload
+    peaks = load_peaks()
+    w = scaled_workload(get_workload("c5"), n_layers=1)
+    w.gen_device = str(device)
+    lw = LoadedWorkload(w, device)
+    ml = lw.ml
+    pre, dec = [int(i) for i in w.prefill_ids], [int(i) for i in w.decode_ids]
+    for i0 in range(0, len(dec), 64):
+        lw.route(0, dec[i0:i0 + 64])                          # the running requests were routed earlier
+    H = w.hidden_batch(0, pre, device)
+    cu_p = torch.from_numpy(w.cu_seqlens(pre)).to(device)
+    slots_p = torch.tensor(pre, dtype=torch.int32, device=device)
+    cu, slots, T = lw.seq_arrays(pre, dec)
+    n_seq = len(pre) + len(dec)
+    ws = ml.alloc_group_ws(1, n_seq, T)
+    g = ml.groups(ws[0], n_seq, T)
+    X = [w.module_input(0, m, T, 0, device) for m in range(7)]
+    Y = [w.base_output(0, m, T, 0, device) for m in range(7)]
+    mods = list(range(7))
+
+    def step(ev=None):
+        rec = (lambda i: ev[i].record()) if ev is not None else (lambda i: None)
+        rec(0)
+        ml.route(0, H, cu_p, slots_p)
+        rec(1)
+        ml.group(0, 1, cu, slots, n_seq, T, ws)
+        ml.apply_prefill_multi(0, mods, X, Y, g)
+        rec(2)
+        ml.apply_decode_multi(0, mods, X, Y, g)
+        rec(3)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize(device)
+    routes = ml.route_table_read(0, w.n_requests).numpy()[:, 0]
+    steps = min(args.steps, 200)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.region_begin()
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize(device)
+    ms_step = t0.elapsed_time(t1) / steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(10)]
+    for e in evs:
+        step(e)
+    torch.cuda.synchronize(device)
+    ph = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(3)]
+    work = algorithmic_work(w, routes, pre, dec)
+    rooflines = {"router": _roof(work["router_bytes"], ph[0], peaks, 2),
+                 "prefill_apply": _roof(work["prefill_bytes"], ph[1], peaks, 3),
+                 "decode_apply": _roof(work["decode_bytes"], ph[2], peaks, 2 if ml.decode_path_for(n_seq, T) == 2 else 1)}
+    err = ml.poll_error()
+    lw.close()
+    sweep = run_decode_sweep(device, peaks)
+    sampler.region_end()
+    breakdown = {"router_us_per_prompt": ph[0] * 1e3 / len(pre), "prefill_tflops": work["prefill_flops"] / (ph[1] * 1e-3) / 1e12,
+                 "decode_rows": len(dec), "decode_distinct_adapters": work["decode_distinct_adapters"],
+                 "decode_batch_sweep": sweep, "device_error_flag": err}
+    args.steps = steps
+    return _line(w, args, 1, T / (ms_step * 1e-3), ms_step, T, dict(rooflines["prefill_apply"], kernel="prefill_apply"),
+                 rooflines, breakdown, steps * 7, sampler.stop(),
+                 {"layers": 1, "prompts": len(pre), "decode_rows": len(dec), "rows": T,
+                  "step": "one layer of the mixed continuous batch: route 8 prompts, one grouping of all 200 sequences, "
+                          "dense-tile apply and gathered apply at 7 call sites; the decode batch sweep (8 layers per "
+                          "batch size, one call per decode step) is in breakdown.decode_batch_sweep"})
+
+
+N_CHECK_PROMPTS = 4
+
+
+def checked_step_outputs(step, device):
+    """One more step on fresh copies of the base outputs (the timed steps update theirs in place over and over):
+    the GPU's routes, and its outputs on the rows of the first N_CHECK_PROMPTS prompts and on every decode row,
+    brought to the host.  They are compared with the oracle inside the CPU-baseline leg."""
+    lw, w, ml = step.lw, step.w, step.lw.ml
+    n_rows = int(sum(int(w.prompt_len[i]) for i in step.prefill_ids[:N_CHECK_PROMPTS]))
+    Yp = [w.base_output(lw.layers[0], m, step.T_p, 0, device) for m in range(7)]
+    Yd = [w.base_output(lw.layers[0], m, step.T_d, 1, device) for m in range(7)]
+    ml.route(0, step.H, step.cu_p, step.slots_p)
+    ml.group(0, 1, step.cu_p, step.slots_p, len(step.prefill_ids), step.T_p, step.ws_p)
+    ml.apply_prefill_multi(0, step.mods, step.Xp, Yp, step.g_p)
+    ml.apply_decode_multi(0, step.mods, step.Xd, Yd, step.g_d)
+    torch.cuda.synchronize(device)
+    out = {"routes": ml.route_table_read(0, w.n_requests).numpy()[:, 0].copy(), "n_rows": n_rows,
+           "Yp": [y[:n_rows].cpu() for y in Yp], "Yd": [y.cpu() for y in Yd], "device_error_flag": ml.poll_error()}
+    del Yp, Yd
     return out
 
 
@@ -430,7 +676,8 @@ def _timed_decode_chain(ml, w, n_layers, cu_d, slots_d, T_d, decode_ids, Xd, Yd,
     def figures(ms):
         gbs = nbytes / n_layers / (ms * 1e-3) / 1e9
         return {"us_per_layer": ms * 1e3, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
-                "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "decode_token_layers_per_s": n / (ms * 1e-3)}
+                "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "decode_token_layers_per_s": n / (ms * 1e-3),
+                "decode_tokens_per_s_full_stack": n / (ms * 1e-3 * n_layers), "layers": n_layers}
 
     # the kernel sets on the same chain (one call per layer), the whole chain as ONE call of
     # milora_apply_decode_layers (every layer its own outputs: the layers of one call run concurrently), then the
@@ -614,9 +861,10 @@ def run_e2e(step, args, world, device, tokens_per_step):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (reported baseline, and the `--impl reference` arm)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(w, n_prompts):
+def oracle_sample_step(w, n_prompts, keep=False):
     """The oracle over a bounded sample of the step: n_prompts prompts routed and applied on all their
-    tokens, and the matching decode tokens.  Returns (token-layers processed, seconds)."""
+    tokens, and the matching decode tokens.  Returns (token-layers processed, seconds) and, with keep, the oracle's
+    route column, top-2 logit gaps and outputs as well."""
     from oracle import reference_run as R
 
     ids = [int(i) for i in w.prefill_ids[:n_prompts]]
@@ -629,12 +877,15 @@ def oracle_sample_step(w, n_prompts):
     Yp = [w.base_output(0, m, T_p, 0) for m in range(7)]
     Xd = [w.module_input(0, m, len(dec), 1) for m in range(7)]
     Yd = [w.base_output(0, m, len(dec), 1) for m in range(7)]
+    kept = {"Yp": [], "Yd": [], "ids": ids, "dec": dec, "token_slot_p": token_slot_p}
     t0 = time.perf_counter()
     table = np.full((w.n_requests, w.n_layers), -1, dtype=np.int32)
-    R.route_requests(w, 0, ids, table, hidden=lambda i: H[i])
+    _, margins = R.route_requests(w, 0, ids, table, hidden=lambda i: H[i])
     R.group_layer(w, token_slot_p, table[:, 0])
     for m in range(7):
-        R.apply_site(w, 0, m, Xp[m], Yp[m], token_slot_p, table[:, 0])
+        y = R.apply_site(w, 0, m, Xp[m], Yp[m], token_slot_p, table[:, 0])
+        if keep:
+            kept["Yp"].append(y)
     if dec:
         # decode requests of the sample need their routes as well (prompt already routed above when shared)
         missing = [i for i in dec if table[i, 0] < 0]
@@ -642,9 +893,25 @@ def oracle_sample_step(w, n_prompts):
             R.route_requests(w, 0, missing, table)
         R.group_layer(w, np.array(dec), table[:, 0])
         for m in range(7):
-            R.apply_site(w, 0, m, Xd[m], Yd[m], np.array(dec), table[:, 0])
+            y = R.apply_site(w, 0, m, Xd[m], Yd[m], np.array(dec), table[:, 0])
+            if keep:
+                kept["Yd"].append(y)
     dt = time.perf_counter() - t0
+    if keep:
+        kept.update(routes=table[:, 0].copy(), margins=dict(zip(ids, margins)), Yp_base=Yp, Yd_base=Yd)
+        return T_p + len(dec), dt, kept
     return T_p + len(dec), dt
+
+
+def _with_threads(n, fn):
+    """fn() with the BLAS / OpenMP pools of numpy limited to n threads; returns (result, threads really used)."""
+    try:
+        from threadpoolctl import threadpool_info, threadpool_limits
+        with threadpool_limits(limits=n):
+            used = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+            return fn(), used
+    except ImportError:
+        return fn(), cpu_threads()
 
 
 def cpu_threads():
@@ -656,17 +923,72 @@ def cpu_threads():
         return 1
 
 
-def cpu_baseline(w, args, n_prompts=64, reps=3):
-    """The oracle, as it stands, over the whole step `reps` times (about 15 s of CPU work)."""
-    tokens, dt = 0, 0.0
-    for _ in range(reps):
-        tk, t = oracle_sample_step(w, n_prompts)
-        tokens += tk
-        dt += t
-    return {"value": tokens / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-            "sample": f"{reps} passes over the first {n_prompts} of {len(w.prefill_ids)} prompts (all their tokens) and the same "
-                      f"{n_prompts} decode requests: {tokens} token-layers in {dt:.2f} s, fp64 numpy",
-            "host_cpus": os.cpu_count()}
+def parity_report(w, gpu, kept):
+    """The GPU's checked step against the oracle's sample (`kept`): route mismatches (excused only where the oracle's
+    top-2 logit gap is below 1e-3: those are counted as near ties), and the max relative error
+    max |y - yref| / max(|yref|, rms(yref)) over the checked rows, on the full output and on the LoRA term alone."""
+    from oracle import milora_oracle as O
+    from oracle import reference_run as R
+    ids = kept["ids"]
+    near, wrong = set(), set()
+    for i in ids:
+        if gpu["routes"][i] != kept["routes"][i]:
+            (near if kept["margins"][i] < 1e-3 else wrong).add(i)
+    differ = np.array(sorted(near | wrong), dtype=np.int64)
+    full = delta = 0.0
+    rows = 0
+    for m in range(7):
+        for yg, yo, yb, slots in ((gpu["Yp"][m], kept["Yp"][m], kept["Yp_base"][m], kept["token_slot_p"]),
+                                  (gpu["Yd"][m][:len(kept["dec"])], kept["Yd"][m], kept["Yd_base"][m], np.array(kept["dec"]))):
+            yg, yb = R.to_f64(yg), R.to_f64(yb)
+            yo = np.asarray(yo)
+            # rows of a request whose GPU route differs from the oracle's (a near tie) legitimately differ: left out
+            ok = ~np.isin(slots, differ)
+            if not ok.any():
+                continue
+            full = max(full, O.max_rel_err(yg[ok], yo[ok]))
+            d_o = yo - yb
+            if np.any(d_o != 0):
+                delta = max(delta, O.max_rel_err((yg - yb)[ok], d_o[ok]))
+            rows += int(ok.sum())
+    tol = 2e-2 if w.dtype == "bf16" else 1e-4
+    return {"prompts_checked": len(ids), "rows_checked_per_module": rows // 7, "route_near_ties": len(near),
+            "route_mismatches": len(wrong), "max_rel_err_full_output": full, "max_rel_err_lora_term": delta,
+            "tolerance": tol, "ok": bool(not wrong and full <= tol),
+            "note": "near tie = GPU and oracle routes differ where the oracle's top-2 logit gap is < 1e-3; the "
+                    "LoRA-term error of a bf16 output includes the rounding of the stored y (|y| 2^-9 against a term "
+                    "of ~0.08), which is why the tests bound it per element instead",
+            "device_error_flag": gpu["device_error_flag"]}
+
+
+def cpu_baseline(w, args, gpu_check=None, n_all=64, n_single=16):
+    """The oracle, as it stands, on the host cores: two passes over the whole step with every core numpy's pools
+    give it, one pass over a quarter of it with one thread; and the parity figures of the GPU's checked step."""
+    cores = os.cpu_count() or 1
+
+    def all_core():
+        tokens, dt = 0, 0.0
+        for _ in range(2):
+            tk, t = oracle_sample_step(w, n_all)
+            tokens += tk
+            dt += t
+        return tokens, dt
+
+    (tok_a, dt_a), used_a = _with_threads(cores, all_core)
+    (tok_1, dt_1), used_1 = _with_threads(1, lambda: oracle_sample_step(w, n_single))
+    parity = None
+    if gpu_check is not None:
+        (_, _, kept), _ = _with_threads(cores, lambda: oracle_sample_step(w, N_CHECK_PROMPTS, keep=True))
+        parity = parity_report(w, gpu_check, kept)
+    base = {"value": tok_a / dt_a, "unit": UNIT, "cores": used_a, "kind": "oracle",
+            "sample": f"2 passes over the first {n_all} of {len(w.prefill_ids)} prompts (all their tokens) and the same "
+                      f"{n_all} decode requests: {tok_a} token-layers in {dt_a:.2f} s, fp64 numpy, thread pools limited "
+                      f"to {used_a} threads",
+            "single_thread": {"value": tok_1 / dt_1, "cores": used_1,
+                              "sample": f"1 pass over the first {n_single} prompts and decode requests: {tok_1} "
+                                        f"token-layers in {dt_1:.2f} s"},
+            "host_cpus": cores}
+    return base, parity
 
 
 def run_reference(args):
@@ -698,7 +1020,9 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2")
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"],
+                    help="c2 (default): the configuration the metric is quoted on; c3, c4, c5: one line each for the "
+                         "32-layer prefill stack, the 13B Zipf decode step and the mixed step with the batch sweep")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-fused", action="store_true", help="leave out the fused-projection timing")
     ap.add_argument("--only-chains", action="store_true",
