@@ -834,8 +834,22 @@ def run_e2e(step, args, world, device, tokens_per_step):
     off = (-ws.data_ptr()) % 256
     ws = ws[off:]
     nb = lambda ts: sum(t.numel() * t.element_size() for t in ts)
-    h2d = nb([Hh, cu_p, slots_p, cu_p, slots_p, cu_d, slots_d]) + nb(Xp.values()) + nb(Yp.values()) + nb(Xd.values()) + nb(Yd.values())
-    d2h = nb(Yp.values()) + nb(Yd.values())
+    # bytes that cross the link per step: H and the index arrays, the route table read back, and, for every sequence,
+    # the X and Y rows of the module it selects up and the Y rows back (milora_step_host sends nothing else)
+    w = step.w
+    routes = ml.route_table_read(0, w.n_requests).numpy()[:, 0]
+    e = w.elem_bytes
+    h2d = nb([Hh, cu_p, slots_p, cu_p, slots_p, cu_d, slots_d])
+    d2h = 2 * routes.size * 4
+    for ids_, one_row in ((step.prefill_ids, False), (step.decode_ids, True)):
+        for i in ids_:
+            m = int(routes[i])
+            if m < 0:
+                continue
+            d1, d2 = w.dims(m)
+            rows = 1 if one_row else int(w.prompt_len[i])
+            h2d += rows * (d1 + d2) * e
+            d2h += rows * d2 * e
     ml.step_host(st_p, ws)
     ml.step_host(st_d, ws)
     torch.cuda.synchronize(device)

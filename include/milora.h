@@ -318,10 +318,13 @@ milora_status milora_linear_prefill(milora_ctx* ctx, int layer, int module, cons
  *             ([cu_prompts_host[n_prompts]][d_model]), slots prompt_slot_host[p]; n_prompts = 0 skips routing;
  *   n_seq sequences of T rows in total (cu_seq_host[n_seq+1], seq_slot_host[n_seq]) form the step;
  *   X_host[m] / Y_host[m] are the [T][d1(m)] inputs and [T][d2(m)] outputs of module m; a NULL pair skips m.
- * The modules are uploaded, applied and copied back one after the other; the copy of one module's output
- * back to the host runs on a stream of the library's own while the next module is uploaded (the link carries
- * both directions at once), and `stream` waits for the last of those copies before the call's work counts as
- * done on it.  The first call creates that stream and its events.
+ * Only the rows the method touches cross the link.  After routing, the call reads the route table back to the
+ * host (the one point where it waits for `stream`), and then, module by module, sends the X and Y rows of the
+ * sequences that select that module (one copy per run of adjacent sequences), applies Eq. 1 and fetches the same
+ * rows of Y.  Rows of sequences that do not select a module are never sent, and their rows of Y_host[m] keep what
+ * they held.  The copy of one module's output back to the host runs on a stream of the library's own while the
+ * next module is uploaded (the link carries both directions at once), and `stream` waits for the last of those
+ * copies before the call's work counts as done on it.  The first call creates that stream and its events.
  * workspace_dev is caller-owned device memory of at least milora_step_host_workspace() bytes,
  * 256-byte aligned; the library allocates no device memory here except what milora_route may grow. */
 typedef struct {

@@ -2,6 +2,8 @@
 #include <algorithm>
 #include <cstring>
 #include <new>
+#include <utility>
+#include <vector>
 
 #include "milora_internal.h"
 
@@ -786,8 +788,11 @@ milora_status milora_step_host(milora_ctx* ctx, const milora_host_step* step, vo
   bool any_site = false;
   for (int m = 0; m < MILORA_NMOD; ++m) any_site = any_site || step->X_host[m];
   if (step->n_seq > 0 && step->T > 0 && any_site) {
-    // The transfers dominate a step from host memory, and the link carries both directions at once: the modules
-    // are processed one after the other, and the copy of module m's output back to the host runs on a second
+    // Only the rows the method touches cross the link: the host reads the route table back (the one point where
+    // the call waits for the stream), and then, module by module, sends the input and base-output rows of the
+    // sequences that select this module and fetches the same rows of the output.  Rows of other sequences are
+    // never sent: the kernels do not touch them on the device, and their place in Y_host keeps what it held.
+    // The link carries both directions at once: the copy of module m's output back to the host runs on a second
     // stream while module m + 1 is being uploaded.
     if (!ctx->copy_ready) {
       MILORA_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
@@ -800,21 +805,54 @@ milora_status milora_step_host(milora_ctx* ctx, const milora_host_step* step, vo
     st = milora_group(ctx, step->layer, 1, reinterpret_cast<const int32_t*>(w + pl.cu_s),
                       reinterpret_cast<const int32_t*>(w + pl.slot_s), step->n_seq, step->T, ws, pl.ws_stride, stream);
     if (st != MILORA_OK) return st;
+    const int K = top_k_of(ctx), NL = ctx->desc.n_layers;
+    try {
+      ctx->h_route_copy.resize((size_t)ctx->desc.max_requests * NL * K);
+    } catch (...) {
+      return MILORA_E_CAPACITY;
+    }
+    MILORA_CUDA(ctx, cudaMemcpyAsync(ctx->h_route_copy.data(), ctx->d_route, ctx->h_route_copy.size() * sizeof(int32_t),
+                                     cudaMemcpyDeviceToHost, s));
+    MILORA_CUDA(ctx, cudaStreamSynchronize(s));
     milora_groups g{ws, step->n_seq, step->T};
+    // row ranges of module m: runs of adjacent sequences that select it
+    std::vector<std::pair<int, int>> runs;
     for (int m = 0; m < MILORA_NMOD; ++m) {
       if (!step->X_host[m]) continue;
       int d1, d2;
       module_dims(ctx->desc, m, &d1, &d2);
-      const size_t y_bytes = (size_t)step->T * d2 * e;
-      MILORA_CUDA(ctx, h2d(pl.X[m], step->X_host[m], (size_t)step->T * d1 * e));
-      MILORA_CUDA(ctx, h2d(pl.Y[m], step->Y_host[m], y_bytes));
+      runs.clear();
+      for (int i = 0; i < step->n_seq; ++i) {
+        const int slot = step->seq_slot_host[i];
+        const int lo = step->cu_seq_host[i], hi = step->cu_seq_host[i + 1];
+        if (slot < 0 || slot >= ctx->desc.max_requests || lo < 0 || hi <= lo || hi > step->T) continue;
+        bool sel = false;
+        for (int j = 0; j < K; ++j) sel = sel || ctx->h_route_copy[((size_t)slot * NL + step->layer) * K + j] == m;
+        if (!sel) continue;
+        if (!runs.empty() && runs.back().second == lo) runs.back().second = hi;
+        else runs.emplace_back(lo, hi);
+      }
+      if (runs.empty()) continue;
+      const char* Xh = static_cast<const char*>(step->X_host[m]);
+      char* Yh = static_cast<char*>(step->Y_host[m]);
+      for (const auto& r : runs) {
+        const size_t rows = (size_t)(r.second - r.first);
+        MILORA_CUDA(ctx, cudaMemcpyAsync(w + pl.X[m] + (size_t)r.first * d1 * e, Xh + (size_t)r.first * d1 * e, rows * d1 * e,
+                                         cudaMemcpyHostToDevice, s));
+        MILORA_CUDA(ctx, cudaMemcpyAsync(w + pl.Y[m] + (size_t)r.first * d2 * e, Yh + (size_t)r.first * d2 * e, rows * d2 * e,
+                                         cudaMemcpyHostToDevice, s));
+      }
       st = milora_apply_prefill(ctx, step->layer, m, w + pl.X[m], w + pl.Y[m], &g, stream);
       if (st != MILORA_OK) return st;
       st = milora_apply_decode(ctx, step->layer, m, w + pl.X[m], w + pl.Y[m], &g, stream);
       if (st != MILORA_OK) return st;
       MILORA_CUDA(ctx, cudaEventRecord(ctx->ev_site[m], s));
       MILORA_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_site[m], 0));
-      MILORA_CUDA(ctx, cudaMemcpyAsync(step->Y_host[m], w + pl.Y[m], y_bytes, cudaMemcpyDeviceToHost, ctx->copy_stream));
+      for (const auto& r : runs) {
+        const size_t rows = (size_t)(r.second - r.first);
+        MILORA_CUDA(ctx, cudaMemcpyAsync(Yh + (size_t)r.first * d2 * e, w + pl.Y[m] + (size_t)r.first * d2 * e, rows * d2 * e,
+                                         cudaMemcpyDeviceToHost, ctx->copy_stream));
+      }
     }
     // the caller's stream is done only when every output has arrived (and the workspace may be reused)
     MILORA_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->copy_stream));

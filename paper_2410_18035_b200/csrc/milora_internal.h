@@ -176,6 +176,7 @@ struct milora_ctx {
   cudaEvent_t ev_site[MILORA_NMOD];             // "module m is done" / "all copies back are done"
   cudaEvent_t ev_done;
   bool copy_ready;
+  std::vector<int32_t> h_route_copy;            // milora_step_host: the route table as the host read it back
   milora::Arena arena;
   std::string cuda_error;
 };

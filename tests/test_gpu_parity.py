@@ -673,11 +673,15 @@ def test_step_from_host_buffers_matches_oracle():
     Ybs = {m: w.base_output(0, m, T, 3) for m in range(7)}
     Ys = {m: pin(Ybs[m].clone()) for m in range(7)}
     step = ml.make_host_step(0, cu_p, slot_p, H, pin(cu), pin(slots), T, Xs, Ys)
-    ws = torch.empty(ml.step_host_workspace(step) + 256, dtype=torch.uint8, device="cuda")
+    # the workspace starts as NaN patterns: only the rows of routed sequences are sent to the device, and only those
+    # rows may come back, so no other row of Y_host can pick up what the workspace held
+    ws = torch.full((ml.step_host_workspace(step) + 256,), 255, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 256:]
     ml.step_host(step, ws)
     torch.cuda.synchronize()
     assert ml.poll_error() == 0
+    for m in range(7):
+        assert not bool(torch.isnan(Ys[m].float()).any()), f"module {m}: an unsent row came back from the workspace"
     table = ml.route_table_read(0, w.n_requests).numpy()
     tmp = np.full((w.n_requests, 1), -1, dtype=np.int32)
     _, margins = R.route_requests(w, 0, prefill, tmp)
