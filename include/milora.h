@@ -119,8 +119,15 @@ milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, con
                                      const float* coef_host, int n_a, int n_b, void* stream);
 
 /* Drop every adapter and router of a tenant (host-side table update; takes effect for calls
- * made afterwards).  Fails with MILORA_E_STATE while a request slot is bound to the tenant. */
+ * made afterwards).  Fails with MILORA_E_STATE while a request slot is bound to the tenant.  The tenant's copies
+ * go back to the library's pool, from which later registrations are served first, so a server that admits and drops
+ * tenants does not grow; the caller must make sure that no call that could still read them (an apply on a group
+ * block built while the tenant was registered) is running or will be made. */
 milora_status milora_unregister_tenant(milora_ctx* ctx, int tenant);
+/* Bytes of the library's pool that registered adapters and routers occupy right now (copies in the library's
+ * layouts: A^T and B row-major, plus, in bf16 contexts whose dimensions allow it, the two operand images: twice
+ * the adapter's own size). */
+milora_status milora_resident_bytes(const milora_ctx* ctx, size_t* adapter_pool_bytes);
 
 /* ---- request slots -----------------------------------------------------------------------
  * Bind a slot to a tenant when a request is admitted; release it when the request ends.
@@ -200,7 +207,14 @@ milora_status milora_gate_table_write(milora_ctx* ctx, int slot_begin, int n_slo
  *   seg_offset[]   bucket boundaries in perm
  *   perm[]         active token rows ordered by (module, tenant, row)
  * followed by the work lists the apply kernels consume (dense tiles of consecutive rows for
- * long sequences; gathered rows for short ones). */
+ * long sequences; gathered rows for short ones).
+ *
+ * A block depends on the batch (which slots, which row ranges), on the routes of its slots and on the adapters of
+ * their tenants, and on nothing else.  Routes are written once per request (Section 3.3), so the block of a decode
+ * batch stays valid from step to step: build it when the batch changes (a request joins or leaves, a slot is
+ * reopened, one of its tenants registers an adapter again or is dropped) and reuse it for every step in between.
+ * The grouping launch costs about as much as the decode apply of one layer; calling it every step doubles the
+ * cost of a decode step for nothing. */
 typedef struct {
   size_t header, mod_offset, mod_tile_offset, mod_gather_offset;
   size_t seg_key, seg_offset, perm, tiles, gather_rows, gather;

@@ -67,6 +67,7 @@ SIGNATURES = {
     "milora_register_adapter": (_I, [_VP, _I, _I, _I, _I, _F, _VP, _VP, _VP]),
     "milora_register_router": (_I, [_VP, _I, _I, _VP, _VP, _I, _VP, _I, C.POINTER(_F), _I, _I, _VP]),
     "milora_unregister_tenant": (_I, [_VP, _I]),
+    "milora_resident_bytes": (_I, [_VP, C.POINTER(C.c_size_t)]),
     "milora_request_open": (_I, [_VP, _I, _I]),
     "milora_request_close": (_I, [_VP, _I]),
     "milora_route": (_I, [_VP, _I, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP]),
@@ -199,6 +200,11 @@ class Milora:
 
     def unregister_tenant(self, tenant):
         self._check(self.lib.milora_unregister_tenant(self.h, tenant), "milora_unregister_tenant")
+
+    def resident_bytes(self) -> int:
+        out = C.c_size_t(0)
+        self._check(self.lib.milora_resident_bytes(self.h, C.byref(out)), "milora_resident_bytes")
+        return out.value
 
     def request_open(self, slot, tenant):
         self._check(self.lib.milora_request_open(self.h, slot, tenant), "milora_request_open")

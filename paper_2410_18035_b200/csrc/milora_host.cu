@@ -20,6 +20,20 @@ milora_status cuda_fail(milora_ctx* ctx, cudaError_t e, const char* where) {
 void* Arena::alloc(size_t bytes, cudaError_t* err) {
   *err = cudaSuccess;
   bytes = (bytes + 255) & ~size_t(255);
+  // first fit among the blocks that were given back; what is left of a larger block stays on the list
+  for (size_t i = 0; i < free_blocks.size(); ++i) {
+    if (free_blocks[i].size >= bytes) {
+      char* p = free_blocks[i].base;
+      if (free_blocks[i].size == bytes) {
+        free_blocks[i] = free_blocks.back();
+        free_blocks.pop_back();
+      } else {
+        free_blocks[i].base += bytes;
+        free_blocks[i].size -= bytes;
+      }
+      return p;
+    }
+  }
   for (auto& c : chunks) {
     if (c.size - c.used >= bytes) {
       void* p = c.base + c.used;
@@ -35,9 +49,27 @@ void* Arena::alloc(size_t bytes, cudaError_t* err) {
   return base;
 }
 
+void Arena::give_back(void* p, size_t bytes) {
+  bytes = (bytes + 255) & ~size_t(255);
+  if (!p || bytes == 0) return;
+  try {
+    free_blocks.push_back({static_cast<char*>(p), bytes});
+  } catch (...) {
+    // the list could not grow: the block stays unused until the context is destroyed
+  }
+}
+
+size_t Arena::bytes_in_use() const {
+  size_t n = 0;
+  for (const auto& c : chunks) n += c.used;
+  for (const auto& b : free_blocks) n -= b.size;
+  return n;
+}
+
 void Arena::release() {
   for (auto& c : chunks) cudaFree(c.base);
   chunks.clear();
+  free_blocks.clear();
 }
 
 void module_dims(const milora_model_desc& d, int module, int* d1, int* d2) {
@@ -281,6 +313,9 @@ milora_status milora_register_adapter(milora_ctx* ctx, int tenant, int layer, in
   void* store = const_cast<void*>(ent.At);
   if (!store || ctx->adapter_bytes[idx] != total) {
     cudaError_t e;
+    if (store) ctx->arena.give_back(store, ctx->adapter_bytes[idx]);      // another rank than before: the old block is free
+    ent.At = nullptr;
+    ctx->adapter_bytes[idx] = 0;
     store = ctx->arena.alloc(total, &e);
     if (!store) return cuda_fail(ctx, e, "adapter pool cudaMalloc");
     ctx->adapter_bytes[idx] = total;
@@ -328,6 +363,9 @@ milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, con
   void* store = const_cast<void*>(ent.W);
   if (!store || ctx->router_bytes[idx] != bytes_w + bytes_sa) {
     cudaError_t e;
+    if (store) ctx->arena.give_back(store, ctx->router_bytes[idx]);
+    ent.W = nullptr;
+    ctx->router_bytes[idx] = 0;
     store = ctx->arena.alloc(bytes_w + bytes_sa, &e);
     if (!store) return cuda_fail(ctx, e, "router pool cudaMalloc");
     ctx->router_bytes[idx] = bytes_w + bytes_sa;
@@ -362,13 +400,27 @@ milora_status milora_unregister_tenant(milora_ctx* ctx, int tenant) {
   for (int l = 0; l < L; ++l) {
     for (int m = 0; m < MILORA_NMOD; ++m) {
       size_t idx = adapter_index(tenant, l, m, L);
-      ctx->h_adapters[idx].rank = 0;  // storage pointer is kept for reuse by a later registration
+      // the copies go back to the pool (the caller has made sure nothing that reads them is still running)
+      AdapterEntry& ent = ctx->h_adapters[idx];
+      ctx->arena.give_back(const_cast<void*>(ent.At), ctx->adapter_bytes[idx]);
+      ctx->adapter_bytes[idx] = 0;
+      std::memset(&ent, 0, sizeof(ent));
       mark(ctx->adapters_dirty_lo, ctx->adapters_dirty_hi, idx);
     }
     size_t r = (size_t)tenant * L + l;
-    ctx->h_routers[r].pool = -1;  // marks "not registered" while keeping the storage pointer
+    RouterEntry& rt = ctx->h_routers[r];
+    ctx->arena.give_back(const_cast<void*>(rt.W), ctx->router_bytes[r]);
+    ctx->router_bytes[r] = 0;
+    std::memset(&rt, 0, sizeof(rt));
+    rt.pool = -1;
     mark(ctx->routers_dirty_lo, ctx->routers_dirty_hi, r);
   }
+  return MILORA_OK;
+}
+
+milora_status milora_resident_bytes(const milora_ctx* ctx, size_t* adapter_pool_bytes) {
+  if (!ctx || !adapter_pool_bytes) return MILORA_E_ARG;
+  *adapter_pool_bytes = ctx->arena.bytes_in_use();
   return MILORA_OK;
 }
 

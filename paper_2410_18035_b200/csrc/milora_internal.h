@@ -120,10 +120,17 @@ struct StreamLayer {
 };
 static_assert(sizeof(StreamLayer) == 144, "StreamLayer is copied as 9 x 16 bytes");
 
+// Pool behind the adapter and router copies: 64 MB (or larger) cudaMalloc chunks carved front to back, plus a list
+// of blocks that were given back (a tenant that left, an adapter registered again at another rank), which
+// allocations look through first.  Blocks are not merged; a server that churns tenants of a few sizes reuses them.
 struct Arena {
   struct Chunk { char* base; size_t size, used; };
+  struct Block { char* base; size_t size; };
   std::vector<Chunk> chunks;
+  std::vector<Block> free_blocks;
   void* alloc(size_t bytes, cudaError_t* err);
+  void give_back(void* p, size_t bytes);
+  size_t bytes_in_use() const;      // carved bytes minus bytes on the free list
   void release();
 };
 

@@ -404,6 +404,41 @@ def test_tenant_without_adapter_is_excluded():
     lw.close()
 
 
+def test_tenant_churn_reuses_the_pool():
+    """A server that drops tenants and admits others (at other ranks too) must not grow: the copies of a dropped
+    tenant go back to the pool and later registrations are served from there; after the churn a tenant's adapters
+    still give the oracle's result."""
+    base = get_workload("c1")
+    w = scaled_workload(base, name="churn", dtype="bf16", d_model=256, d_ff=768, d_kv=256, rank=16, n_tenants=4,
+                        request_tenant=np.array([0, 1, 2, 3], dtype=np.int32), has_base_weights=False, n_layers=1)
+    lw = _loaded(w)
+    ml = lw.ml
+    full = ml.resident_bytes()
+    assert full > 0
+    for i in range(4):
+        ml.request_close(i)
+    seen = []
+    for rnd in range(6):
+        for tenant in range(4):
+            ml.unregister_tenant(tenant)
+        assert ml.resident_bytes() == 0
+        rank = (16, 8, 16, 4, 12, 16)[rnd]
+        for tenant in range(4):
+            lw.register_router(tenant, 0, 0)
+            for m in range(7):
+                A, B = w.adapter(tenant, 0, m, "cuda")
+                ml.register_adapter(tenant, 0, m, A[:, :rank].contiguous(), B[:rank].contiguous(), w.scale)
+        seen.append(ml.resident_bytes())
+    assert seen[-1] == full and max(seen) <= full, f"pool use after churn {seen} against {full} at the start"
+    torch.cuda.synchronize()
+    for i in range(4):
+        ml.request_open(i, i)
+    ids = [0, 1, 2, 3]
+    table_g, table_o, _ = _route_all_layers(lw, ids)
+    _step_parity(lw, 0, ids, [], table_g, tag=31)
+    lw.close()
+
+
 def test_group_edge_cases_and_device_flags():
     w = get_workload("c1")
     lw = _loaded(w)

@@ -77,3 +77,63 @@ def test_shard_by_tenant_structure():
         for a in range(world):
             for b in range(a + 1, world):
                 assert not (tenants[a] & tenants[b])
+
+
+def _c4_routes(w, layer):
+    """A seeded stand-in for layer `layer`'s route column of config 4 (grouping depends on routes and tenants only;
+    routing 256 prompts of 256 x 5120 with the oracle is not needed to test the sharding)."""
+    return np.random.default_rng(1000 + layer).integers(0, 7, size=w.n_requests).astype(np.int32)
+
+
+def _rank_group_c4(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import milora_oracle as O
+    from synth import get_workload
+    from synth.workloads import shard_by_tenant
+
+    w = get_workload("c4")
+    mine = shard_by_tenant(w.request_tenant, world)[rank]
+    out = {}
+    for layer in (0, 17, 39):
+        routes = _c4_routes(w, layer)
+        # this rank's decode step: one row per request of its shard, in request order
+        g = O.group_tokens(mine, w.request_tenant, routes, lambda t, m: True, w.n_tenants)
+        out[f"perm{layer}"] = mine[g["perm"]]                 # as request ids, comparable across ranks
+        out[f"key{layer}"] = g["seg_key"]
+        out[f"off{layer}"] = g["seg_offset"]
+    dist.barrier()
+    np.savez(os.path.join(out_dir, f"rank{rank}.npz"), **out)
+    dist.destroy_process_group()
+
+
+def test_one_c4_batch_sharded_by_tenant_groups_like_one_process(tmp_path):
+    """One decode batch of config 4 (256 requests, Zipf tenants) split over two ranks by tenant: every (module, tenant)
+    bucket of the single-process grouping lands on exactly one rank, whole and in the same row order, for layers at
+    both ends and in the middle of the stack; no rank sees a request of the other."""
+    from oracle import milora_oracle as O
+    from synth import get_workload
+    from synth.workloads import shard_by_tenant
+
+    world = 2
+    mp.spawn(_rank_group_c4, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    w = get_workload("c4")
+    shards = shard_by_tenant(w.request_tenant, world)
+    ranks = [np.load(tmp_path / f"rank{r}.npz") for r in range(world)]
+    everyone = np.arange(w.n_requests)
+    for layer in (0, 17, 39):
+        routes = _c4_routes(w, layer)
+        g = O.group_tokens(everyone, w.request_tenant, routes, lambda t, m: True, w.n_tenants)
+        full = {int(k): g["perm"][g["seg_offset"][s]:g["seg_offset"][s + 1]].tolist() for s, k in enumerate(g["seg_key"])}
+        seen = {}
+        for r in range(world):
+            keys, off, perm = ranks[r][f"key{layer}"], ranks[r][f"off{layer}"], ranks[r][f"perm{layer}"]
+            assert set(perm.tolist()) == set(shards[r].tolist())
+            assert np.all(np.diff(keys) > 0)                                   # canonical order: module, then tenant
+            for s, k in enumerate(keys):
+                assert int(k) not in seen, "a bucket is split over two ranks"
+                seen[int(k)] = perm[off[s]:off[s + 1]].tolist()
+                assert (int(k) % w.n_tenants) % world == r                     # the tenant's home rank
+        assert seen == full
