@@ -49,10 +49,10 @@ KERNEL_SOURCES = {
 
 
 def recorded_traffic(workload_name):
-    """DRAM bytes per step per kernel from the committed ncu capture (profiles/traffic_c2.txt); a kernel whose
-    sources no longer hash to the recorded value gets None (its counters are out of date)."""
+    """DRAM bytes per step per kernel from the committed ncu capture (profiles/traffic_c2.txt, taken on the full-size
+    step); a kernel whose sources no longer hash to the recorded value gets None (its counters are out of date)."""
     import hashlib
-    if not workload_name.startswith("c2"):
+    if not workload_name.startswith("c2") or "_first" in workload_name:
         return {}
     path = os.path.join(ROOT, "profiles", "traffic_c2.txt")
     out = {}
@@ -180,7 +180,8 @@ def algorithmic_work(w, routes_col, prefill_ids, decode_ids):
 class Step:
     """Device-resident inputs of one step and the sequence of library calls that make it."""
 
-    def __init__(self, lw, device):
+    def __init__(self, lw, device, light=False):
+        """light: without the prompt rows' module inputs and outputs (7 GB at config 2); enough for the decode chains."""
         w = lw.w
         self.lw, self.w, self.device = lw, w, device
         self.prefill_ids = [int(i) for i in w.prefill_ids]
@@ -195,8 +196,9 @@ class Step:
         self.g_d = ml.groups(self.ws_d[0], len(self.decode_ids), self.T_d)
         self.Xp, self.Yp, self.Xd, self.Yd = [], [], [], []
         for m in range(7):
-            self.Xp.append(w.module_input(lw.layers[0], m, self.T_p, 0, device))
-            self.Yp.append(w.base_output(lw.layers[0], m, self.T_p, 0, device))
+            if not light:
+                self.Xp.append(w.module_input(lw.layers[0], m, self.T_p, 0, device))
+                self.Yp.append(w.base_output(lw.layers[0], m, self.T_p, 0, device))
             self.Xd.append(w.module_input(lw.layers[0], m, self.T_d, 1, device))
             self.Yd.append(w.base_output(lw.layers[0], m, self.T_d, 1, device))
         self.n_launches = 0
@@ -245,7 +247,20 @@ def run_ours(args, rank, world, device):
         return {"c3": run_c3, "c4": run_c4, "c5": run_c5}[args.config](args, device, sampler)
     w = get_workload(args.config, seed=rank)          # weak scaling: every rank serves its own tenants' requests
     w.gen_device = str(device)                        # draw the (multi-GB) inputs with the device generator
+    if args.prompts is not None and args.prompts < len(w.prefill_ids):
+        # profiler captures: the same step on the first few requests only (a quarter of the bytes at 16 prompts)
+        from synth.workloads import scaled_workload
+        w = scaled_workload(w, prefill_ids=w.prefill_ids[:args.prompts], decode_ids=w.decode_ids[:args.prompts],
+                            name=w.name + f"_first{args.prompts}")
     lw = LoadedWorkload(w, device, layers=[0])
+    if args.only_decode_stack:
+        # a small process for profiler captures: the decode chain of the 7B stack alone, a few GB on the device
+        if rank == 0:
+            step = Step(lw, device, light=True)
+            lw.ml.route(0, step.H, step.cu_p, step.slots_p)
+            print(json.dumps({"decode_stack": run_decode_stack(step, device, load_peaks(), n_layers=args.chain_layers,
+                                                               rounds=3)}))
+        return None
     step = Step(lw, device)
     tokens_per_step = step.T_p + step.T_d
 
@@ -1042,6 +1057,11 @@ def main():
     ap.add_argument("--only-chains", action="store_true",
                     help="print only the decode-chain figures (both decode kernel sets) and exit; not a bench line")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle timing")
+    ap.add_argument("--only-decode-stack", action="store_true",
+                    help="profiling runs: only the decode chain of the 7B stack (--chain-layers layers), a few GB on the device")
+    ap.add_argument("--chain-layers", type=int, default=8)
+    ap.add_argument("--prompts", type=int, default=None,
+                    help="profiling runs: only the first N prompts and decode requests of the step (not a bench line)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

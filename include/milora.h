@@ -317,6 +317,11 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
  * Wt_dev is W_m transposed, [d2][d1] row-major (the layout in which an nn.Linear keeps its weight);
  * bias_dev is d2 values or NULL; all in bf16.  Rows of short sequences (the gathered list: decode tokens)
  * receive only the base projection here; follow with milora_apply_decode for their LoRA term.
+ * When to use it: measured on a B200 at the LLaMA-2-7B sizes (32,768 rows), this call takes 0.09-0.11 ms (q site) to
+ * 0.21 ms (down site) longer than a library GEMM of the base projection alone, while the separate
+ * milora_apply_prefill for all seven call sites of the layer costs 0.22 ms in total; a caller whose own GEMM is as
+ * fast as the library's should therefore keep it and call milora_apply_prefill afterwards.  The fused call pays
+ * where the caller has no GEMM of that quality, or where Y must not be written twice.
  * Three launches (shrink, piece packing, persistent GEMM).  Returns MILORA_E_SHAPE unless the context is
  * bf16, max_rank <= 32, d1 is a multiple of 64, d2 a multiple of 256 and T >= 128; such callers use their own
  * GEMM followed by milora_apply_prefill.  Grows an internal scratch buffer like milora_route does. */

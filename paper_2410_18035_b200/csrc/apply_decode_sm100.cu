@@ -360,7 +360,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 4) decode
     }
     // all kC x n x r partial sums have landed here; the peers wait for theirs likewise, so nobody is written after it left
     if (!mbar_wait(xbar, xparity)) {
+      // A peer's partial sums never came.  This CTA's shared memory is still the target of the stores that are
+      // missing, and of its own bulk copies: it stays for a second, equally bounded, wait on both before it leaves,
+      // so that whatever is merely late has landed; a peer that is gone for good has raised the flag itself.
       if (tid == 0) atomicOr(a.err, ERR_WAIT_TIMEOUT);
+      mbar_wait(xbar, xparity);
       if (STAGE_B) mbar_wait(bar, bparity);
       return;
     }

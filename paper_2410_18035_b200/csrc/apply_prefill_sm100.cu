@@ -84,6 +84,19 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
   return false;
 }
 
+// After a wait has run out (`abort` is set) copies that were started may still be on their way into this CTA's
+// shared memory.  The thread that started them gives every ring stage one more, equally bounded, wait for the last
+// phase it asked for, so that whatever is merely late has landed before the CTA frees its tensor memory and leaves.
+// `issued` copies went to stages 0, 1, ... in turn; full(s) is the barrier of stage s.
+template <class FullOf>
+__device__ __forceinline__ void drain_ring(volatile int* abort, int issued, int stages, FullOf full) {
+  if (!*abort) return;
+  for (int s = 0; s < stages && s < issued; ++s) {
+    const int last = ((issued - 1 - s) / stages) * stages + s;      // last copy that went to stage s
+    mbar_wait(full(s), (uint32_t)(last / stages) & 1u);
+  }
+}
+
 __device__ __forceinline__ uint32_t tmem_cols_for(int rp) { return rp <= 32 ? 32u : 64u; }
 
 // ------------------------------------------------------------------------------------------------------
@@ -142,6 +155,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
   tc_fence_after();
   const uint32_t tmem_base = *slot_ptr;
 
+  int issued = 0;       // copies started by this thread (the copy thread only)
   if (nk > 0) {
     if (warp == 0 && lane == 0) {
       // ---- copies: X tile by TMA, A image chunk by one bulk copy ----
@@ -152,6 +166,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
         mbar_expect_tx(full(s), kXStage + rp * 128);
         tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
         bulk_g2s(as + s * a_stage, img + (size_t)(kc0 + i) * rp * 128, rp * 128, full(s));
+        issued = i + 1;
       }
     } else if (warp == 1 && lane == 0) {
       // ---- MMAs: D[128 x rp] += X[128 x 16] * A[16 x rp], four per stage ----
@@ -198,6 +213,7 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
         *reinterpret_cast<uint4*>(dst + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
     }
   }
+  if (warp == 0 && lane == 0) drain_ring(abort_ptr, issued, kShrinkStages, full);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, ncols);
@@ -267,6 +283,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
   }
   __syncthreads();
   const int row0 = job.start;
+  int issued = 0;                       // copies started by this thread (the copy thread only)
   auto issue_stage = [&](int i) {       // y tile (two 64-column boxes) and B image chunk of n chunk i
     const int s = i % kExpandStages;
     mbar_expect_tx(full(s), kYStage + rp * 256);
@@ -280,6 +297,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
     // first pass over the ring: these copies do not depend on the shrink kernel
     if (lane == 0)
       for (int i = 0; i < nn && i < kExpandStages; ++i) issue_stage(i);
+      issued = min(nn, kExpandStages);
   }
 
   // epilogue threads also build the A operand: V = s * sum_k V_k, bf16, 8 x 16-byte core-matrix rows
@@ -331,6 +349,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
         const int s = i % kExpandStages, ph = (i / kExpandStages) & 1;
         if (!wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
         issue_stage(i);
+        issued = i + 1;
       }
     }
   } else if (warp == 1) {
@@ -416,6 +435,7 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
   }
   __syncwarp();
   pdl_wait();                           // returns at once here; keeps "every thread waited before it exits" true
+  if (warp == 0 && lane == 0) drain_ring(abort_ptr, issued, kExpandStages, full);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kCols);
@@ -571,6 +591,7 @@ __global__ void __launch_bounds__(kLinThreads, 1) linear_lora_kernel(const __gri
   };
   const TileJob* tiles = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles);
   const bool bad = (base & 1023) != 0 || a.rpad > kLinRPadMax;
+  int ring_issued = 0, piece_issued = 0;        // copies started by this thread (the copy thread only)
   if (bad && tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
 
   if (!bad && warp == 0) {
@@ -588,6 +609,7 @@ __global__ void __launch_bounds__(kLinThreads, 1) linear_lora_kernel(const __gri
           mbar_expect_tx(full(s), kLinAStage + kLinBStage);
           tma_load_2d(as + s * kLinAStage, &a.xmap, k * kLinBK, mb * kLinBM, full(s));
           tma_load_2d(bs + s * kLinBStage, &a.wmap, k * kLinBK, nb * kLinBN, full(s));
+          ring_issued = it + 1;
         }
         const int np = min(a.piece_cnt[mb], kMaxPieces);
         for (int p = 0; p < np && ok; ++p, ++lit) {
@@ -599,6 +621,7 @@ __global__ void __launch_bounds__(kLinThreads, 1) linear_lora_kernel(const __gri
           mbar_expect_tx(lfull, rp * 256u + rp * 512u);
           bulk_g2s(vs, a.vimg + (size_t)pj * ((size_t)kTileRows * a.rpad * 2), rp * 256u, lfull);
           bulk_g2s(lbs, static_cast<const char*>(job.B_img) + (size_t)(2 * nb) * rp * 256u, rp * 512u, lfull);
+          piece_issued = lit + 1;
         }
       }
     }
@@ -694,6 +717,10 @@ __global__ void __launch_bounds__(kLinThreads, 1) linear_lora_kernel(const __gri
     }
   }
   __syncwarp();
+  if (warp == 0 && lane == 0) {
+    drain_ring(abort_ptr, ring_issued, kLinStages, full);
+    drain_ring(abort_ptr, piece_issued, 1, [&](int) { return lfull; });
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kCols);
