@@ -27,6 +27,11 @@
  *   - Matrices are dense row-major.  Element type of activations, adapters and router
  *     weights is the context's dtype (fp32 or bf16); accumulation is always fp32.
  *   - A context is not thread-safe; use one per host thread or lock around it.
+ *   - The compute calls of one context share scratch buffers that the library owns and grows on demand (router
+ *     partial sums, prefill partial products, the fused projection's piece images, the decode kernels' counters
+ *     and partial sums): order all compute calls of a context on ONE stream.  Two calls on different streams would
+ *     race on the scratch, and a growth (cudaFree / cudaMalloc after synchronising the call's own stream) could
+ *     free a buffer that a kernel on the other stream still reads.
  *   - Device-side index problems (a slot id out of range inside a device array) never
  *     fault: the offending item is skipped and a flag is raised that milora_poll_error reads.
  */
