@@ -320,6 +320,7 @@ def run_ours(args, rank, world, device):
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
     fused = stack = stack13 = mixed = sweep = None
+    router_alone = run_router_alone(step, device, work["router_bytes"], load_peaks()) if rank == 0 else None
     if rank == 0 and not args.skip_fused and w.dtype == "bf16":
         mixed = run_mixed_step(step, device)
         fused = run_fused_projection(step, routes, device, load_peaks())
@@ -376,6 +377,7 @@ def run_ours(args, rank, world, device):
             "prefill_frac_of_bf16_peak": work["prefill_flops"] / (prefill_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "router_us_per_prompt": route_ms * 1e3 / len(step.prefill_ids),
             "router_gbs": rooflines["router"]["achieved"],
+            "router_back_to_back": router_alone,
             "group_prefill_us": gp_ms * 1e3,
             "group_decode": "built once when the requests were routed and reused by every step (Section 3.3)",
             "ms_per_step_with_phase_events": float(phase_ms.sum()),
@@ -589,6 +591,33 @@ def run_c5(args, device, sampler):
                   "step": "one layer of the mixed continuous batch: route 8 prompts, one grouping of all 200 sequences, "
                           "dense-tile apply and gathered apply at 7 call sites; the decode batch sweep (8 layers per "
                           "batch size, one call per decode step) is in breakdown.decode_batch_sweep"})
+
+
+def run_router_alone(step, device, nbytes, peaks, iters=40):
+    """milora_route called back to back on two copies of H (2 x 268 MB, so no call finds its input in L2), one event
+    pair around all calls: the router's cost per call without the event pair and the neighbours it has inside the
+    step (there an event on either side keeps it from overlapping the kernels around it)."""
+    ml = step.lw.ml
+    H2 = step.H.clone()
+
+    def pair():
+        ml.route(0, step.H, step.cu_p, step.slots_p)
+        ml.route(0, H2, step.cu_p, step.slots_p)
+
+    for _ in range(3):
+        pair()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        pair()
+    e1.record()
+    torch.cuda.synchronize(device)
+    ms = e0.elapsed_time(e1) / (2 * iters)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    del H2
+    return {"ms_per_call": ms, "us_per_prompt": ms * 1e3 / len(step.prefill_ids), "gbs": gbs,
+            "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "calls": 2 * iters}
 
 
 N_CHECK_PROMPTS = 4

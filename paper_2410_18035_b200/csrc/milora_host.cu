@@ -205,6 +205,7 @@ milora_status milora_create(const milora_model_desc* desc, milora_ctx** out) {
   ctx->d_lin = nullptr; ctx->lin_bytes = 0;
   ctx->d_dsplit = nullptr; ctx->dsplit_floats = 0; ctx->dsplit_dirty = true;
   ctx->dsplit_occ_s = 0; ctx->dsplit_occ_e = 0; ctx->decode_path = MILORA_DECODE_AUTO;
+  ctx->n_routers_whole_row = 0; ctx->route_bulk_attr_set = false;
   ctx->copy_stream = nullptr; ctx->ev_done = nullptr; ctx->copy_ready = false;
   ctx->d_stream = nullptr; ctx->stream_jobs_cap = 0; ctx->stream_frag_bytes = 0; ctx->stream_part_bytes = 0;
   ctx->stream_dirty = true; ctx->stream_attr_set = false; ctx->stream_epoch = 0; ctx->stream_unit_stages = 0;
@@ -360,6 +361,10 @@ milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, con
   size_t bytes_w = ((size_t)MILORA_NMOD * d * ctx->elem + 255) & ~size_t(255);
   size_t bytes_sa = ((size_t)d * ctx->elem + 255) & ~size_t(255);
   RouterEntry& ent = ctx->h_routers[idx];
+  auto whole_row = [](const RouterEntry& r) {
+    return r.W != nullptr && (r.pool == MILORA_POOL_LAST || r.pool == MILORA_POOL_SELFATTN);
+  };
+  if (whole_row(ent)) --ctx->n_routers_whole_row;        // replaced below
   void* store = const_cast<void*>(ent.W);
   if (!store || ctx->router_bytes[idx] != bytes_w + bytes_sa) {
     cudaError_t e;
@@ -388,6 +393,7 @@ milora_status milora_register_router(milora_ctx* ctx, int tenant, int layer, con
   ent.act = act;
   ent.n_a = n_a;
   ent.n_b = n_b;
+  if (whole_row(ent)) ++ctx->n_routers_whole_row;
   mark(ctx->routers_dirty_lo, ctx->routers_dirty_hi, idx);
   return MILORA_OK;
 }
@@ -409,6 +415,7 @@ milora_status milora_unregister_tenant(milora_ctx* ctx, int tenant) {
     }
     size_t r = (size_t)tenant * L + l;
     RouterEntry& rt = ctx->h_routers[r];
+    if (rt.W != nullptr && (rt.pool == MILORA_POOL_LAST || rt.pool == MILORA_POOL_SELFATTN)) --ctx->n_routers_whole_row;
     ctx->arena.give_back(const_cast<void*>(rt.W), ctx->router_bytes[r]);
     ctx->router_bytes[r] = 0;
     std::memset(&rt, 0, sizeof(rt));

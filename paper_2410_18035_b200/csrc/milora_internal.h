@@ -166,6 +166,8 @@ struct milora_ctx {
   bool dsplit_dirty;                            // counters must be cleared before the next launch pair
   int dsplit_occ_s, dsplit_occ_e;               // resident CTAs per SM of its two kernels (0 = not asked yet)
   int decode_path;                              // milora_decode_path
+  int n_routers_whole_row;                      // registered routers that pool by last token or self-attention
+  bool route_bulk_attr_set;
   // persistent multi-layer decode kernel (apply_decode_stream.cu)
   void* d_stream;                               // control words, job states, v fragments, partial sums
   size_t stream_jobs_cap, stream_frag_bytes, stream_part_bytes;   // what d_stream is laid out for

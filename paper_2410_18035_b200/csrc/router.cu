@@ -325,6 +325,256 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
   }
 }
 
+// ---- pass 1, bulk-copy form (mean and max pooling) ----------------------------------------------------------
+// The same chunks and the same partial sums as above, but H comes in through cp.async.bulk: a unit is one chunk of
+// a prompt (kRows rows) x one 2 KB strip of columns; the CTA copies 16 rows of the strip per stage (16 bulk copies of
+// 2 KB, one mbarrier) through a ring of three stages, so 96 KB per CTA and 192 KB per SM are on their way at any
+// time without a register being held for them (a plain read of this form runs at 6.9-7.1 TB/s on a B200; the
+// register-fed loads above at 5.3).  256 threads: lane l of each half owns the 16-byte column group l of the strip,
+// the first half adds the even rows of a stage, the second half the odd ones, each in row order; the two halves
+// meet when the unit ends (even rows + odd rows), so a chunk's sum does not depend on anything but the prompt.
+// Thread 0 issues the copies, one stage for every stage consumed, across unit boundaries; units come from the same
+// counter as above, asked for one unit ahead.
+constexpr int kBulkStages = 3;
+constexpr int kBulkStageRows = 16;
+constexpr int kBulkStrip = 2048;                                  // bytes of a row per unit
+constexpr int kBulkStageBytes = kBulkStageRows * kBulkStrip;
+constexpr int kBulkUnitRing = 4;
+struct BulkUnit {
+  const char* src;      // first row of the unit, at the strip's first byte
+  float* part;          // partial sums of the chunk, at the strip's first column
+  int32_t n_rows, strip_bytes, pool, valid;
+};
+
+__device__ __forceinline__ uint32_t bulk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool bulk_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads + 32, 2) pool_bulk_kernel(RouteArgs a) {
+  extern __shared__ __align__(128) unsigned char sm_raw[];
+  unsigned char* ring = sm_raw;
+  int32_t* chunk_start = reinterpret_cast<int32_t*>(sm_raw + kBulkStages * kBulkStageBytes);
+  int32_t* pool_sm = chunk_start + (a.P + 1);
+  int32_t* row_lo_sm = pool_sm + a.P;          // checked row ranges, so that the copy warp never waits for cu_seqlens
+  int32_t* row_hi_sm = row_lo_sm + a.P;
+  __shared__ int32_t carry;
+  __shared__ int32_t wsum[kWarps];
+  __shared__ uint64_t full[kBulkStages], empty[kBulkStages];
+  __shared__ BulkUnit unit_q[kBulkUnitRing];
+  __shared__ float red[kThreads / 2][8];
+  __shared__ volatile int32_t s_failed;          // a worker warp gave up on a wait: all of them leave together
+  const int kRows = a.rows;
+  constexpr int V = VecOf<T>::N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool worker = tid < kThreads;          // warps 0..7 add rows up, warp 8 issues the copies
+  const int d = a.d;
+  const size_t row_bytes = (size_t)d * sizeof(T);
+  if (tid == 0) {
+    for (int i = 0; i < kBulkStages; ++i) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bulk_smem_u32(&full[i])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bulk_smem_u32(&empty[i])), "r"(kWarps));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    carry = 0;
+    s_failed = 0;
+  }
+  pdl_wait();
+  pdl_launch_dependents();
+  __syncthreads();
+
+  // per-CTA prefix over prompts: chunks per prompt (from the checked row ranges)
+  for (int base = 0; base < a.P; base += kThreads) {
+    const int p = base + tid;
+    int chunks = 0;
+    if (worker && p < a.P) {
+      int row_lo, row_hi;
+      prompt_rows(a, p, &row_lo, &row_hi);
+      row_lo_sm[p] = row_lo;
+      row_hi_sm[p] = row_hi;
+      const int n_p = row_hi - row_lo;
+      if (n_p > 0) chunks = (n_p + kRows - 1) / kRows;
+    }
+    int sc = chunks;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int tc = __shfl_up_sync(0xffffffffu, sc, o);
+      if (lane >= o) sc += tc;
+    }
+    if (worker && lane == 31) wsum[warp] = sc;
+    __syncthreads();
+    int off = carry;
+    for (int w = 0; w < warp && w < kWarps; ++w) off += wsum[w];
+    if (worker && p < a.P) chunk_start[p] = off + sc - chunks;
+    __syncthreads();
+    if (tid == kThreads - 1) carry = off + sc;
+    __syncthreads();
+  }
+  if (tid == 0) chunk_start[a.P] = carry;
+  __syncthreads();
+  const int total_units = chunk_start[a.P] * a.n_strips;
+
+  if (!worker) {
+    // ---- copy warp: units from the counter (asked for one unit ahead), one stage of 16 row copies at a time,
+    //      one lane per row; a stage is refilled as soon as the eight worker warps have handed it back ----
+    int u_next = blockIdx.x, n_queued = 0, g_issued = 0;
+    uint32_t fetched = 0;
+    bool gave_up = false;
+    while (!gave_up) {
+      const int u = u_next;
+      if (u >= total_units) break;
+      if (lane == 0) fetched = (uint32_t)gridDim.x + (uint32_t)atomicAdd(a.sched, 1);
+      const int cg = u / a.n_strips, strip = u % a.n_strips;
+      int lo = 0, hi = a.P;                       // prompt of this chunk: last p with chunk_start[p] <= cg
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (chunk_start[mid] <= cg) lo = mid; else hi = mid;
+      }
+      const int p = lo;
+      const int r0 = row_lo_sm[p] + (cg - chunk_start[p]) * kRows;
+      const int nr = min(kRows, row_hi_sm[p] - r0);
+      const int sb = (int)min((size_t)kBulkStrip, row_bytes - (size_t)strip * kBulkStrip);
+      if (cg < a.max_chunks && nr > 0 && sb > 0) {
+        BulkUnit un;
+        un.src = static_cast<const char*>(a.H) + (size_t)r0 * row_bytes + (size_t)strip * kBulkStrip;
+        un.part = a.partial + (size_t)cg * d + (size_t)strip * (kBulkStrip / sizeof(T));
+        un.n_rows = nr; un.strip_bytes = sb; un.pool = p; un.valid = 1;      // pool: the prompt, for now
+        if (lane == 0) unit_q[n_queued % kBulkUnitRing] = un;
+        ++n_queued;
+        const int n_stages = (nr + kBulkStageRows - 1) / kBulkStageRows;
+        for (int j = 0; j < n_stages && !gave_up; ++j, ++g_issued) {
+          const int st = g_issued % kBulkStages;
+          if (g_issued >= kBulkStages) {
+            const uint32_t parity = (uint32_t)(g_issued / kBulkStages - 1) & 1u;
+            bool freed = false;
+            for (uint32_t spin = 0; spin < (4u << 20); ++spin)
+              if (bulk_try_wait(bulk_smem_u32(&empty[st]), parity)) { freed = true; break; }
+            if (!freed) { gave_up = true; break; }
+          }
+          const uint32_t bar = bulk_smem_u32(&full[st]);
+          const int r_first = j * kBulkStageRows, rows = min(kBulkStageRows, nr - r_first);
+          if (lane == 0)
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(rows * sb)) : "memory");
+          __syncwarp();
+          if (lane < rows)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                             bulk_smem_u32(ring + st * kBulkStageBytes + lane * kBulkStrip)),
+                         "l"(un.src + (size_t)(r_first + lane) * row_bytes), "r"((uint32_t)sb), "r"(bar)
+                         : "memory");
+        }
+      }
+      u_next = (int)__shfl_sync(0xffffffffu, fetched, 0);
+    }
+    // the end marker travels like a stage: its record, then an arrive on the next stage's barrier
+    if (!gave_up) {
+      const int st = g_issued % kBulkStages;
+      bool freed = g_issued < kBulkStages;
+      if (!freed) {
+        const uint32_t parity = (uint32_t)(g_issued / kBulkStages - 1) & 1u;
+        for (uint32_t spin = 0; spin < (4u << 20); ++spin)
+          if (bulk_try_wait(bulk_smem_u32(&empty[st]), parity)) { freed = true; break; }
+      }
+      if (freed && lane == 0) {
+        unit_q[n_queued % kBulkUnitRing].valid = 0;
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bulk_smem_u32(&full[st])) : "memory");
+      }
+      gave_up = !freed;
+    }
+    if (gave_up && lane == 0) atomicOr(a.tab.err, ERR_WAIT_TIMEOUT);
+    return;
+  }
+
+  // ---- worker warps ----
+  // The pooler of each prompt sits behind a chain of look-ups (slot, tenant, router entry); it is only needed when
+  // rows are added up, so the chain runs while the first copies are on their way.  A prompt without a router has
+  // its rows copied for nothing; its units are dropped below.
+  for (int p = tid; p < a.P; p += kThreads) {
+    int slot;
+    const RouterEntry* r = router_of(a, p, &slot);
+    pool_sm[p] = r ? r->pool : -1;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+  const int half = tid >> 7, l = tid & 127;
+  int g_done = 0;
+  auto wait_full = [&](int n) {          // bounded wait for stage number n; a warp that gives up tells the others
+    const uint32_t bar = bulk_smem_u32(&full[n % kBulkStages]), parity = (uint32_t)(n / kBulkStages) & 1u;
+    for (uint32_t spin = 0; spin < (4u << 20); ++spin)
+      if (bulk_try_wait(bar, parity)) return true;
+    s_failed = 1;
+    return false;
+  };
+  for (int k = 0;; ++k) {
+    // the unit's record is released by the arrive on its first stage's barrier
+    BulkUnit un;
+    un.valid = 0;
+    un.n_rows = 0;
+    bool ok = wait_full(g_done);
+    if (ok) un = unit_q[k % kBulkUnitRing];
+    if (ok && !un.valid) break;            // the end marker: every worker warp sees it
+    const int pool = ok ? pool_sm[un.pool] : -1;
+    const bool is_max = pool == MILORA_POOL_MAX;
+    const bool col_ok = ok && l * 16 < un.strip_bytes && pool >= 0;
+    float acc[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = is_max ? -FLT_MAX : 0.f;
+    const int n_stages = ok ? (un.n_rows + kBulkStageRows - 1) / kBulkStageRows : 0;
+    for (int j = 0; j < n_stages && ok; ++j, ++g_done) {
+      const int st = g_done % kBulkStages;
+      if (j > 0) ok = wait_full(g_done);
+      if (!ok) break;
+      const int rows = min(kBulkStageRows, un.n_rows - j * kBulkStageRows);
+      if (col_ok) {
+        const unsigned char* base = ring + st * kBulkStageBytes + l * 16;
+        if (is_max) {
+#pragma unroll 8
+          for (int r = half; r < rows; r += 2) {
+            float v[V];
+            unpack16(*reinterpret_cast<const uint4*>(base + r * kBulkStrip), v);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] = fmaxf(acc[i], v[i]);
+          }
+        } else {
+#pragma unroll 8
+          for (int r = half; r < rows; r += 2) {
+            float v[V];
+            unpack16(*reinterpret_cast<const uint4*>(base + r * kBulkStrip), v);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] += v[i];
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bulk_smem_u32(&empty[st])) : "memory");
+    }
+    // the halves meet: even rows + odd rows.  Every worker warp reaches these two barriers, also one that gave up.
+    if (half == 1 && col_ok) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) red[l][i] = acc[i];
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    const bool stop = s_failed != 0;
+    if (half == 0 && col_ok && !stop) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] = is_max ? fmaxf(acc[i], red[l][i]) : acc[i] + red[l][i];
+      float* dst = un.part + l * V;
+#pragma unroll
+      for (int i = 0; i < V; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");      // red is reused by the next unit
+    if (stop) break;
+  }
+  if (s_failed && tid == 0) atomicOr(a.tab.err, ERR_WAIT_TIMEOUT);
+}
+
 // ---- pass 2: one CTA per prompt combines the partials in chunk order and routes -----------------------
 // 512 threads: at d = 4096 (bf16) every thread owns one 16-byte column group, so the chain a warp has to run
 // after pass 1 has finished (fetch the partial sums, eight accurate tanh, 56 multiply-adds) is gone through once.
@@ -511,6 +761,7 @@ struct RoutePlan {
   int n_strips, rows;
   size_t max_chunks, scratch_floats, max_units;
   int T_total;
+  bool bulk;      // pass 1 through bulk copies (every registered router pools by mean or max)
 };
 
 RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
@@ -523,6 +774,13 @@ RoutePlan plan_route(const milora_ctx* ctx, int P, int T_total) {
   const size_t warp_slots = (size_t)ctx->sm_count * 5 * kWarps;
   const size_t units128 = ((size_t)T_total / 128 + P) * pl.n_strips;
   pl.rows = units128 * 10 >= warp_slots * 6 ? 128 : 64;
+  // Last-token and self-attention pooling need whole rows or a single row: they keep the register-fed kernel.
+  pl.bulk = ctx->n_routers_whole_row == 0;
+  if (pl.bulk) {
+    // 2 KB strips of 64-row chunks: at config 2 that is 2048 units for 296 CTAs, seven rounds with a thin last one
+    pl.n_strips = (int)(((size_t)d * ctx->elem + kBulkStrip - 1) / kBulkStrip);
+    pl.rows = 64;
+  }
   const int kRows = pl.rows;
   pl.max_chunks = (size_t)T_total / kRows + P;
   pl.scratch_floats = pl.max_chunks * d + 2 * pl.max_chunks;
@@ -544,16 +802,35 @@ milora_status run_route(milora_ctx* ctx, const RoutePlan& pl, int layer, const v
   a.sched = sched;
   a.layer = layer; a.P = P; a.d = ctx->desc.d_model; a.n_strips = pl.n_strips; a.rows = pl.rows;
   a.T_total = pl.T_total; a.max_chunks = (int)pl.max_chunks;
+  RoutePlan plan = pl;
+  if (plan.bulk && (reinterpret_cast<uintptr_t>(H) & 15)) {
+    // bulk copies want 16-byte aligned rows; the scratch is large enough for either plan (64-row chunks need most)
+    plan.bulk = false;
+    const int V = ctx->desc.dtype == MILORA_F32 ? 4 : 8;
+    a.n_strips = plan.n_strips = (ctx->desc.d_model + 32 * V - 1) / (32 * V);
+    plan.max_units = plan.max_chunks * plan.n_strips;
+  }
   const size_t smem = (size_t)(2 * P + 1) * sizeof(int32_t);
+  const size_t bulk_tables = (size_t)(4 * P + 1) * sizeof(int32_t);
   const bool f32 = ctx->desc.dtype == MILORA_F32;
   // pass 1: one wave of resident CTAs (a warp's first unit is assigned by index, so every CTA must start at once)
   int per_sm = 0;
   if (f32) MILORA_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pool_partial_kernel<float>, kThreads, smem));
   else MILORA_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pool_partial_kernel<__nv_bfloat16>, kThreads, smem));
   if (per_sm < 1) per_sm = 1;
-  int grid = (int)std::min<size_t>((pl.max_units + kWarps - 1) / kWarps, (size_t)ctx->sm_count * per_sm);
+  int grid = (int)std::min<size_t>((plan.max_units + kWarps - 1) / kWarps, (size_t)ctx->sm_count * per_sm);
   if (grid < 1) grid = 1;
-  if (f32) MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<float>, dim3(grid), dim3(kThreads), smem, s, a));
+  if (plan.bulk) {
+    const size_t bsmem = (size_t)kBulkStages * kBulkStageBytes + bulk_tables;
+    if (!ctx->route_bulk_attr_set) {
+      MILORA_CUDA(ctx, cudaFuncSetAttribute(pool_bulk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024));
+      MILORA_CUDA(ctx, cudaFuncSetAttribute(pool_bulk_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024));
+      ctx->route_bulk_attr_set = true;
+    }
+    const int bgrid = (int)std::max<size_t>(1, std::min<size_t>((size_t)ctx->sm_count * 2, plan.max_units));
+    if (f32) MILORA_CUDA(ctx, launch_pdl(pool_bulk_kernel<float>, dim3(bgrid), dim3(kThreads + 32), bsmem, s, a));
+    else MILORA_CUDA(ctx, launch_pdl(pool_bulk_kernel<__nv_bfloat16>, dim3(bgrid), dim3(kThreads + 32), bsmem, s, a));
+  } else if (f32) MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<float>, dim3(grid), dim3(kThreads), smem, s, a));
   else MILORA_CUDA(ctx, launch_pdl(pool_partial_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), smem, s, a));
   // pass 2: one CTA per prompt
   if (f32) MILORA_CUDA(ctx, launch_pdl(route_finalize_kernel<float>, dim3(P), dim3(kFinThreads), 0, s, a));
