@@ -252,6 +252,12 @@ def run_ours(args, rank, world, device):
         from synth.workloads import scaled_workload
         w = scaled_workload(w, prefill_ids=w.prefill_ids[:args.prompts], decode_ids=w.decode_ids[:args.prompts],
                             name=w.name + f"_first{args.prompts}")
+    if args.only_shared_prefill:
+        # a small process for profiler captures: the k = 3 prefill apply alone, one of its two forms
+        if rank == 0:
+            print(json.dumps({"shared_input_prefill_k3": run_shared_prefill(w, device, load_peaks(),
+                                                                            mode=args.only_shared_prefill, iters=2)}))
+        return None
     lw = LoadedWorkload(w, device, layers=[0])
     if args.only_decode_stack:
         # a small process for profiler captures: the decode chain of the 7B stack alone, a few GB on the device
@@ -319,7 +325,7 @@ def run_ours(args, rank, world, device):
     ms_per_step = total_ms / args.steps
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
-    fused = stack = stack13 = mixed = sweep = None
+    fused = stack = stack13 = mixed = sweep = shared_k3 = None
     router_alone = run_router_alone(step, device, work["router_bytes"], load_peaks()) if rank == 0 else None
     if rank == 0 and not args.skip_fused and w.dtype == "bf16":
         mixed = run_mixed_step(step, device)
@@ -327,6 +333,7 @@ def run_ours(args, rank, world, device):
         stack = run_decode_stack(step, device, load_peaks())
         stack13 = run_decode_13b(device, load_peaks())
         sweep = run_decode_sweep(device, load_peaks())
+        shared_k3 = run_shared_prefill(w, device, load_peaks())
     # ---- end to end: pinned host inputs -> device -> path -> host -------------------------------
     e2e = None if args.skip_e2e else run_e2e(step, args, world, device, tokens_per_step)
     gpu_check = checked_step_outputs(step, device) if (rank == 0 and not args.skip_cpu) else None
@@ -386,6 +393,7 @@ def run_ours(args, rank, world, device):
             "decode_stack_13b_zipf": stack13,
             "decode_batch_sweep": sweep,
             "mixed_batch_step": mixed,
+            "shared_input_prefill_k3": shared_k3,
         },
         "roofline": dict(rooflines[dom], kernel=dom),
         "rooflines": rooflines,
@@ -852,6 +860,55 @@ def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=8
     return {"workload": "c5_llama3_8b_decode_sweep_bf16", "layers": n_layers, "rank": 16, "sweep": out}
 
 
+def run_shared_prefill(w, device, peaks, mode="both", iters=20):
+    """Section 3.3 with k = 3: every prompt selects q, k and v (the table is written by hand; the router is not
+    what is measured here), which read the same input.  `separate` gives milora_apply_prefill_multi three distinct
+    X matrices, `shared` gives milora_apply_prefill_shared one: every X tile is then copied once for the three
+    shrinks.  Algorithmic bytes: X once per matrix read plus y read and written per module."""
+    from paper_2410_18035_b200.workload_runner import LoadedWorkload
+    lw = LoadedWorkload(w, device, layers=[0], top_k=3)
+    ml = lw.ml
+    ids = [int(i) for i in w.prefill_ids]
+    rows = np.zeros((w.n_requests, 1, 3), dtype=np.int32)
+    for i in range(w.n_requests):
+        rows[i, 0] = np.roll([0, 1, 2], i % 3)
+    ml.route_table_write(0, rows)
+    cu, slots, T = lw.seq_arrays(ids, [])
+    ws = ml.alloc_group_ws(1, len(ids), T)
+    ml.group(0, 1, cu, slots, len(ids), T, ws)
+    groups = ml.groups(ws[0], len(ids), T)
+    gen = torch.Generator(device=device).manual_seed(7)
+    dims = [ml.module_dims(m) for m in range(3)]
+    X = [torch.randn(T, dims[m][0], device=device, generator=gen).to(torch.bfloat16) for m in range(3)]
+    Y = [torch.randn(T, dims[m][1], device=device, generator=gen).to(torch.bfloat16) for m in range(3)]
+    calls = {"separate": lambda: ml.apply_prefill_multi(0, [0, 1, 2], X, Y, groups),
+             "shared": lambda: ml.apply_prefill_shared(0, [0, 1, 2], X[0], Y, groups)}
+    xb = X[0].numel() * 2
+    yb = sum(2 * y.numel() * 2 for y in Y)
+    out = {"tokens": T, "top_k": 3, "modules": "q,k,v", "launches_per_call": 2}
+    for name, fn in calls.items():
+        if mode not in ("both", name):
+            continue
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(device)
+        ms = e0.elapsed_time(e1) / iters
+        nbytes = (xb if name == "shared" else 3 * xb) + yb
+        out[name] = {"ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6,
+                     "frac_of_measured_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
+    err = ml.poll_error()
+    lw.close()
+    if err:
+        raise RuntimeError(f"shared-input prefill: device error flags {err}")
+    return out
+
+
 def run_e2e(step, args, world, device, tokens_per_step):
     """Same step through milora_step_host: every input starts in pinned HOST memory, the C ABI copies it
     in, runs the path and copies every output back; all of it is inside the timed region."""
@@ -1088,6 +1145,8 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle timing")
     ap.add_argument("--only-decode-stack", action="store_true",
                     help="profiling runs: only the decode chain of the 7B stack (--chain-layers layers), a few GB on the device")
+    ap.add_argument("--only-shared-prefill", choices=["shared", "separate", "both"], default=None,
+                    help="profiling runs: only the k = 3 prefill apply on q, k, v, with one shared input matrix or three")
     ap.add_argument("--chain-layers", type=int, default=8)
     ap.add_argument("--prompts", type=int, default=None,
                     help="profiling runs: only the first N prompts and decode requests of the step (not a bench line)")
@@ -1114,7 +1173,7 @@ def main():
     if world > 1:
         torch.distributed.barrier()
     out = run_ours(args, rank, world, device)
-    if rank == 0:
+    if rank == 0 and out is not None:           # the profiling modes print their own line
         print(json.dumps(out), flush=True)
     if world > 1:
         torch.distributed.destroy_process_group()

@@ -223,6 +223,8 @@ milora_status milora_gate_table_write(milora_ctx* ctx, int slot_begin, int n_slo
 typedef struct {
   size_t header, mod_offset, mod_tile_offset, mod_gather_offset;
   size_t seg_key, seg_offset, perm, tiles, gather_rows, gather;
+  size_t seq_tile;           /* [n_seq][8]: first dense tile of (sequence, module m) at [m], -1 if none; [7] = bit mask
+                                of the modules that have tiles for the sequence */
   size_t total;              /* int32 elements of one layer block (multiple of 4) */
   int max_tiles, max_gather;
 } milora_group_layout_t;
@@ -314,6 +316,16 @@ milora_status milora_apply_decode_multi(milora_ctx* ctx, int layer, int n_sites,
 milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites, const int* modules,
                                          const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                          void* stream);
+
+/* Modules of one layer that read the SAME input matrix X_dev [T][d1] (q, k, v read the attention input; gate and up
+ * the MLP input; all listed modules must have the same d1, else MILORA_E_ARG): Y_dev[i] [T][d2(modules[i])] +=
+ * s (x W^A) W^B of module modules[i] on the rows whose request selects it (Eq. 1 with the routing of Section 3.3).
+ * With top_k == 1 a row selects one module and this is milora_apply_prefill_multi.  With top_k > 1 a sequence
+ * that selects several of the listed modules has every 128-row tile of X read once for all of them (up to three
+ * modules per pass), instead of once per module.  milora_apply_prefill_multi does the same whenever it is given
+ * equal X_dev pointers.  Results are those of separate milora_apply_prefill calls, bit for bit. */
+milora_status milora_apply_prefill_shared(milora_ctx* ctx, int layer, int n_sites, const int* modules, const void* X_dev,
+                                          void* const* Y_dev, const milora_groups* groups, void* stream);
 
 /* ---- fused projection (Eq. 1 in one pass) ---------------------------------------------------------
  * Y_dev [T][d2] = X_dev [T][d1] . W_m + b_m for EVERY row of the step, plus s (x W^A) W^B on the rows of long

@@ -37,7 +37,8 @@ class ModelDesc(C.Structure):
 
 class GroupLayout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("header", "mod_offset", "mod_tile_offset", "mod_gather_offset", "seg_key",
-                                           "seg_offset", "perm", "tiles", "gather_rows", "gather", "total")]
+                                           "seg_offset", "perm", "tiles", "gather_rows", "gather", "seq_tile",
+                                           "total")]
     _fields_ += [("max_tiles", C.c_int), ("max_gather", C.c_int)]
 
 
@@ -87,6 +88,7 @@ SIGNATURES = {
     "milora_apply_prefill": (_I, [_VP, _I, _I, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_apply_decode_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
     "milora_apply_prefill_multi": (_I, [_VP, _I, _I, C.POINTER(_I), C.POINTER(_VP), C.POINTER(_VP), C.POINTER(Groups), _VP]),
+    "milora_apply_prefill_shared": (_I, [_VP, _I, _I, C.POINTER(_I), _VP, C.POINTER(_VP), C.POINTER(Groups), _VP]),
     "milora_linear_prefill": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, C.POINTER(Groups), _VP]),
     "milora_step_host_workspace": (_I, [_VP, C.POINTER(HostStep), C.POINTER(C.c_size_t)]),
     "milora_step_host": (_I, [_VP, C.POINTER(HostStep), _VP, C.c_size_t, _VP]),
@@ -374,6 +376,16 @@ class Milora:
 
     def apply_prefill_multi(self, layer, modules, Xs, Ys, groups: Groups, stream=None):
         self._multi(self.lib.milora_apply_prefill_multi, "milora_apply_prefill_multi", layer, modules, Xs, Ys, groups, stream)
+
+    def apply_prefill_shared(self, layer, modules, X, Ys, groups: Groups, stream=None):
+        """milora_apply_prefill_shared: the listed modules all read X ([T, d1]); Ys[i] is module i's output."""
+        n = len(modules)
+        for m, Y in zip(modules, Ys):
+            self._xy(m, X, Y, groups.T)
+        mods = (C.c_int * n)(*modules)
+        ys = (C.c_void_p * n)(*[Y.data_ptr() for Y in Ys])
+        self._check(self.lib.milora_apply_prefill_shared(self.h, layer, n, mods, _ptr(X), ys, C.byref(groups),
+                                                         _stream(stream)), "milora_apply_prefill_shared")
 
     def linear_prefill(self, layer, module, X, Wt, Y, groups: Groups, bias=None, stream=None):
         """milora_linear_prefill: Y = X W + b + LoRA term of the routed prompt rows; Wt is [d2, d1]."""

@@ -53,6 +53,9 @@ struct ShrinkArgs {
   milora_group_layout_t lay;
   float* vscratch;     // [kKSplit][max_tiles * 128][rpad]: indexed by tile, since with top-k routing a row sits in several tiles
   int T, rpad;
+  // shared-input variant only
+  int share[kMaxSites];        // sites with equal values read the same X matrix
+  int K, n_ent, stages;        // selected modules per sequence, entries of the batch, depth of the copy ring
 };
 
 struct ExpandArgs {
@@ -214,6 +217,204 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
     }
   }
   if (warp == 0 && lane == 0) drain_ring(abort_ptr, issued, kShrinkStages, full);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, ncols);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// shrink, shared input
+// ------------------------------------------------------------------------------------------------------
+// With top-k routing (Section 3.3 allows k > 1) a sequence selects several modules of a layer, and q, k, v (or gate
+// and up) read the same X.  Every selected module has its own tiles over the sequence's rows; tile r of each
+// sibling covers the same 128 rows.  Here one CTA takes up to kMaxShare sibling tiles at once: every X stage is
+// copied once and multiplied with each sibling's A image into its own tensor-memory columns.  The sibling with
+// the lowest module number leads; the CTAs of the others return at once.  The
+// partial products land where the plain shrink kernel would have put them, so the expand kernel does not change.
+constexpr int kMaxShare = 3;
+
+__device__ __forceinline__ uint32_t tmem_cols_pow2(int cols) {
+  uint32_t c = 32;
+  while ((int)c < cols) c <<= 1;
+  return c;
+}
+
+__global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_shared_kernel(const __grid_constant__ ShrinkArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ks = blockIdx.x % kKSplit;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int n_tiles = min(a.ws[a.lay.header + H_NTILES], a.lay.max_tiles);
+  const int tile_idx = n_tiles - 1 - (int)(blockIdx.x / kKSplit);
+  if (tile_idx < 0) return;
+  const TileJob* tiles = reinterpret_cast<const TileJob*>(a.ws + a.lay.tiles);
+  const TileJob job = tiles[tile_idx];
+  const int si = find_site(a.sites, job.module);
+  if (si < 0) return;
+  const uint32_t base = smem_u32(smem_raw);
+  const int stages = a.stages;
+  const int ent = job.ent & 0xffff, tiled = (job.ent >> 16) & 0x7f;
+  bool bad = (base & 1023) || ent >= a.n_ent || job.module < 0 || job.module >= MILORA_NMOD || !(tiled >> job.module & 1) ||
+             job.count < 1 || job.count > kTileRows || job.start < 0 || job.start + job.count > a.T || stages < 2;
+  if (bad) {
+    if (tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  // ---- the siblings: modules with tiles for this sequence whose site reads the same X, by module number; the
+  // record of the tile says which modules those are, so a CTA that does not lead leaves without another load ----
+  int sib = 0;
+#pragma unroll
+  for (int m = 0; m < MILORA_NMOD; ++m) {
+    const int sj = find_site(a.sites, m);
+    if ((tiled >> m & 1) && sj >= 0 && a.share[sj] == a.share[si]) sib |= 1 << m;
+  }
+  if (__popc(sib & ((1 << job.module) - 1)) % kMaxShare) return;      // an earlier sibling leads this tile
+  int mem_mod[kMaxShare], mem_tile[kMaxShare];
+  int n_mem = 0;
+#pragma unroll
+  for (int m = 0; m < MILORA_NMOD; ++m)
+    if (m >= job.module && (sib >> m & 1) && n_mem < kMaxShare) mem_mod[n_mem++] = m;
+  const int32_t* seq_tile = a.ws + a.lay.seq_tile + 8 * (size_t)(ent / a.K);
+#pragma unroll
+  for (int m = 0; m < kMaxShare; ++m) mem_tile[m] = m < n_mem ? seq_tile[mem_mod[m]] : -1;
+  const int r = tile_idx - mem_tile[0];                 // this tile's position among the tiles of its sequence
+  bad = mem_tile[0] < 0 || r < 0;
+
+  const void* img[kMaxShare];
+  int rp[kMaxShare], col[kMaxShare];
+  TileJob sjob[kMaxShare];
+#pragma unroll
+  for (int m = 0; m < kMaxShare; ++m) {
+    const int t = mem_tile[m] + r;
+    bad = bad || (m < n_mem && (mem_tile[m] < 0 || t >= n_tiles));
+    mem_tile[m] = t;
+    if (m > 0 && m < n_mem && !bad) sjob[m] = tiles[t];
+  }
+  sjob[0] = job;
+  int cols = 0;
+#pragma unroll
+  for (int m = 0; m < kMaxShare; ++m) {
+    img[m] = nullptr; rp[m] = 0; col[m] = cols;
+    if (m < n_mem && !bad) {
+      img[m] = sjob[m].At_img;
+      rp[m] = sjob[m].rank_pad;
+      bad = bad || !img[m] || rp[m] < 16 || rp[m] > a.rpad || (rp[m] & 15) || sjob[m].start != job.start ||
+            sjob[m].count != job.count || sjob[m].module != mem_mod[m];
+      cols += rp[m];
+    }
+  }
+  if (bad) {
+    if (tid == 0) atomicOr(a.err, ERR_BAD_ITEM);
+    return;
+  }
+  const int d1 = a.sites.d1[si];
+  const int nchunks = d1 / kBK, cps = (nchunks + kKSplit - 1) / kKSplit;
+  const int kc0 = ks * cps, kc1 = min(nchunks, kc0 + cps), nk = max(kc1 - kc0, 0);
+
+  const uint32_t xs = base;
+  const uint32_t as = xs + stages * kXStage;
+  const uint32_t a_one = (uint32_t)a.rpad * 128u;           // one sibling's A chunk
+  const uint32_t a_stage = kMaxShare * a_one;
+  const uint32_t bars = as + stages * a_stage;
+  auto full = [&](int i) { return bars + 8u * i; };
+  auto empty = [&](int i) { return bars + 8u * (stages + i); };
+  const uint32_t accb = bars + 16u * stages;
+  const uint32_t slot = accb + 8u;
+  volatile uint32_t* slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - base));
+  volatile int* abort_ptr = reinterpret_cast<volatile int*>(smem_raw + (slot + 4 - base));
+  const uint32_t ncols = tmem_cols_pow2(cols);
+
+  if (tid == 0) {
+    *abort_ptr = 0;
+    for (int i = 0; i < stages; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), n_mem); }
+    mbar_init(accb, n_mem);
+    fence_barrier_init();
+    prefetch_tensormap(&a.xmap[si]);
+  }
+  __syncthreads();
+  if (warp == 0) { tmem_alloc(slot, ncols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *slot_ptr;
+
+  // One thread starts a copy or an MMA every fifty to a hundred cycles, and a stage arrives from memory about every
+  // 1400: the copies of a stage (X tile, one A chunk per sibling) stay with one thread, and every sibling's four
+  // MMAs get a thread of their own (warps 1, 2, 3), each of which commits to the stage's `empty` barrier.
+  int issued = 0;
+  if (nk > 0) {
+    if (warp == 0) {
+      if (lane == 0) {
+        // ---- copies: the X tile once, one A image chunk per sibling ----
+        for (int i = 0; i < nk; ++i) {
+          const int s = i % stages, ph = (i / stages) & 1;
+          if (i >= stages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
+          mbar_expect_tx(full(s), kXStage + cols * 128);
+          tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
+#pragma unroll
+          for (int m = 0; m < kMaxShare; ++m)
+            if (m < n_mem)
+              bulk_g2s(as + s * a_stage + m * a_one, static_cast<const char*>(img[m]) + (size_t)(kc0 + i) * rp[m] * 128,
+                       rp[m] * 128, full(s));
+          issued = i + 1;
+        }
+      }
+    } else if (lane == 0 && warp - 1 < n_mem) {
+      // ---- MMAs of sibling warp - 1: D_m[128 x rp_m] += X[128 x 16] * A_m[16 x rp_m], four per stage ----
+      int rp_m = 0, col_m = 0;
+#pragma unroll
+      for (int m = 0; m < kMaxShare; ++m)
+        if (m == warp - 1) { rp_m = rp[m]; col_m = col[m]; }
+      const uint32_t idesc = idesc_bf16_f32(kTileRows, rp_m);
+      const uint32_t lbo = (uint32_t)(rp_m / 8) * 128u;        // A image: k-adjacent core matrices
+      const uint32_t a_m = as + (uint32_t)(warp - 1) * a_one;
+      bool ok = true;
+      for (int i = 0; i < nk && ok; ++i) {
+        const int s = i % stages, ph = (i / stages) & 1;
+        ok = wait_bar(full(s), ph, abort_ptr, a.err);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kBK / 16; ++kk) {
+          const uint64_t da = smem_desc(xs + s * kXStage + kk * 32, 16, 1024, 2);
+          const uint64_t db = smem_desc(a_m + s * a_stage + kk * 2 * lbo, lbo, 128, 0);
+          mma_bf16_ss(tmem_base + col_m, da, db, idesc, (i | kk) != 0);
+        }
+        mma_commit(empty(s));
+      }
+      mma_commit(accb);
+    }
+  }
+  __syncwarp();
+
+  // ---- epilogue: every sibling's fp32 partial product to its own tile of the scratch ----
+  bool ok = true;
+  if (nk > 0) ok = wait_bar(accb, 0, abort_ptr, a.err);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  const int row = warp * 32 + lane;
+#pragma unroll
+  for (int m = 0; m < kMaxShare; ++m) {
+    if (m >= n_mem) continue;
+    float* dst = a.vscratch + (((size_t)ks * a.lay.max_tiles + mem_tile[m]) * kTileRows + row) * a.rpad;
+    for (int c0 = 0; c0 < rp[m]; c0 += 16) {
+      uint32_t v[16];
+      if (nk > 0 && ok) {
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + col[m] + c0, v);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = 0u;
+      }
+      if (row < job.count) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4)
+          *reinterpret_cast<uint4*>(dst + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+      }
+    }
+  }
+  if (warp == 0 && lane == 0) drain_ring(abort_ptr, issued, stages, full);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, ncols);
@@ -863,7 +1064,33 @@ static milora_status launch_prefill(milora_ctx* ctx, const ApplySites& sites, co
   MILORA_CUDA(ctx, cudaFuncSetAttribute(prefill_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)expand_smem));
   const size_t grid_s = (size_t)lay.max_tiles * kKSplit, grid_e = (size_t)lay.max_tiles * kNSplit;
   if (grid_s > 0x7fffffffull || grid_e > 0x7fffffffull) return MILORA_E_CAPACITY;
-  MILORA_CUDA(ctx, launch_pdl(prefill_shrink_kernel, dim3((unsigned)grid_s), dim3(kShrinkThreads), shrink_smem, s, sa));
+  // Sites that were given the same X (q, k, v; gate, up) and a context that selects several modules per sequence:
+  // the shared-input shrink copies every X tile once for all of a sequence's modules among them.
+  bool any_shared = false;
+  for (int i = 0; i < kMaxSites; ++i) sa.share[i] = i;
+  for (int i = 0; i < sites.n; ++i)
+    for (int j = 0; j < i; ++j)
+      if (sites.site[j].X == sites.site[i].X && sites.site[j].d1 == sites.site[i].d1) {
+        sa.share[i] = sa.share[j];
+        any_shared = true;
+        break;
+      }
+  sa.K = top_k_of(ctx);
+  sa.n_ent = g->n_seq * sa.K;
+  sa.stages = kShrinkStages;
+  if (any_shared && sa.K > 1) {
+    const size_t per = (size_t)kXStage + (size_t)kMaxShare * rpad * 128;
+    const size_t two_per_sm = 113 * 1024 - 256, one_per_sm = 220 * 1024 - 256;
+    int stages = (int)std::min<size_t>(kShrinkStages, two_per_sm / per);
+    if (stages < 4) stages = (int)std::min<size_t>(kShrinkStages, one_per_sm / per);
+    if (stages < 2) return MILORA_E_SHAPE;
+    sa.stages = stages;
+    const size_t smem = (size_t)stages * per + 256;
+    MILORA_CUDA(ctx, cudaFuncSetAttribute(prefill_shrink_shared_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MILORA_CUDA(ctx, launch_pdl(prefill_shrink_shared_kernel, dim3((unsigned)grid_s), dim3(kShrinkThreads), smem, s, sa));
+  } else {
+    MILORA_CUDA(ctx, launch_pdl(prefill_shrink_kernel, dim3((unsigned)grid_s), dim3(kShrinkThreads), shrink_smem, s, sa));
+  }
   if (shrink_only) return MILORA_OK;
   MILORA_CUDA(ctx, launch_pdl(prefill_expand_kernel, dim3((unsigned)grid_e), dim3(kExpandThreads), expand_smem, s, ea));
   return MILORA_OK;

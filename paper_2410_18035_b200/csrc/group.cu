@@ -92,6 +92,7 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
   int32_t* ws = a.ws + (size_t)blockIdx.x * a.ws_stride;
   const int max_tenants = a.tab.max_tenants;
   const int K = a.tab.top_k, n_ent = a.n_ent;
+  int32_t* seq_tile = ws + a.lay.seq_tile;      // [n_seq][8]: first dense tile per module (-1: none), [7] = module mask
   pdl_launch_dependents();
   pdl_wait();
 
@@ -113,6 +114,7 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
     if (ok && len > 0) tenant = a.tab.slot_tenant[slot];
     const bool tenant_ok = tenant >= 0 && tenant < max_tenants;
     bool any = false;
+    int tiled = 0;                             // modules that get dense tiles for this sequence
     for (int j = 0; j < K; ++j) {
       int c = INT_MAX;
       float gt = 1.f;
@@ -130,7 +132,10 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
       }
       comp[i * K + j] = c;
       ent_gate[i * K + j] = gt;
+      if (c != INT_MAX && len >= kLongSeq) tiled |= 1 << ((c >> kSeqBits) / max_tenants);
     }
+    for (int m = 0; m < MILORA_NMOD; ++m) seq_tile[8 * i + m] = -1;
+    seq_tile[8 * i + 7] = tiled;
     if (!any) excl += len;
   }
   int n_excl;
@@ -216,7 +221,9 @@ __global__ void __launch_bounds__(kGMaxThreads) group_kernel(GroupArgs a) {
       const AdapterEntry e = a.tab.adapters[adapter_index(key % max_tenants, layer, module, a.tab.n_layers)];
       TileJob w;
       w.At = e.At; w.B = e.B; w.At_img = e.At_img; w.B_img = e.B_img;
-      w.rank = e.rank; w.scale = e.scale * ent_gate[ent]; w.module = module; w.seg = seg; w.rank_pad = e.rank_pad; w.pad = 0;
+      w.rank = e.rank; w.scale = e.scale * ent_gate[ent]; w.module = module; w.seg = seg; w.rank_pad = e.rank_pad;
+      w.ent = ent | (seq_tile[8 * (ent / K) + 7] << 16);
+      seq_tile[8 * (ent / K) + module] = o_tile;
       for (int r = 0; r < len; r += kTileRows) {
         w.start = lo + r;
         w.count = min(kTileRows, len - r);

@@ -105,6 +105,7 @@ milora_group_layout_t group_layout(int n_seq, int T, int top_k) {
   // gathered rows belong to sequences shorter than kLongSeq, so there are at most (kLongSeq - 1) per entry
   L.max_gather = (int)(std::min(TT, (size_t)(kLongSeq - 1) * n_ent) / kGatherRows + n_ent + 1);
   L.gather = o; o += (size_t)L.max_gather * kJobInts;
+  L.seq_tile = o; o += (size_t)n_seq * 8;
   L.total = round4(o);
   return L;
 }
@@ -750,6 +751,22 @@ milora_status milora_apply_prefill_multi(milora_ctx* ctx, int layer, int n_sites
                                          const void* const* X_dev, void* const* Y_dev, const milora_groups* groups,
                                          void* stream) {
   return apply_common(ctx, layer, n_sites, modules, X_dev, Y_dev, groups, true, stream);
+}
+
+milora_status milora_apply_prefill_shared(milora_ctx* ctx, int layer, int n_sites, const int* modules, const void* X_dev,
+                                          void* const* Y_dev, const milora_groups* groups, void* stream) {
+  if (!ctx || !modules || n_sites < 1 || n_sites > kMaxSites) return MILORA_E_ARG;
+  const void* X[kMaxSites];
+  int d1_first = 0;
+  for (int i = 0; i < n_sites; ++i) {
+    if (modules[i] < 0 || modules[i] >= MILORA_NMOD) return MILORA_E_ARG;
+    int d1, d2;
+    module_dims(ctx->desc, modules[i], &d1, &d2);
+    if (i == 0) d1_first = d1;
+    if (d1 != d1_first) return MILORA_E_ARG;      // modules that read one matrix have one input width
+    X[i] = X_dev;
+  }
+  return apply_common(ctx, layer, n_sites, modules, X, Y_dev, groups, true, stream);
 }
 
 milora_status milora_linear_prefill(milora_ctx* ctx, int layer, int module, const void* X_dev, const void* Wt_dev,

@@ -65,7 +65,8 @@ struct TileJob {         // `count` consecutive rows starting at `start`
   const void* B_img;
   int32_t rank;
   float scale;
-  int32_t module, count, seg, start, rank_pad, pad;
+  int32_t module, count, seg, start, rank_pad;
+  int32_t ent;             // bits 0..15: entry index (sequence * top_k + j); bits 16..22: modules with tiles for the sequence
 };
 static_assert(sizeof(GatherJob) == 64 && sizeof(TileJob) == 64, "job records are 64 bytes");
 

@@ -42,10 +42,13 @@ def _route_all_layers(lw, ids, **okw):
     return table_g, table_o, excused
 
 
-def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, gate=None, decode_path="auto"):
+def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, gate=None, decode_path="auto",
+                 shared=None):
     """group + apply (prefill and decode lists) on one step; compares grouping and all 7 module outputs.
     table is [R, L] (top-1) or [R, L, k]; gate, when given, holds the [R, L, k] weights of the selected modules.
-    decode_path picks the kernel set of milora_apply_decode (bf16 contexts)."""
+    decode_path picks the kernel set of milora_apply_decode (bf16 contexts).  shared: lists of modules that are
+    given one input matrix; the prefill rows then go through milora_apply_prefill_shared (use_multi: through
+    milora_apply_prefill_multi with equal X pointers)."""
     w, ml = lw.w, lw.ml
     ml.set_decode_path(decode_path)
     layer = lw.layers[li]
@@ -68,7 +71,17 @@ def _step_parity(lw, li, prefill_ids, decode_ids, table, tag, use_multi=False, g
         else:
             Yb = w.base_output(layer, m, T, tag, "cuda")
         Xs.append(X); Ybs.append(Yb); Ys.append(Yb.clone())
-    if use_multi:
+    for mods in shared or []:
+        for m in mods[1:]:
+            Xs[m] = Xs[mods[0]]
+    if shared and not use_multi:
+        rest = [m for m in range(7) if not any(m in mods for mods in shared)]
+        for mods in shared:
+            ml.apply_prefill_shared(li, list(mods), Xs[mods[0]], [Ys[m] for m in mods], groups)
+        for m in rest:
+            ml.apply_prefill(li, m, Xs[m], Ys[m], groups)
+        ml.apply_decode_multi(li, list(range(7)), Xs, Ys, groups)
+    elif use_multi:
         ml.apply_prefill_multi(li, list(range(7)), Xs, Ys, groups)
         ml.apply_decode_multi(li, list(range(7)), Xs, Ys, groups)
     else:
@@ -169,7 +182,8 @@ def test_ragged_mixed_batch(dtype, d, d_ff, d_kv, r, decode_path):
 
 @pytest.mark.parametrize("dtype,d,d_ff,d_kv,r,k,gate", [("f32", 256, 688, 256, 8, 3, 0), ("bf16", 512, 1408, 128, 16, 3, 0),
                                                         ("bf16", 512, 1408, 512, 32, 2, 1), ("f32", 256, 688, 256, 8, 7, 1),
-                                                        ("bf16", 256, 688, 256, 40, 3, 1)])
+                                                        ("bf16", 256, 688, 256, 40, 3, 1), ("bf16", 2048, 1408, 256, 16, 3, 0),
+                                                        ("bf16", 512, 1408, 512, 64, 5, 1)])
 def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
     """Eq. 3 with k > 1 (Section 4.5 sweeps k): the route table holds the k best modules in order, every token
     is bucketed once per selected module and receives each selected module's LoRA term, optionally weighted by
@@ -211,6 +225,13 @@ def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
     for li in range(2):
         _step_parity(lw, li, prefill, decode, table, tag=11, gate=gate_arg, decode_path="cluster")
         _step_parity(lw, li, prefill[::-1], decode, table, tag=12, use_multi=True, gate=gate_arg, decode_path="split")
+        # q, k, v read one matrix and gate, up another (Section 3.1 lists the seven modules of a block): one X tile
+        # feeds the shrink of every selected module of the group
+        _step_parity(lw, li, prefill, decode, table, tag=13, gate=gate_arg, shared=[(0, 1, 2), (4, 5)])
+        _step_parity(lw, li, prefill[::-1], decode, table, tag=14, use_multi=True, gate=gate_arg,
+                     shared=[(0, 1, 2), (4, 5)])
+        # more siblings than one pass takes: five modules on one matrix
+        _step_parity(lw, li, prefill, decode, table, tag=15, use_multi=True, gate=gate_arg, shared=[(5, 0, 4, 2, 1)])
     # restoring a table by hand: duplicates inside a cell are refused
     from paper_2410_18035_b200 import MiloraError
     if k >= 2:
