@@ -1116,6 +1116,9 @@ milora_status launch_linear_prefill_bf16(milora_ctx* ctx, int layer, int module,
   if ((reinterpret_cast<uintptr_t>(X) & 15) || (reinterpret_cast<uintptr_t>(Y) & 15) ||
       (reinterpret_cast<uintptr_t>(Wt) & 15) || (reinterpret_cast<uintptr_t>(bias) & 1))
     return MILORA_E_SHAPE;
+  // every check the host can make comes before the first thing is put on the stream
+  LinearArgs la;
+  if (!make_map(&la.xmap, X, T, d1, kLinBM) || !make_map(&la.wmap, Wt, d2, d1, kLinBN)) return MILORA_E_SHAPE;
   const milora_group_layout_t lay = group_layout(g->n_seq, g->T, top_k_of(ctx));
   const int n_mblk = (T + kLinBM - 1) / kLinBM, n_nblk = d2 / kLinBN;
   const size_t img_bytes = (size_t)kTileRows * rpad * 2;
@@ -1147,8 +1150,6 @@ milora_status launch_linear_prefill_bf16(milora_ctx* ctx, int layer, int module,
   if (lay.max_tiles > 0)
     MILORA_CUDA(ctx, launch_pdl(linear_vpack_kernel, dim3((unsigned)lay.max_tiles), dim3(kTileRows), 0, s, pa));
 
-  LinearArgs la;
-  if (!make_map(&la.xmap, X, T, d1, kLinBM) || !make_map(&la.wmap, Wt, d2, d1, kLinBN)) return MILORA_E_SHAPE;
   la.err = ctx->d_err; la.ws = g->ws_dev; la.lay = lay; la.vimg = lin; la.piece_cnt = pa.piece_cnt; la.piece_job = pa.piece_job;
   la.bias = static_cast<const __nv_bfloat16*>(bias); la.Y = static_cast<__nv_bfloat16*>(Y);
   la.T = T; la.d1 = d1; la.d2 = d2; la.rpad = rpad; la.n_mblk = n_mblk; la.n_nblk = n_nblk;

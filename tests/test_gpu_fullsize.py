@@ -304,3 +304,50 @@ def test_config2_fused_projection_full_size():
         assert (differs[routed] > 0.5).all() and (differs[~routed] < 0.02).all()
         del Wt, X, Y
     lw.close()
+
+
+def test_config2_top3_shared_input_full_size():
+    """Section 3.3 with k = 3 at config 2's sizes: q, k, v read one matrix and gate, up another.  The shared-input
+    call must give, bit for bit, what one call per module gives, and on sampled rows the oracle's value."""
+    w = get_workload("c2")
+    w.gen_device = "cuda"
+    lw = _loaded(w, layers=[0], top_k=3)
+    ml = lw.ml
+    ids = list(range(64))
+    lw.route(0, ids)
+    table = ml.route_table_read(0, w.n_requests).numpy().reshape(w.n_requests, 1, 3)[:, 0].copy()
+    assert all(len(set(row.tolist())) == 3 for row in table[ids])
+    cu, slots, T = lw.seq_arrays(ids, [])
+    ws = ml.alloc_group_ws(1, len(ids), T)
+    ml.group(0, 1, cu, slots, len(ids), T, ws)
+    groups = ml.groups(ws[0], len(ids), T)
+    cu_h = cu.cpu().numpy()
+    token_slot = np.repeat(slots.cpu().numpy(), np.diff(cu_h))
+    shared = [(0, 1, 2), (4, 5)]
+    # the sharing must really occur: prompts that select at least two modules of a group
+    n_sharing = sum(int(np.isin(table[i], mods).sum() >= 2) for i in ids for mods in shared)
+    assert n_sharing >= 8, "the routed table gives the shared-input kernel nothing to share"
+    Xs = {mods: w.module_input(0, mods[0], T, 21, "cuda") for mods in shared}
+    rng = np.random.default_rng(5)
+    rows = _sample_rows(cu_h, rng, per_seq=3)
+    for mods in shared:
+        X = Xs[mods]
+        Ybs = [w.base_output(0, m, T, 21, "cuda") for m in mods]
+        Y_shared = [y.clone() for y in Ybs]
+        Y_single = [y.clone() for y in Ybs]
+        ml.apply_prefill_shared(0, list(mods), X, Y_shared, groups)
+        for m, Y in zip(mods, Y_single):
+            ml.apply_prefill(0, m, X, Y, groups)
+        torch.cuda.synchronize()
+        assert ml.poll_error() == 0
+        for m, Yb, Ys, Y1 in zip(mods, Ybs, Y_shared, Y_single):
+            assert torch.equal(Ys, Y1), f"module {m}: shared-input call differs from the single call"
+            active = torch.from_numpy((table[token_slot] == m).any(axis=1)).cuda()
+            assert torch.equal(Ys[~active], Yb[~active]), f"module {m}: an unrouted row changed"
+            sel = rows[(table[token_slot[rows]] == m).any(axis=1)]
+            if sel.size == 0:
+                continue
+            idx = torch.from_numpy(sel).cuda()
+            y_o = R.apply_site(w, 0, m, X[idx].cpu(), Yb[idx].cpu(), token_slot, table, rows=sel)
+            assert_apply_close(Ys[idx], y_o, Yb[idx], w.dtype, what=f"c2 top-3 shared input, module {m}")
+    lw.close()
