@@ -623,8 +623,29 @@ def run_router_alone(step, device, nbytes, peaks, iters=40):
     torch.cuda.synchronize(device)
     ms = e0.elapsed_time(e1) / (2 * iters)
     gbs = nbytes / (ms * 1e-3) / 1e9
-    del H2
-    return {"ms_per_call": ms, "us_per_prompt": ms * 1e3 / len(step.prefill_ids), "gbs": gbs,
+
+    # What the kernel before the router leaves behind: one call between its own event pair, after a kernel that
+    # WROTE 512 MB (its last lines sit dirty in L2 and go to DRAM while the router reads, as the y tiles of the
+    # prefill apply do inside the step) and after a kernel that only READ 512 MB (nothing to write back).
+    scratch = torch.empty(256 << 20, dtype=torch.bfloat16, device=device)
+
+    def single(before):
+        total = 0.0
+        for k in range(8):
+            before()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            ml.route(0, step.H if k % 2 else H2, step.cu_p, step.slots_p)
+            a1.record()
+            torch.cuda.synchronize(device)
+            total += a0.elapsed_time(a1)
+        return total / 8 * 1e3
+
+    after_write_us = single(lambda: scratch.fill_(1.0))
+    after_read_us = single(lambda: scratch.max())
+    del H2, scratch
+    return {"ms_per_call": ms, "single_call_after_512MB_written_us": after_write_us,
+            "single_call_after_512MB_read_us": after_read_us, "us_per_prompt": ms * 1e3 / len(step.prefill_ids), "gbs": gbs,
             "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS, "calls": 2 * iters}
 
 
