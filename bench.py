@@ -897,7 +897,7 @@ def run_decode_sweep(device, peaks, batches=(1, 4, 16, 64, 128, 256), n_layers=8
         out.append({"batch": b, "us_per_layer": r["us_per_layer_launch"], "gbs": r["gbs"],
                     "frac_of_measured_hbm": r["frac_of_measured_hbm"],
                     "algorithmic_bytes_per_layer": r["algorithmic_bytes_per_layer"],
-                    "chosen": "split" if lw.ml.decode_path_for(b, b) == 2 else "cluster",
+                    "chosen": {1: "cluster", 2: "split", 3: "stream"}[lw.ml.decode_path_for(b, b)],
                     "us_per_layer_by_path": {k: v["us_per_layer"] for k, v in r["by_decode_path"].items()},
                     "one_call_all_layers": r["one_call_all_layers"],
                     "device_error_flag": r["device_error_flag"]})

@@ -263,9 +263,9 @@ milora_status milora_apply_prefill(milora_ctx* ctx, int layer, int module, const
  *                          second launch takes them as bf16 value + bf16 remainder, i.e. to 2^-17), which the first call (and any call with a larger
  *                          batch than every earlier one) grows with cudaMalloc after a stream sync.  Highest
  *                          bandwidth when the step's adapters exceed what one wave of clusters covers.
- *   MILORA_DECODE_AUTO     (default) SPLIT when the work list has room for more than two jobs per SM (on a B200:
- *                          decode batches from about 240 requests, and every batch that mixes prompts with
- *                          decode rows), else CLUSTER.
+ *   MILORA_DECODE_AUTO     (default) STREAM for batches of 96 sequences or more where the context allows it (see
+ *                          STREAM); otherwise SPLIT when the work list has room for more than two jobs per SM (on
+ *                          a B200: every smaller batch that mixes prompts with decode rows), else CLUSTER.
  *   MILORA_DECODE_STREAM   one persistent launch (one CTA per SM) whose warps each stream pieces of the adapters'
  *                          operand images through their own ring of shared-memory buffers (cp.async.bulk) and
  *                          contract them on mma.sync tiles; x W^A goes from its producers to the consumers of W^B

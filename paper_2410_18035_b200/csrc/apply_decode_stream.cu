@@ -503,6 +503,32 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
   __syncthreads();
   pdl_wait();
 
+  // Layer records and the first job of every (layer, module): every thread of the CTA takes a share, so that the
+  // look-ups of a 32-layer call (two dependent loads each) run side by side instead of one warp's eight rounds.
+  {
+    const int L = a.n_layers;
+    const uint4* src = reinterpret_cast<const uint4*>(a.layers);
+    uint4* dst = reinterpret_cast<uint4*>(sm.layers);
+    if (a.layers) {
+      for (int i = tid; i < L * (int)(sizeof(StreamLayer) / 16); i += SH::kThreads) dst[i] = src[i];
+    } else if (tid == 0) {
+      sm.layers[0] = a.one;
+    }
+    if (tid < MILORA_NMOD) {
+      const int ss = (a.d1[tid] + a.cols - 1) / a.cols, se = (a.d2[tid] + a.cols - 1) / a.cols;
+      sm.upj[0][tid] = (ss + a.unit_stages - 1) / a.unit_stages;
+      sm.upj[1][tid] = (se + a.unit_stages - 1) / a.unit_stages;
+    }
+    __syncthreads();
+    for (int i = tid; i < L * (MILORA_NMOD + 1); i += SH::kThreads) {
+      const int li = i / (MILORA_NMOD + 1), m = i % (MILORA_NMOD + 1);
+      const StreamLayer& Ly = sm.layers[li];
+      const int n_jobs = max(0, min(Ly.ws[Ly.off_header + H_NGATHER], Ly.max_gather));
+      sm.first[li][m] = max(0, min(Ly.ws[Ly.off_mod_gather + m], n_jobs));
+    }
+    __syncthreads();
+  }
+
   if (warp >= kWarps) {
     // ================= scheduler =================
     const int sched = warp - kWarps;
@@ -510,29 +536,6 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
     const int L = a.n_layers;
     const int n_seg = 2 * L * MILORA_NMOD;
     if (sched == 0) {
-    // layer records and the unit table
-    {
-      const uint4* src = reinterpret_cast<const uint4*>(a.layers);
-      uint4* dst = reinterpret_cast<uint4*>(sm.layers);
-      if (a.layers) {
-        for (int i = lane; i < L * (int)(sizeof(StreamLayer) / 16); i += 32) dst[i] = src[i];
-      } else if (lane == 0) {
-        sm.layers[0] = a.one;
-      }
-      if (lane < MILORA_NMOD) {
-        const int ss = (a.d1[lane] + a.cols - 1) / a.cols, se = (a.d2[lane] + a.cols - 1) / a.cols;
-        sm.upj[0][lane] = (ss + a.unit_stages - 1) / a.unit_stages;
-        sm.upj[1][lane] = (se + a.unit_stages - 1) / a.unit_stages;
-      }
-    }
-    __syncwarp();
-    for (int i = lane; i < L * (MILORA_NMOD + 1); i += 32) {
-      const int li = i / (MILORA_NMOD + 1), m = i % (MILORA_NMOD + 1);
-      const StreamLayer& Ly = sm.layers[li];
-      const int n_jobs = max(0, min(Ly.ws[Ly.off_header + H_NGATHER], Ly.max_gather));
-      sm.first[li][m] = max(0, min(Ly.ws[Ly.off_mod_gather + m], n_jobs));
-    }
-    __syncwarp();
     {
       // unit counts per (queue position, module), then their prefix sums, 32 entries per pass
       int carry = 0;
@@ -794,10 +797,14 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
   const int workers = ctx->sm_count * n_warps;
   int us = ctx->stream_unit_stages;
   if (us < 1) {
-    // enough units that every worker gets several; long units save partial sums and look-ups
+    // A unit costs its worker's scheduler lane a round (locate, fetch and decode the job record) and the job a
+    // partial sum, so units are several stages long as soon as there are stages enough for every worker: single
+    // stages while there is less than one per worker, four as a rule, eight where a worker gets 6 to 25 stages in
+    // all (measured on 1 to 32 layers of the 7B shapes at 64 rows: 4-stage units are best at 1, 2, 16 and 32 layers,
+    // 8-stage units at 4, 8 and 12, where every worker then gets its units by index without asking the counter).
     const double est = stages_per_job * std::max(1, n_seq_hint) * std::min(n_layers, kMaxStreamLayers);
-    us = (int)(est / (workers * 4.0));
-    us = std::max(1, std::min(us, 4));
+    const double per_worker = est / workers;
+    us = per_worker < 1.0 ? 1 : (per_worker < 2.0 ? 2 : ((per_worker >= 6.0 && per_worker < 26.0) ? 8 : 4));
   }
   a.unit_stages = us;
   int kcmax = 1;

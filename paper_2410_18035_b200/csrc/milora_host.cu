@@ -583,6 +583,10 @@ milora_status milora_group(milora_ctx* ctx, int layer_begin, int n_layers, const
 static milora_decode_path pick_decode_path(const milora_ctx* ctx, int n_seq, int T) {
   if (ctx->decode_path == MILORA_DECODE_STREAM && !decode_stream_supported(ctx)) return MILORA_DECODE_CLUSTER;
   if (ctx->decode_path != MILORA_DECODE_AUTO) return (milora_decode_path)ctx->decode_path;
+  // One layer per call, measured (8B and 13B shapes, rank 16 and 32): up to 64 sequences the cluster kernel is the
+  // quickest (12.9 against 15.7 us at 64), from 128 on the persistent kernel (20.1 against 21.6 us at 128, 30.2
+  // against 34.2 at 256, 40.9 against 49.8 on the 13B step).
+  if (n_seq >= 96 && decode_stream_supported(ctx)) return MILORA_DECODE_STREAM;
   const milora_group_layout_t lay = group_layout(n_seq, T, top_k_of(ctx));
   return lay.max_gather > 2 * ctx->sm_count ? MILORA_DECODE_SPLIT : MILORA_DECODE_CLUSTER;
 }

@@ -209,7 +209,8 @@ def test_config3_full_stack_ragged_prefill():
 def test_config4_full_stack_zipf_decode():
     """LLaMA-2-13B shapes, all 40 layers registered, rank 32, 256 decode requests whose tenants follow Zipf(1.1) over
     1000 ids (every drawn tenant gets backing: about 110 tenants x 40 layers x 7 adapters), 256-token prompts:
-    routes (40 x 256) and groupings on every layer, the gathered apply on four layers with the two-launch kernels,
+    routes (40 x 256) and groupings on every layer, the gathered apply on four layers with the library's own choice
+    (the persistent kernel), on one layer each with the other two kernel sets,
     and the whole stack in one milora_apply_decode_layers call."""
     w = get_workload("c4")
     w.gen_device = "cuda"
@@ -219,12 +220,12 @@ def test_config4_full_stack_zipf_decode():
     assert per_tenant * n_active < 0.8 * free, f"{n_active} tenants x {per_tenant >> 20} MB do not fit this device"
     lw = _loaded(w)
     ids = list(range(w.n_requests))
-    assert lw.ml.decode_path_for(len(ids), len(ids)) == 2       # a batch of this size takes the two-launch kernels
+    assert lw.ml.decode_path_for(len(ids), len(ids)) == 3       # a batch of this size takes the persistent kernel
     _full_stack(lw, [], ids, np.random.default_rng(2), max_excused=120, decode_path="auto")
     rng = np.random.default_rng(22)
     table = lw.ml.route_table_read(0, w.n_requests).numpy()
     _check_step(lw, 0, [], ids, table[:, 0], tag=1, rng=rng, decode_path="cluster")
-    _check_step(lw, 39, [], ids, table[:, 39], tag=2, rng=rng, decode_path="stream")
+    _check_step(lw, 39, [], ids, table[:, 39], tag=2, rng=rng, decode_path="split")
     lw.close()
 
 
