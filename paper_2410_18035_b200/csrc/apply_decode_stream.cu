@@ -194,6 +194,15 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ void locate_unit(const StreamArgs& a, Smem& sm, int n_seg, int u, int w, int slot, int* seg,
                                             UnitLoc* x) {
   int sg = *seg;
+  if (sg + 8 < n_seg && sm.seg_base[sg + 8] <= u) {
+    // far ahead (a lane's first units): last segment whose base is <= u, by bisection
+    int lo = sg + 8, hi = n_seg - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sm.seg_base[mid] <= u) lo = mid; else hi = mid - 1;
+    }
+    sg = lo;
+  }
   while (sg + 1 < n_seg && sm.seg_base[sg + 1] <= u) ++sg;
   *seg = sg;
   const int p = sg / MILORA_NMOD;
@@ -527,6 +536,17 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       sm.first[li][m] = max(0, min(Ly.ws[Ly.off_mod_gather + m], n_jobs));
     }
     __syncthreads();
+    // unit counts per (queue position, module), left where their prefix sums will stand
+    for (int i = tid; i < 2 * L * MILORA_NMOD; i += SH::kThreads) {
+      const int p = i / MILORA_NMOD, m = i % MILORA_NMOD;
+      int li, phase;
+      pos_to_layer(p, L, &li, &phase);
+      const StreamLayer& Ly = sm.layers[li];
+      int v = max(0, sm.first[li][m + 1] - sm.first[li][m]) * sm.upj[phase][m];
+      if (Ly.X[m] == nullptr || Ly.Y[m] == nullptr) v = 0;
+      sm.seg_base[i + 1] = v;
+    }
+    __syncthreads();
   }
 
   if (warp >= kWarps) {
@@ -537,20 +557,12 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
     const int n_seg = 2 * L * MILORA_NMOD;
     if (sched == 0) {
     {
-      // unit counts per (queue position, module), then their prefix sums, 32 entries per pass
+      // prefix sums of the unit counts, 32 entries per pass
       int carry = 0;
       if (lane == 0) sm.seg_base[0] = 0;
       for (int b = 0; b < n_seg; b += 32) {
         const int i = b + lane;
-        int v = 0;
-        if (i < n_seg) {
-          const int p = i / MILORA_NMOD, m = i % MILORA_NMOD;
-          int li, phase;
-          pos_to_layer(p, L, &li, &phase);
-          const StreamLayer& Ly = sm.layers[li];
-          v = max(0, sm.first[li][m + 1] - sm.first[li][m]) * sm.upj[phase][m];
-          if (Ly.X[m] == nullptr || Ly.Y[m] == nullptr) v = 0;
-        }
+        int v = i < n_seg ? sm.seg_base[i + 1] : 0;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const int t = __shfl_up_sync(0xffffffffu, v, o);
@@ -799,12 +811,11 @@ milora_status launch_apply_decode_stream(milora_ctx* ctx, StreamLayer* layers, i
   if (us < 1) {
     // A unit costs its worker's scheduler lane a round (locate, fetch and decode the job record) and the job a
     // partial sum, so units are several stages long as soon as there are stages enough for every worker: single
-    // stages while there is less than one per worker, four as a rule, eight where a worker gets 6 to 25 stages in
-    // all (measured on 1 to 32 layers of the 7B shapes at 64 rows: 4-stage units are best at 1, 2, 16 and 32 layers,
-    // 8-stage units at 4, 8 and 12, where every worker then gets its units by index without asking the counter).
+    // stages while there is less than one per worker, then two, four, and eight from six stages per worker on
+    // (measured on 1 to 32 layers of the 7B shapes at 64 rows and on the 13B shapes at 256).
     const double est = stages_per_job * std::max(1, n_seq_hint) * std::min(n_layers, kMaxStreamLayers);
     const double per_worker = est / workers;
-    us = per_worker < 1.0 ? 1 : (per_worker < 2.0 ? 2 : ((per_worker >= 6.0 && per_worker < 26.0) ? 8 : 4));
+    us = per_worker < 1.0 ? 1 : (per_worker < 2.0 ? 2 : (per_worker < 6.0 ? 4 : 8));
   }
   a.unit_stages = us;
   int kcmax = 1;
