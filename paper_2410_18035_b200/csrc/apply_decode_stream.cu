@@ -586,7 +586,12 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       const uint32_t buf0 = smem_u32(smem_raw) + (uint32_t)(w * kBufs) * a.buf_stride;
       int n_fetched = 0, n_located = 0, n_issued = 0, n_kept = 0, is = 0, seg = 0;
       bool dry = false, have_cur = false, stop_sent = false;
-      uint32_t next_dyn = atomicAdd(&a.ctrl[0], 1u);     // used by the third look-ahead; the answer has time to come
+      // How far a lane looks ahead decides what the workers still hold when the queue runs dry, i.e. how long the
+      // last of them works alone.  Short units (one or two stages, 2 to 4 us) need the full depth to hide the
+      // counter's and the record's round trips: two located units and one claimed number.  Long units give the
+      // lane time: one located unit, and the counter is asked when the number is needed.
+      const bool deep = a.unit_stages <= 2;
+      uint32_t next_dyn = deep ? atomicAdd(&a.ctrl[0], 1u) : 0u;     // used by the third look-ahead; the answer has time to come
       UnitLoc q0, q1;
       Unit cur;
       auto fetch_q1 = [&]() {
@@ -596,8 +601,12 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
         if (n_fetched < kStaticRounds) {
           u = wid + n_fetched * n_workers;
         } else {
-          u = kStaticRounds * n_workers + (int)next_dyn;
-          next_dyn = atomicAdd(&a.ctrl[0], 1u);          // for the call after this one
+          if (deep) {
+            u = kStaticRounds * n_workers + (int)next_dyn;
+            next_dyn = atomicAdd(&a.ctrl[0], 1u);        // for the call after this one
+          } else {
+            u = kStaticRounds * n_workers + (int)atomicAdd(&a.ctrl[0], 1u);
+          }
         }
         ++n_fetched;
         if (u >= total) { dry = true; return; }
@@ -606,7 +615,7 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
       };
       fetch_q1();
       q0 = q1;
-      fetch_q1();
+      if (deep) fetch_q1(); else q1.valid = false;
       uint32_t round = 0;
       for (; round < kSchedSpin && !stop_sent; ++round) {
         if (!have_cur && q0.valid) {
@@ -616,8 +625,14 @@ __global__ void __launch_bounds__(SH::kThreads, 1) decode_stream_kernel(StreamAr
           if (q1.valid) cp_async_wait<1>(); else cp_async_wait<0>();
           const bool ok = decode_unit(a, sm, q0, sm.rec[w][q0.slot], &cur, &sm.unit[w][slot]);
           if (!ok && q0.sub == 0 && q0.phase == 0) atomicOr(a.err, ERR_BAD_ITEM);
-          q0 = q1;
-          fetch_q1();
+          if (deep) {
+            q0 = q1;
+            fetch_q1();
+          } else {
+            fetch_q1();
+            q0 = q1;
+            q1.valid = false;
+          }
           if (ok) {
             have_cur = true;
             is = 0;
