@@ -330,8 +330,10 @@ milora_status launch_group(milora_ctx* ctx, int layer_begin, int n_layers, const
   if (smem > 48 * 1024) {
     MILORA_CUDA(ctx, cudaFuncSetAttribute(group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
-  // few sequences (a decode batch): a smaller block makes every barrier and scan cheaper
-  const int threads = std::max(128, std::min(kGMaxThreads, n_pad));
+  // few sequences (a decode batch): a smaller block makes every barrier and scan cheaper; many rows (prompts): perm is
+  // written by one warp per sequence, 32 rows per pass, and wants warps (32,768 rows: 3.9 us with 4 warps, 1 with 16)
+  int threads = std::max(128, std::min(kGMaxThreads, n_pad));
+  threads = std::max(threads, std::min(kGMaxThreads, (T / 64) & ~31));
   MILORA_CUDA(ctx, launch_pdl(group_kernel, dim3(n_layers), dim3(threads), smem, s, a));
   return MILORA_OK;
 }
