@@ -49,6 +49,11 @@ def test_status_strings(lib):
     lib.milora_decode_path_for.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
     assert lib.milora_set_decode_path(None, 2) == 1
     assert lib.milora_decode_path_for(None, 1, 1, None) == 1
+    lib.milora_apply_prefill_shared.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    assert lib.milora_apply_prefill_shared(None, 0, 1, None, None, None, None, None) == 1
+    lib.milora_apply_decode_layers.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    assert lib.milora_apply_decode_layers(None, None, 1, None) == 1
 
 
 def test_product_path_does_not_touch_the_oracle():

@@ -232,6 +232,20 @@ def test_top_k_routing_grouping_and_apply(dtype, d, d_ff, d_kv, r, k, gate):
                      shared=[(0, 1, 2), (4, 5)])
         # more siblings than one pass takes: five modules on one matrix
         _step_parity(lw, li, prefill, decode, table, tag=15, use_multi=True, gate=gate_arg, shared=[(5, 0, 4, 2, 1)])
+    # modules that do not have the same input width cannot share an input matrix
+    if dtype == "bf16":
+        import ctypes as C
+        from paper_2410_18035_b200 import MiloraError
+        cu_s, slots_s, T_s = lw.seq_arrays(prefill, [])
+        ws_s = lw.ml.alloc_group_ws(1, len(prefill), T_s)
+        lw.ml.group(0, 1, cu_s, slots_s, len(prefill), T_s, ws_s)
+        g_s = lw.ml.groups(ws_s[0], len(prefill), T_s)
+        Xq = w.module_input(lw.layers[0], 0, T_s, 16, "cuda")
+        Yq, Yd = w.base_output(lw.layers[0], 0, T_s, 16, "cuda"), w.base_output(lw.layers[0], 6, T_s, 16, "cuda")
+        mods = (C.c_int * 2)(0, 6)
+        ys = (C.c_void_p * 2)(Yq.data_ptr(), Yd.data_ptr())
+        st = lw.ml.lib.milora_apply_prefill_shared(lw.ml.h, 0, 2, mods, C.c_void_p(Xq.data_ptr()), ys, C.byref(g_s), None)
+        assert st == 1, "q and down read matrices of different widths: MILORA_E_ARG"
     # restoring a table by hand: duplicates inside a cell are refused
     from paper_2410_18035_b200 import MiloraError
     if k >= 2:
