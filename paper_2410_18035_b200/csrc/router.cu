@@ -347,6 +347,30 @@ struct BulkUnit {
 };
 
 __device__ __forceinline__ uint32_t bulk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// L2 policies: H is read once (evict first), the partial sums are read back by pass 2 some tens of microseconds
+// later, after 268 MB of H have gone through the 126 MB L2 (evict last; pass 2 reads them as evict first again).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z),
+               "f"(v.w), "l"(pol)
+               : "memory");
+}
+__device__ __forceinline__ float4 ld_f4_hint(const float* p, uint64_t pol) {
+  float4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(pol));
+  return v;
+}
 __device__ __forceinline__ bool bulk_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -426,6 +450,7 @@ __global__ void __launch_bounds__(kThreads + 32, 2) pool_bulk_kernel(RouteArgs a
   if (!worker) {
     // ---- copy warp: units from the counter (asked for one unit ahead), one stage of 16 row copies at a time,
     //      one lane per row; a stage is refilled as soon as the eight worker warps have handed it back ----
+    const uint64_t pol_h = l2_policy_evict_first();
     int u_next = blockIdx.x, n_queued = 0, g_issued = 0;
     uint32_t fetched = 0;
     bool gave_up = false;
@@ -466,10 +491,11 @@ __global__ void __launch_bounds__(kThreads + 32, 2) pool_bulk_kernel(RouteArgs a
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(rows * sb)) : "memory");
           __syncwarp();
           if (lane < rows)
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                             bulk_smem_u32(ring + st * kBulkStageBytes + lane * kBulkStrip)),
-                         "l"(un.src + (size_t)(r_first + lane) * row_bytes), "r"((uint32_t)sb), "r"(bar)
-                         : "memory");
+            asm volatile(
+                "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                    bulk_smem_u32(ring + st * kBulkStageBytes + lane * kBulkStrip)),
+                "l"(un.src + (size_t)(r_first + lane) * row_bytes), "r"((uint32_t)sb), "r"(bar), "l"(pol_h)
+                : "memory");
         }
       }
       u_next = (int)__shfl_sync(0xffffffffu, fetched, 0);
@@ -504,6 +530,7 @@ __global__ void __launch_bounds__(kThreads + 32, 2) pool_bulk_kernel(RouteArgs a
   }
   asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
   const int half = tid >> 7, l = tid & 127;
+  const uint64_t pol_part = l2_policy_evict_last();
   int g_done = 0;
   auto wait_full = [&](int n) {          // bounded wait for stage number n; a warp that gives up tells the others
     const uint32_t bar = bulk_smem_u32(&full[n % kBulkStages]), parity = (uint32_t)(n / kBulkStages) & 1u;
@@ -567,7 +594,7 @@ __global__ void __launch_bounds__(kThreads + 32, 2) pool_bulk_kernel(RouteArgs a
       for (int i = 0; i < V; ++i) acc[i] = is_max ? fmaxf(acc[i], red[l][i]) : acc[i] + red[l][i];
       float* dst = un.part + l * V;
 #pragma unroll
-      for (int i = 0; i < V; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+      for (int i = 0; i < V; i += 4) st_f4_hint(dst + i, make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]), pol_part);
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");      // red is reused by the next unit
     if (stop) break;
@@ -634,6 +661,7 @@ __global__ void __launch_bounds__(kFinThreads) route_finalize_kernel(RouteArgs a
   const float* part0 = a.partial + (size_t)chunk0 * d;
   const float* st0 = a.stats + 2 * (size_t)chunk0;
   pdl_wait();                                   // the partial sums of pass 1
+  const uint64_t pol_read = l2_policy_evict_first();
   float gmax = -FLT_MAX, denom = 1.f;
   if (sa) {
     for (int c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, st0[2 * c]);
@@ -658,7 +686,7 @@ __global__ void __launch_bounds__(kFinThreads) route_finalize_kernel(RouteArgs a
         wgt[k] = sa ? st0[2 * c] : 0.f;
 #pragma unroll
         for (int i = 0; i < V / 4; ++i)
-          q[k][i] = *reinterpret_cast<const float4*>(part0 + (size_t)c * d + c0 + 4 * i);
+          q[k][i] = ld_f4_hint(part0 + (size_t)c * d + c0 + 4 * i, pol_read);
       }
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
