@@ -163,11 +163,12 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_kernel(const __
     if (warp == 0 && lane == 0) {
       // ---- copies: X tile by TMA, A image chunk by one bulk copy ----
       const char* img = static_cast<const char*>(job.At_img);
+      const uint64_t pol_x = l2_evict_first_policy();      // x is read once; the A images are read again by other tiles
       for (int i = 0; i < nk; ++i) {
         const int s = i % kShrinkStages, ph = (i / kShrinkStages) & 1;
         if (i >= kShrinkStages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
         mbar_expect_tx(full(s), kXStage + rp * 128);
-        tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
+        tma_load_2d_hint(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s), pol_x);
         bulk_g2s(as + s * a_stage, img + (size_t)(kc0 + i) * rp * 128, rp * 128, full(s));
         issued = i + 1;
       }
@@ -346,12 +347,13 @@ __global__ void __launch_bounds__(kShrinkThreads) prefill_shrink_shared_kernel(c
   if (nk > 0) {
     if (warp == 0) {
       if (lane == 0) {
-        // ---- copies: the X tile once, one A image chunk per sibling ----
+        // ---- copies: the X tile once (read once: evict first), one A image chunk per sibling ----
+        const uint64_t pol_x = l2_evict_first_policy();
         for (int i = 0; i < nk; ++i) {
           const int s = i % stages, ph = (i / stages) & 1;
           if (i >= stages && !wait_bar(empty(s), ph ^ 1, abort_ptr, a.err)) break;
           mbar_expect_tx(full(s), kXStage + cols * 128);
-          tma_load_2d(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s));
+          tma_load_2d_hint(xs + s * kXStage, &a.xmap[si], (kc0 + i) * kBK, job.start, full(s), pol_x);
 #pragma unroll
           for (int m = 0; m < kMaxShare; ++m)
             if (m < n_mem)
@@ -485,11 +487,12 @@ __global__ void __launch_bounds__(kExpandThreads) prefill_expand_kernel(const __
   __syncthreads();
   const int row0 = job.start;
   int issued = 0;                       // copies started by this thread (the copy thread only)
+  const uint64_t pol_y = l2_evict_first_policy();       // y is read once; the B images are read again by other tiles
   auto issue_stage = [&](int i) {       // y tile (two 64-column boxes) and B image chunk of n chunk i
     const int s = i % kExpandStages;
     mbar_expect_tx(full(s), kYStage + rp * 256);
-    tma_load_2d(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s));
-    tma_load_2d(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s));
+    tma_load_2d_hint(ys + s * kYStage, &a.ymap[si], (nc0 + i) * kBN, row0, full(s), pol_y);
+    tma_load_2d_hint(ys + s * kYStage + kYStage / 2, &a.ymap[si], (nc0 + i) * kBN + 64, row0, full(s), pol_y);
     bulk_g2s(bs + s * b_stage, static_cast<const char*>(job.B_img) + (size_t)(nc0 + i) * rp * 256, rp * 256, full(s));
   };
   if (warp == 0) {
