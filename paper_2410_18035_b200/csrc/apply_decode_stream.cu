@@ -285,7 +285,9 @@ __device__ __forceinline__ void issue_stage(const StreamArgs& a, const Unit& un,
   const int n_rows = un.phase == 0 ? un.n : 0;
   // the arrive releases the words and the unit's record to the worker, whose wait on the barrier acquires them
   mbar_expect_tx(bar, bytes_img + (uint32_t)n_rows * bytes_row);
-  bulk_g2s(buf, un.img + (size_t)c_off * un.rp * 2, bytes_img, bar);
+  // the operand images are read once per launch: evict first, so that what the launch reads again (partial sums,
+  // fragments, job records, the rows of y it adds to) keeps its place in L2
+  bulk_g2s_hint(buf, un.img + (size_t)c_off * un.rp * 2, bytes_img, bar, l2_evict_first_policy());
   const uint32_t rstride = (uint32_t)a.cols * 2 + kRowPad;
   for (int t = 0; t < n_rows; ++t)
     bulk_g2s(buf + a.stage_bytes + t * rstride, un.x0 + ((size_t)un.rows[t] * un.d + c_off) * 2, bytes_row, bar);
