@@ -91,6 +91,31 @@ __device__ inline void block_sum(float (&v)[NV], float* smem /* [NV][NW] */) {
   }
 }
 
+// L2 policies: H is read once (evict first), the partial sums are read back by pass 2 some tens of microseconds
+// later, after 268 MB of H have gone through the 126 MB L2 (evict last; pass 2 reads them as evict first again).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z),
+               "f"(v.w), "l"(pol)
+               : "memory");
+}
+__device__ __forceinline__ float4 ld_f4_hint(const float* p, uint64_t pol) {
+  float4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(pol));
+  return v;
+}
+
 // 128-bit streaming load that the compiler keeps in program order with the other loads of a batch.
 __device__ __forceinline__ uint4 ldg16_stream(const void* p) {
   uint4 q;
@@ -199,6 +224,7 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = a.d;
   const T* H = static_cast<const T*>(a.H);
+  const uint64_t pol_part = l2_policy_evict_last();      // the partial sums stay in L2 for pass 2
   // Pass 2 reads the prompt lengths, slots and router table before its own wait; it may do so only once
   // everything ahead of this kernel has completed, so the trigger comes after the wait here.
   pdl_wait();
@@ -307,7 +333,7 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
         reduce_rows<T, kRedWeighted>(H + (size_t)r0 * d + c0, d, nr, u_sm, acc);
 #pragma unroll
         for (int i = 0; i < V; i += 4)
-          *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+          st_f4_hint(part + c0 + i, make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]), pol_part);
       }
       __syncwarp();
       continue;
@@ -320,7 +346,7 @@ __global__ void __launch_bounds__(kThreads) pool_partial_kernel(RouteArgs a) {
       else reduce_rows<T, kRedSum>(col, d, nr, u_sm, acc);
 #pragma unroll
       for (int i = 0; i < V; i += 4)
-        *reinterpret_cast<float4*>(part + c0 + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+        st_f4_hint(part + c0 + i, make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]), pol_part);
     }
   }
 }
@@ -347,30 +373,6 @@ struct BulkUnit {
 };
 
 __device__ __forceinline__ uint32_t bulk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// L2 policies: H is read once (evict first), the partial sums are read back by pass 2 some tens of microseconds
-// later, after 268 MB of H have gone through the 126 MB L2 (evict last; pass 2 reads them as evict first again).
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t pol) {
-  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z),
-               "f"(v.w), "l"(pol)
-               : "memory");
-}
-__device__ __forceinline__ float4 ld_f4_hint(const float* p, uint64_t pol) {
-  float4 v;
-  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "l"(p), "l"(pol));
-  return v;
-}
 __device__ __forceinline__ bool bulk_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
