@@ -41,6 +41,25 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def copy_bandwidth_here(device, nbytes=512 << 20, iters=10):
+    """A device-to-device copy of 512 MB timed in this process (read + written bytes per second, the convention of the
+    measured peak): context for the roofline fractions, whose denominator was measured on another box of the pool."""
+    a = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    b = torch.empty_like(a)
+    for _ in range(3):
+        b.copy_(a)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        b.copy_(a)
+    e1.record()
+    torch.cuda.synchronize(device)
+    ms = e0.elapsed_time(e1) / iters
+    del a, b
+    return 2.0 * nbytes / (ms * 1e-3) / 1e9
+
+
 KERNEL_SOURCES = {
     "router": ["router.cu"],
     "prefill_apply": ["apply_prefill_sm100.cu", "sm100_ptx.cuh"],
@@ -350,13 +369,15 @@ def run_ours(args, rank, world, device):
         "decode_apply": {"ms": decode_ms, "launches": 1, "bytes": work["decode_bytes"]},
     }
     traffic = recorded_traffic(w.name)
+    copy_here = copy_bandwidth_here(device)
     rooflines = {}
     for name, k in per_kernel.items():
         gbs = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
         rooflines[name] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": gbs / peaks["hbm_gbs"], "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
                            "peak_source": peaks["source"], "ms_per_step": k["ms"], "launches_per_step": k["launches"],
-                           "algorithmic_bytes_per_step": k["bytes"], "traffic": traffic.get(name)}
+                           "algorithmic_bytes_per_step": k["bytes"], "traffic": traffic.get(name),
+                           "copy_gbs_in_this_process": copy_here, "frac_of_copy_in_this_process": gbs / copy_here}
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
